@@ -1,0 +1,157 @@
+/*
+ * avsg.h - C ABI of the AVSG per-decode-step operator for NVIDIA B200 (sm_100a).
+ *
+ * For every request's top-K selected token ids of one decode iteration the
+ * operator (paper Sec. 3.1, Algorithm 4)
+ *   1. matches the ids against a device-resident KV buffer of S slots
+ *      (hit / miss, Eq. 1),
+ *   2. reserves slots for the misses under the lifetime policy (Algorithm 1
+ *      passes 1-3, Algorithm 3, CollectDead Eq. 12); the tokens of one
+ *      multi-token-prediction iteration are processed in order through one
+ *      shared table (Sec. 3.6),
+ *   3. copies only the missed KV rows from host memory into their slots, the
+ *      miss list being cut evenly over all SMs (Sec. 3.4, Eq. 6),
+ *   4. forgets speculative entries (ids >= verified length, end of Alg. 4),
+ * and returns the slot table that sparse attention reads.
+ *
+ * Conventions
+ *   - "table" = one persistent (request, layer) buffer with its state.
+ *   - Every function returns AVSG_OK (0) or a negative AVSG_E* code and never
+ *     throws, traps or aborts.  avsg_strerror() names a code.
+ *   - Pointers are marked HOST or DEVICE.  The library never takes ownership
+ *     of caller memory.  The context owns all state, the KV buffers and the
+ *     scratch it needs; everything is allocated in avsg_create().
+ *   - Calls on one context must not overlap in time (one stream at a time).
+ *   - Kernel-side problems (a bounded loop that ran out, an index out of
+ *     range) never fault: the kernel records a code in a status word that
+ *     avsg_stats(), avsg_export_state() and avsg_sync_status() report as
+ *     AVSG_EDEVICE_STATUS.
+ */
+#ifndef AVSG_H
+#define AVSG_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AVSG_OK              0
+#define AVSG_EINVAL         -1   /* bad argument                                        */
+#define AVSG_ENOMEM         -2   /* host or device allocation failed                    */
+#define AVSG_ECUDA          -3   /* a CUDA runtime call failed                          */
+#define AVSG_ECAPACITY      -4   /* buffer_slots < n_tokens * topk (Eq. 7 violated)     */
+#define AVSG_EDEVICE_STATUS -5   /* a kernel reported a problem in the status word      */
+#define AVSG_EUNSUPPORTED   -6   /* shape outside what this build supports              */
+
+/* How Stage Two moves the missed rows (Sec. 3.4; App. D strategies). */
+#define AVSG_XFER_SM_BALANCED   0u  /* miss list cut evenly over all SMs (the operator)  */
+#define AVSG_XFER_COPY_ENGINE   1u  /* comparator: miss list read back, one async copy
+                                       per run of consecutive rows on the copy engine    */
+#define AVSG_XFER_REQUEST_LEVEL 2u  /* comparator S1: one thread block per request       */
+#define AVSG_XFER_ALL_K         3u  /* comparator "KV offload": no reuse, all n_tokens*K
+                                       rows move; position (g,i) -> slot g*K+i           */
+
+typedef struct avsg_ctx avsg_ctx;   /* opaque */
+
+typedef struct {
+    uint32_t num_tables;     /* persistent tables, each with its own S-slot buffer      */
+    uint32_t buffer_slots;   /* S: power of two, 32 .. 8192                             */
+    uint32_t row_bytes;      /* bytes per KV row, multiple of 16                        */
+    uint32_t max_topk;       /* largest K of any step                                   */
+    uint32_t max_tokens;     /* largest N_q = N_mtp + 1; max_tokens*max_topk <= S (Eq. 7) */
+    int32_t  max_lifetime;   /* L in 1 .. 126 (paper default 16)                        */
+    uint32_t transfer_mode;  /* AVSG_XFER_*                                             */
+    int32_t  device;         /* CUDA device ordinal                                     */
+} avsg_config;
+
+typedef struct {
+    uint32_t        n;             /* tables taking part in this call (1 .. num_tables)  */
+    const uint32_t *table_ids;     /* HOST [n]   distinct, each < num_tables             */
+    uint32_t        n_tokens;      /* N_q of this call (<= max_tokens)                   */
+    uint32_t        topk;          /* K of this call (<= max_topk)                       */
+    const int32_t  *indices;       /* DEVICE [n][n_tokens][topk] selected ids; unique
+                                      within a token; negative = padding                 */
+    const void *const *kv_base;    /* HOST [n]   per table: base of its host KV, pinned
+                                      (cudaHostAlloc / cudaHostRegister) so the GPU can
+                                      read it in place; a device pointer also works      */
+    const uint64_t *row_stride;    /* HOST [n] bytes between host rows, multiple of 16;
+                                      NULL = row_bytes                                   */
+    const int32_t  *verified_len;  /* HOST [n]   N of Alg. 4: ids >= N are speculative   */
+    int32_t        *slots;         /* DEVICE out [n][n_tokens][topk]: slot per id,
+                                      -1 for padding                                     */
+    uint8_t        *hit;           /* DEVICE out [n][n_tokens][topk] 1 = hit, or NULL    */
+    int32_t        *miss_count;    /* DEVICE out [n][n_tokens] n_g per token, or NULL    */
+} avsg_step_args;
+
+typedef struct {
+    uint64_t steps;            /* avsg_step calls x tables                               */
+    uint64_t tokens;           /* query tokens processed                                 */
+    uint64_t hits, misses;     /* over all valid ids                                     */
+    uint64_t rows_copied;      /* rows moved host -> device                              */
+    uint64_t bytes_copied;     /* rows_copied * row_bytes                                */
+    uint64_t extra_decays;     /* unit decays beyond the pre-decay (Alg. 1 while-loop)   */
+    float    last_stage_one_us;/* device time of the last call's match+reserve kernels
+                                  and of its transfer; 0 unless timing is enabled        */
+    float    last_transfer_us;
+    uint64_t last_rows;        /* rows the last call moved                               */
+} avsg_stats_t;
+
+/* Allocates all state: tables empty and dead ("each request starts with an
+ * empty cache", App. E), buffers zeroed.  *out is set only on success. */
+int avsg_create(const avsg_config *cfg, avsg_ctx **out);
+int avsg_destroy(avsg_ctx *ctx);
+
+/* A request ended: its tables become empty and dead again.  HOST table_ids[n].
+ * Synchronous. */
+int avsg_reset(avsg_ctx *ctx, const uint32_t *table_ids, uint32_t n);
+
+/* One decode iteration for the listed tables (Algorithm 4), asynchronous on
+ * cuda_stream (a cudaStream_t; NULL = default stream).  When the stream has
+ * finished this call, buffer[table][slots[...]] holds host row x for every
+ * non-padding id x.  Host KV, indices and outputs must stay valid until then.
+ * Host arrays of the argument block are consumed before the call returns. */
+int avsg_step(avsg_ctx *ctx, const avsg_step_args *args, void *cuda_stream);
+
+/* Same, but indices / slots / hit / miss_count are HOST pointers (pinned for
+ * asynchrony); the library stages them through its own device buffers on the
+ * stream: one upload of the ids, one download per requested output. */
+int avsg_step_host(avsg_ctx *ctx, const avsg_step_args *args, void *cuda_stream);
+
+/* DEVICE base of a table's S rows of row_bytes (what attention gathers from). */
+int avsg_buffer(avsg_ctx *ctx, uint32_t table_id, void **d_rows);
+
+/* Waits for the device, then reports cumulative counters.  Returns
+ * AVSG_EDEVICE_STATUS (and still fills *out) if a kernel flagged a problem. */
+int avsg_stats(avsg_ctx *ctx, avsg_stats_t *out);
+
+/* Waits for the device; returns AVSG_EDEVICE_STATUS if a kernel flagged a
+ * problem, and the raw status word in *status_word when not NULL. */
+int avsg_sync_status(avsg_ctx *ctx, uint32_t *status_word);
+
+/* Table state for checkpoints and parity checks.  HOST tok[S] (cached id per
+ * slot, -1 empty) and life[S] (lifetime, -1 dead).  Synchronous. */
+int avsg_export_state(avsg_ctx *ctx, uint32_t table_id, int32_t *tok, int8_t *life);
+int avsg_import_state(avsg_ctx *ctx, uint32_t table_id, const int32_t *tok, const int8_t *life);
+
+/* Device-side snapshot of every table's (tok, life) and its restore, both
+ * asynchronous on the stream: lets a measurement replay one step many times. */
+int avsg_save_state(avsg_ctx *ctx, void *cuda_stream);
+int avsg_restore_state(avsg_ctx *ctx, void *cuda_stream);
+
+/* Switches the Stage Two strategy of later calls (AVSG_XFER_*). */
+int avsg_set_transfer_mode(avsg_ctx *ctx, uint32_t mode);
+
+/* enable != 0: later calls record CUDA events around Stage One and Stage Two;
+ * avsg_stats() then reports the last call's device times. */
+int avsg_set_timing(avsg_ctx *ctx, int enable);
+
+/* Stage Two geometry: thread blocks (0 = one per SM) and threads per block. */
+int avsg_set_transfer_geometry(avsg_ctx *ctx, uint32_t blocks, uint32_t threads);
+
+const char *avsg_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AVSG_H */

@@ -1,0 +1,271 @@
+"""Thin ctypes binding of libavsg.so: argument marshalling only.
+
+Every step of the operator runs in the CUDA kernels behind the C ABI
+(include/avsg.h).  PyTorch supplies device tensors, pinned host tensors and
+streams.  If the library is missing the import of this module still works, but
+any use raises: there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Union
+
+import numpy as np
+
+from . import build as _build
+
+OK, EINVAL, ENOMEM, ECUDA, ECAPACITY, EDEVICE_STATUS, EUNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
+XFER_SM_BALANCED, XFER_COPY_ENGINE, XFER_REQUEST_LEVEL, XFER_ALL_K = 0, 1, 2, 3
+
+EXPORTS = (
+    "avsg_create", "avsg_destroy", "avsg_reset", "avsg_step", "avsg_step_host", "avsg_buffer", "avsg_stats",
+    "avsg_sync_status", "avsg_export_state", "avsg_import_state", "avsg_save_state", "avsg_restore_state",
+    "avsg_set_transfer_mode", "avsg_set_timing", "avsg_set_transfer_geometry", "avsg_strerror",
+)
+
+
+class AvsgConfig(ctypes.Structure):
+    _fields_ = [("num_tables", ctypes.c_uint32), ("buffer_slots", ctypes.c_uint32), ("row_bytes", ctypes.c_uint32),
+                ("max_topk", ctypes.c_uint32), ("max_tokens", ctypes.c_uint32), ("max_lifetime", ctypes.c_int32),
+                ("transfer_mode", ctypes.c_uint32), ("device", ctypes.c_int32)]
+
+
+class AvsgStepArgs(ctypes.Structure):
+    _fields_ = [("n", ctypes.c_uint32), ("table_ids", ctypes.c_void_p), ("n_tokens", ctypes.c_uint32),
+                ("topk", ctypes.c_uint32), ("indices", ctypes.c_void_p), ("kv_base", ctypes.c_void_p),
+                ("row_stride", ctypes.c_void_p), ("verified_len", ctypes.c_void_p), ("slots", ctypes.c_void_p),
+                ("hit", ctypes.c_void_p), ("miss_count", ctypes.c_void_p)]
+
+
+class AvsgStats(ctypes.Structure):
+    _fields_ = [("steps", ctypes.c_uint64), ("tokens", ctypes.c_uint64), ("hits", ctypes.c_uint64),
+                ("misses", ctypes.c_uint64), ("rows_copied", ctypes.c_uint64), ("bytes_copied", ctypes.c_uint64),
+                ("extra_decays", ctypes.c_uint64), ("last_stage_one_us", ctypes.c_float),
+                ("last_transfer_us", ctypes.c_float), ("last_rows", ctypes.c_uint64)]
+
+
+class AvsgError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__("%s (code %d)" % (what, code))
+        self.code = code
+
+
+_lib = None
+
+
+def load_library():
+    """Loads libavsg.so (built in-tree by build.build_library); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_build.LIB):
+        raise RuntimeError("libavsg.so is missing: run `python __graft_entry__.py` (needs nvcc) to build it; "
+                           "there is no CPU fallback")
+    lib = ctypes.CDLL(_build.LIB)
+    vp, u32, i32 = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_int
+    lib.avsg_create.argtypes, lib.avsg_create.restype = [ctypes.POINTER(AvsgConfig), ctypes.POINTER(vp)], i32
+    lib.avsg_destroy.argtypes, lib.avsg_destroy.restype = [vp], i32
+    lib.avsg_reset.argtypes, lib.avsg_reset.restype = [vp, vp, u32], i32
+    lib.avsg_step.argtypes, lib.avsg_step.restype = [vp, ctypes.POINTER(AvsgStepArgs), vp], i32
+    lib.avsg_step_host.argtypes, lib.avsg_step_host.restype = [vp, ctypes.POINTER(AvsgStepArgs), vp], i32
+    lib.avsg_buffer.argtypes, lib.avsg_buffer.restype = [vp, u32, ctypes.POINTER(vp)], i32
+    lib.avsg_stats.argtypes, lib.avsg_stats.restype = [vp, ctypes.POINTER(AvsgStats)], i32
+    lib.avsg_sync_status.argtypes, lib.avsg_sync_status.restype = [vp, ctypes.POINTER(u32)], i32
+    lib.avsg_export_state.argtypes, lib.avsg_export_state.restype = [vp, u32, vp, vp], i32
+    lib.avsg_import_state.argtypes, lib.avsg_import_state.restype = [vp, u32, vp, vp], i32
+    lib.avsg_save_state.argtypes, lib.avsg_save_state.restype = [vp, vp], i32
+    lib.avsg_restore_state.argtypes, lib.avsg_restore_state.restype = [vp, vp], i32
+    lib.avsg_set_transfer_mode.argtypes, lib.avsg_set_transfer_mode.restype = [vp, u32], i32
+    lib.avsg_set_timing.argtypes, lib.avsg_set_timing.restype = [vp, i32], i32
+    lib.avsg_set_transfer_geometry.argtypes, lib.avsg_set_transfer_geometry.restype = [vp, u32, u32], i32
+    lib.avsg_strerror.argtypes, lib.avsg_strerror.restype = [i32], ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != OK:
+        raise AvsgError(rc, "%s: %s" % (what, load_library().avsg_strerror(rc).decode()))
+
+
+def pinned_empty(nbytes: int):
+    """Pinned (page-locked, device-mapped) host bytes for a table's host KV."""
+    import torch
+    return torch.empty(int(nbytes), dtype=torch.uint8, pin_memory=True)
+
+
+def _addr(x) -> int:
+    """Address of a torch tensor / numpy array, or an integer address itself."""
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return int(x.data_ptr())
+    if isinstance(x, np.ndarray):
+        return int(x.ctypes.data)
+    raise TypeError("expected a tensor, an array or an address, got %r" % type(x))
+
+
+def _stream_handle(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream or None
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+class _DevView:
+    """Wraps a raw device pointer so that torch can view it without a copy."""
+
+    def __init__(self, ptr: int, shape, typestr: str, owner):
+        self.__cuda_array_interface__ = {"shape": tuple(shape), "typestr": typestr, "data": (ptr, False),
+                                         "version": 3, "strides": None}
+        self._owner = owner
+
+
+class StepOutput:
+    __slots__ = ("slots", "hit", "miss_count")
+
+    def __init__(self, slots, hit, miss_count):
+        self.slots, self.hit, self.miss_count = slots, hit, miss_count
+
+
+class PreparedCall:
+    """The argument block of one recurring call (same tables, same host KV): built once, re-used per step."""
+
+    def __init__(self, ctx: "Context", table_ids: Sequence[int], kv: Sequence, n_tokens: int, topk: int,
+                 row_stride: Optional[Sequence[int]] = None):
+        n = len(table_ids)
+        assert len(kv) == n
+        self.ctx, self.n, self.n_tokens, self.topk = ctx, n, n_tokens, topk
+        self._keep = list(kv)
+        self._tids = (ctypes.c_uint32 * n)(*[int(t) for t in table_ids])
+        self._kv = (ctypes.c_void_p * n)(*[_addr(k) for k in kv])
+        self._stride = (ctypes.c_uint64 * n)(*[int(s) for s in row_stride]) if row_stride is not None else None
+        self._vlen = (ctypes.c_int32 * n)()
+        a = AvsgStepArgs()
+        a.n, a.n_tokens, a.topk = n, n_tokens, topk
+        a.table_ids = ctypes.addressof(self._tids)
+        a.kv_base = ctypes.addressof(self._kv)
+        a.row_stride = ctypes.addressof(self._stride) if self._stride is not None else None
+        a.verified_len = ctypes.addressof(self._vlen)
+        self.args = a
+
+    def run(self, indices, verified_len: Sequence[int], slots, hit=None, miss_count=None, stream=None,
+            host: bool = False) -> None:
+        """indices / slots / hit / miss_count: tensors (device, or pinned host when host=True) or addresses."""
+        self._vlen[:] = [int(v) for v in verified_len]
+        a = self.args
+        a.indices, a.slots = _addr(indices), _addr(slots)
+        a.hit = _addr(hit) if hit is not None else None
+        a.miss_count = _addr(miss_count) if miss_count is not None else None
+        lib = self.ctx._lib
+        fn = lib.avsg_step_host if host else lib.avsg_step
+        _check(fn(self.ctx._h, ctypes.byref(a), _stream_handle(stream)), "avsg_step")
+
+
+class Context:
+    """Owns the device state of num_tables tables (see avsg_create)."""
+
+    def __init__(self, num_tables: int, buffer_slots: int, row_bytes: int, max_topk: int, max_tokens: int = 1,
+                 max_lifetime: int = 16, transfer_mode: int = XFER_SM_BALANCED, device: int = 0):
+        self._lib = load_library()
+        self._h = ctypes.c_void_p()
+        cfg = AvsgConfig(num_tables, buffer_slots, row_bytes, max_topk, max_tokens, max_lifetime, transfer_mode,
+                         device)
+        _check(self._lib.avsg_create(ctypes.byref(cfg), ctypes.byref(self._h)), "avsg_create")
+        self.num_tables, self.S, self.row_bytes = num_tables, buffer_slots, row_bytes
+        self.max_topk, self.max_tokens, self.L, self.device = max_topk, max_tokens, max_lifetime, device
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            self._lib.avsg_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the hot call ---------------------------------------------------------------------------------
+    def prepare(self, table_ids, kv, n_tokens: int, topk: int, row_stride=None) -> PreparedCall:
+        return PreparedCall(self, table_ids, kv, n_tokens, topk, row_stride)
+
+    def step(self, table_ids, indices, kv, verified_len, row_stride=None, want_hit: bool = True,
+             want_miss_count: bool = True, stream=None) -> StepOutput:
+        """One decode iteration. indices: int32 CUDA tensor [n, n_tokens, topk]. Returns device tensors."""
+        import torch
+        assert indices.is_cuda and indices.dtype == torch.int32 and indices.is_contiguous() and indices.dim() == 3
+        n, n_q, K = indices.shape
+        call = PreparedCall(self, table_ids, kv, n_q, K, row_stride)
+        slots = torch.empty_like(indices)
+        hit = torch.empty(indices.shape, dtype=torch.uint8, device=indices.device) if want_hit else None
+        mc = torch.empty((n, n_q), dtype=torch.int32, device=indices.device) if want_miss_count else None
+        call.run(indices, verified_len, slots, hit, mc, stream)
+        return StepOutput(slots, hit, mc)
+
+    def step_host(self, table_ids, indices, kv, verified_len, row_stride=None, want_hit: bool = True,
+                  want_miss_count: bool = True, stream=None) -> StepOutput:
+        """Same with host tensors in and out (pinned for asynchrony); returns pinned host tensors."""
+        import torch
+        assert not indices.is_cuda and indices.dtype == torch.int32 and indices.is_contiguous() and indices.dim() == 3
+        n, n_q, K = indices.shape
+        call = PreparedCall(self, table_ids, kv, n_q, K, row_stride)
+        slots = torch.empty(indices.shape, dtype=torch.int32, pin_memory=True)
+        hit = torch.empty(indices.shape, dtype=torch.uint8, pin_memory=True) if want_hit else None
+        mc = torch.empty((n, n_q), dtype=torch.int32, pin_memory=True) if want_miss_count else None
+        call.run(indices, verified_len, slots, hit, mc, stream, host=True)
+        return StepOutput(slots, hit, mc)
+
+    # -- state ----------------------------------------------------------------------------------------
+    def reset(self, table_ids: Sequence[int]) -> None:
+        ids = (ctypes.c_uint32 * len(table_ids))(*[int(t) for t in table_ids])
+        _check(self._lib.avsg_reset(self._h, ids, len(table_ids)), "avsg_reset")
+
+    def buffer(self, table_id: int):
+        """The table's S rows as a uint8 CUDA tensor [S, row_bytes] (a view, no copy)."""
+        import torch
+        p = ctypes.c_void_p()
+        _check(self._lib.avsg_buffer(self._h, table_id, ctypes.byref(p)), "avsg_buffer")
+        return torch.as_tensor(_DevView(p.value, (self.S, self.row_bytes), "|u1", self),
+                               device="cuda:%d" % self.device)
+
+    def export_state(self, table_id: int):
+        tok = np.empty(self.S, np.int32)
+        life = np.empty(self.S, np.int8)
+        _check(self._lib.avsg_export_state(self._h, table_id, tok.ctypes.data, life.ctypes.data), "avsg_export_state")
+        return tok, life
+
+    def import_state(self, table_id: int, tok, life) -> None:
+        tok = np.ascontiguousarray(tok, dtype=np.int32)
+        life = np.ascontiguousarray(life, dtype=np.int8)
+        assert tok.size == self.S and life.size == self.S
+        _check(self._lib.avsg_import_state(self._h, table_id, tok.ctypes.data, life.ctypes.data), "avsg_import_state")
+
+    def save_state(self, stream=None) -> None:
+        _check(self._lib.avsg_save_state(self._h, _stream_handle(stream)), "avsg_save_state")
+
+    def restore_state(self, stream=None) -> None:
+        _check(self._lib.avsg_restore_state(self._h, _stream_handle(stream)), "avsg_restore_state")
+
+    # -- knobs and counters ---------------------------------------------------------------------------
+    def set_transfer_mode(self, mode: int) -> None:
+        _check(self._lib.avsg_set_transfer_mode(self._h, mode), "avsg_set_transfer_mode")
+
+    def set_timing(self, enable: bool) -> None:
+        _check(self._lib.avsg_set_timing(self._h, int(enable)), "avsg_set_timing")
+
+    def set_transfer_geometry(self, blocks: int, threads: int) -> None:
+        _check(self._lib.avsg_set_transfer_geometry(self._h, blocks, threads), "avsg_set_transfer_geometry")
+
+    def sync_status(self) -> int:
+        w = ctypes.c_uint32(0)
+        _check(self._lib.avsg_sync_status(self._h, ctypes.byref(w)), "avsg_sync_status")
+        return w.value
+
+    def stats(self) -> dict:
+        s = AvsgStats()
+        _check(self._lib.avsg_stats(self._h, ctypes.byref(s)), "avsg_stats")
+        return {name: getattr(s, name) for name, _ in AvsgStats._fields_}

@@ -1,0 +1,465 @@
+// C ABI of the AVSG decode-step operator (see include/avsg.h): argument
+// checking, device state, kernel launches.  No step of the operator runs on
+// the host; there is no CPU fallback.
+#include <new>
+#include <string.h>
+#include <vector>
+
+#include "avsg.h"
+#include "avsg_kernels.cuh"
+
+using namespace avsg;
+
+struct avsg_ctx {
+    avsg_config cfg;
+    uint32_t logS = 0, logH = 0;
+    uint32_t list_stride = 0;          // entries per miss-list segment
+    int sm_count = 0;
+    uint32_t xfer_blocks = 0, xfer_threads = 256;
+    bool timing = false, events_recorded = false;
+
+    int32_t* d_tok = nullptr;
+    int8_t* d_life = nullptr;
+    uint8_t* d_buffer = nullptr;
+    TableStats* d_stats = nullptr;
+    int2* d_list = nullptr;
+    SegDesc* d_seg = nullptr;
+    uint32_t* d_status = nullptr;
+    int32_t* d_tok_snap = nullptr;
+    int8_t* d_life_snap = nullptr;
+    // staging of avsg_step_host
+    int32_t* d_idx_stage = nullptr;
+    int32_t* d_slots_stage = nullptr;
+    uint8_t* d_hit_stage = nullptr;
+    int32_t* d_mc_stage = nullptr;
+    // copy-engine comparator (pinned host copies of the miss list)
+    SegDesc* h_seg = nullptr;
+    int2* h_list = nullptr;
+
+    std::vector<uint64_t> kv_host, kv_dev;     // last validated host KV base per table
+    std::vector<uint32_t> seen;                // distinctness check of table ids
+    uint32_t epoch = 0;
+    std::vector<const void*> call_kv_host;     // host pointers of the current call (copy-engine mode)
+    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+    uint64_t last_rows = 0;
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+#define CU(call) do { if ((call) != cudaSuccess) return AVSG_ECUDA; } while (0)
+
+bool is_pow2(uint32_t v) { return v && !(v & (v - 1)); }
+uint32_t ilog2(uint32_t v) { uint32_t l = 0; while ((1u << l) < v) ++l; return l; }
+
+void free_all(avsg_ctx* c)
+{
+    cudaFree(c->d_tok); cudaFree(c->d_life); cudaFree(c->d_buffer); cudaFree(c->d_stats);
+    cudaFree(c->d_list); cudaFree(c->d_seg); cudaFree(c->d_status);
+    cudaFree(c->d_tok_snap); cudaFree(c->d_life_snap);
+    cudaFree(c->d_idx_stage); cudaFree(c->d_slots_stage); cudaFree(c->d_hit_stage); cudaFree(c->d_mc_stage);
+    if (c->h_seg) cudaFreeHost(c->h_seg);
+    if (c->h_list) cudaFreeHost(c->h_list);
+    for (auto& e : c->ev) if (e) cudaEventDestroy(e);
+}
+
+int init_tables(avsg_ctx* c, uint32_t first, uint32_t n)
+{
+    const size_t S = c->cfg.buffer_slots;
+    CU(cudaMemset(c->d_tok + first * S, 0xFF, n * S * sizeof(int32_t)));        // id -1: empty
+    CU(cudaMemset(c->d_life + first * S, 0xFF, n * S));                         // lifetime -1: dead
+    CU(cudaMemset(c->d_buffer + first * S * c->cfg.row_bytes, 0, n * S * c->cfg.row_bytes));
+    CU(cudaMemset(c->d_stats + first, 0, n * sizeof(TableStats)));
+    return AVSG_OK;
+}
+
+// Device-visible address of a host KV base (pinned + mapped host memory, or device memory).
+int resolve_kv(avsg_ctx* c, uint32_t table, const void* host_ptr, uint64_t* dev)
+{
+    const uint64_t h = reinterpret_cast<uint64_t>(host_ptr);
+    if (c->kv_host[table] == h && c->kv_dev[table]) { *dev = c->kv_dev[table]; return AVSG_OK; }
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host_ptr) != cudaSuccess) { cudaGetLastError(); return AVSG_EINVAL; }
+    if (at.type == cudaMemoryTypeUnregistered || at.devicePointer == nullptr) return AVSG_EINVAL;
+    c->kv_host[table] = h;
+    c->kv_dev[table] = reinterpret_cast<uint64_t>(at.devicePointer);
+    *dev = c->kv_dev[table];
+    return AVSG_OK;
+}
+
+int check_args(avsg_ctx* c, const avsg_step_args* a)
+{
+    if (!c || !a) return AVSG_EINVAL;
+    if (a->n == 0 || a->n > c->cfg.num_tables || a->n > (uint32_t)XFER_MAX_SEG) return AVSG_EINVAL;
+    if (!a->table_ids || !a->indices || !a->kv_base || !a->verified_len || !a->slots) return AVSG_EINVAL;
+    if (a->n_tokens == 0 || a->n_tokens > c->cfg.max_tokens || a->topk == 0 || a->topk > c->cfg.max_topk)
+        return AVSG_EINVAL;
+    if ((uint64_t)a->n_tokens * a->topk > c->cfg.buffer_slots) return AVSG_ECAPACITY;      // Eq. 7
+    if (++c->epoch == 0) { std::fill(c->seen.begin(), c->seen.end(), 0u); c->epoch = 1; }
+    for (uint32_t i = 0; i < a->n; ++i) {
+        const uint32_t t = a->table_ids[i];
+        if (t >= c->cfg.num_tables || c->seen[t] == c->epoch) return AVSG_EINVAL;
+        c->seen[t] = c->epoch;
+        if (a->row_stride && (a->row_stride[i] % 16 || a->row_stride[i] < c->cfg.row_bytes)) return AVSG_EINVAL;
+        if (!a->kv_base[i] || (reinterpret_cast<uint64_t>(a->kv_base[i]) & 15u)) return AVSG_EINVAL;
+    }
+    return AVSG_OK;
+}
+
+// Comparator: the miss list goes back to the host, then one asynchronous copy per run of
+// consecutive (host row, slot) pairs is queued on the copy engine.
+int copy_engine_transfer(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream)
+{
+    const uint32_t n = a->n;
+    CU(cudaMemcpyAsync(c->h_seg, c->d_seg, n * sizeof(SegDesc), cudaMemcpyDeviceToHost, stream));
+    CU(cudaStreamSynchronize(stream));
+    uint32_t max_count = 0;
+    for (uint32_t i = 0; i < n; ++i) max_count = c->h_seg[i].count > max_count ? c->h_seg[i].count : max_count;
+    if (max_count == 0) return AVSG_OK;
+    if (max_count > c->list_stride) return AVSG_EDEVICE_STATUS;
+    const size_t pitch = (size_t)c->list_stride * sizeof(int2);
+    CU(cudaMemcpy2DAsync(c->h_list, pitch, c->d_list, pitch, (size_t)max_count * sizeof(int2), n,
+                         cudaMemcpyDeviceToHost, stream));
+    CU(cudaStreamSynchronize(stream));
+    const uint64_t rb = c->cfg.row_bytes;
+    for (uint32_t i = 0; i < n; ++i) {
+        const SegDesc& sd = c->h_seg[i];
+        const int2* e = c->h_list + (size_t)i * c->list_stride;
+        const uint8_t* src_base = static_cast<const uint8_t*>(c->call_kv_host[i]);
+        uint32_t k = 0;
+        while (k < sd.count) {
+            if (e[k].x < 0 || e[k].y < 0 || (uint32_t)e[k].y >= c->cfg.buffer_slots) { ++k; continue; }
+            uint32_t run = 1;
+            if (sd.src_stride == rb)
+                while (k + run < sd.count && e[k + run].x == e[k].x + (int32_t)run && e[k + run].y == e[k].y + (int32_t)run) ++run;
+            CU(cudaMemcpyAsync(reinterpret_cast<void*>(sd.dst_base + (uint64_t)e[k].y * rb),
+                               src_base + (uint64_t)e[k].x * sd.src_stride, run * rb, cudaMemcpyDefault, stream));
+            k += run;
+        }
+    }
+    return AVSG_OK;
+}
+
+int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool host_io)
+{
+    int rc = check_args(c, a);
+    if (rc != AVSG_OK) return rc;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return AVSG_ECUDA;
+
+    const uint32_t n = a->n, K = a->topk, n_q = a->n_tokens;
+    const size_t n_ids = (size_t)n * n_q * K;
+    const int32_t* indices = a->indices;
+    int32_t* slots = a->slots;
+    uint8_t* hit = a->hit;
+    int32_t* miss_count = a->miss_count;
+    if (host_io) {
+        CU(cudaMemcpyAsync(c->d_idx_stage, a->indices, n_ids * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+        indices = c->d_idx_stage;
+        slots = c->d_slots_stage;
+        hit = a->hit ? c->d_hit_stage : nullptr;
+        miss_count = a->miss_count ? c->d_mc_stage : nullptr;
+    }
+    if (c->timing) CU(cudaEventRecord(c->ev[0], stream));
+
+    const uint32_t mode = c->cfg.transfer_mode;
+    c->call_kv_host.assign(a->kv_base, a->kv_base + n);
+    for (uint32_t first = 0; first < n; first += S1_MAX_TABLES) {
+        const uint32_t cnt = n - first < (uint32_t)S1_MAX_TABLES ? n - first : (uint32_t)S1_MAX_TABLES;
+        if (mode == AVSG_XFER_ALL_K) {
+            AllKParams p;
+            p.indices = indices; p.slots = slots; p.hit = hit; p.miss_count = miss_count;
+            p.miss_list = c->d_list; p.seg = c->d_seg; p.stats = c->d_stats; p.buffer = c->d_buffer;
+            p.S = c->cfg.buffer_slots; p.row_bytes = c->cfg.row_bytes; p.K = K; p.n_q = n_q;
+            p.first = first; p.list_stride = c->list_stride;
+            for (uint32_t i = 0; i < cnt; ++i) {
+                p.table_id[i] = a->table_ids[first + i];
+                if ((rc = resolve_kv(c, p.table_id[i], a->kv_base[first + i], &p.kv_base[i])) != AVSG_OK) return rc;
+                p.kv_stride[i] = a->row_stride ? a->row_stride[first + i] : c->cfg.row_bytes;
+            }
+            CU(launch_all_k_prepare(p, cnt, stream));
+        } else {
+            S1Params p;
+            p.tok = c->d_tok; p.life = c->d_life; p.buffer = c->d_buffer; p.stats = c->d_stats;
+            p.miss_list = c->d_list; p.seg = c->d_seg; p.status = c->d_status;
+            p.indices = indices; p.slots = slots; p.hit = hit; p.miss_count = miss_count;
+            p.S = c->cfg.buffer_slots; p.logH = c->logH; p.row_bytes = c->cfg.row_bytes;
+            p.K = K; p.n_q = n_q; p.L = (uint32_t)c->cfg.max_lifetime;
+            p.first = first; p.list_stride = c->list_stride;
+            for (uint32_t i = 0; i < cnt; ++i) {
+                p.table_id[i] = a->table_ids[first + i];
+                p.verified_len[i] = a->verified_len[first + i];
+                if ((rc = resolve_kv(c, p.table_id[i], a->kv_base[first + i], &p.kv_base[i])) != AVSG_OK) return rc;
+                p.kv_stride[i] = a->row_stride ? a->row_stride[first + i] : c->cfg.row_bytes;
+            }
+            CU(launch_stage_one(p, cnt, stream));
+        }
+    }
+    if (c->timing) CU(cudaEventRecord(c->ev[1], stream));
+
+    if (mode == AVSG_XFER_COPY_ENGINE) {
+        if ((rc = copy_engine_transfer(c, a, stream)) != AVSG_OK) return rc;
+    } else {
+        XferParams x;
+        x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
+        x.n_seg = n; x.list_stride = c->list_stride; x.row_bytes = c->cfg.row_bytes;
+        x.request_level = mode == AVSG_XFER_REQUEST_LEVEL; x.S = c->cfg.buffer_slots;
+        const uint32_t blocks = x.request_level ? n : (c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count);
+        CU(launch_transfer(x, blocks, c->xfer_threads, stream));
+    }
+    if (c->timing) { CU(cudaEventRecord(c->ev[2], stream)); c->events_recorded = true; }
+
+    if (host_io) {
+        CU(cudaMemcpyAsync(a->slots, c->d_slots_stage, n_ids * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+        if (a->hit) CU(cudaMemcpyAsync(a->hit, c->d_hit_stage, n_ids, cudaMemcpyDeviceToHost, stream));
+        if (a->miss_count)
+            CU(cudaMemcpyAsync(a->miss_count, c->d_mc_stage, (size_t)n * n_q * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    }
+    return AVSG_OK;
+}
+
+int read_status(avsg_ctx* c, uint32_t* word)
+{
+    uint32_t st = 0;
+    CU(cudaMemcpy(&st, c->d_status, sizeof(st), cudaMemcpyDeviceToHost));
+    if (word) *word = st;
+    return st ? AVSG_EDEVICE_STATUS : AVSG_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int avsg_create(const avsg_config* cfg, avsg_ctx** out)
+{
+    if (!cfg || !out) return AVSG_EINVAL;
+    if (cfg->num_tables == 0 || !is_pow2(cfg->buffer_slots) || cfg->buffer_slots < 32) return AVSG_EINVAL;
+    if (cfg->buffer_slots > 8192) return AVSG_EUNSUPPORTED;
+    if (cfg->row_bytes == 0 || cfg->row_bytes % 16) return AVSG_EINVAL;
+    if (cfg->max_topk == 0 || cfg->max_tokens == 0) return AVSG_EINVAL;
+    if (cfg->max_lifetime < 1 || cfg->max_lifetime > 126) return AVSG_EINVAL;
+    if (cfg->transfer_mode > AVSG_XFER_ALL_K) return AVSG_EINVAL;
+    if ((uint64_t)cfg->max_topk * cfg->max_tokens > cfg->buffer_slots) return AVSG_ECAPACITY;   // Eq. 7
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device < 0 || cfg->device >= ndev) return AVSG_ECUDA;
+    DeviceGuard guard(cfg->device);
+    if (!guard.ok) return AVSG_ECUDA;
+
+    avsg_ctx* c = new (std::nothrow) avsg_ctx();
+    if (!c) return AVSG_ENOMEM;
+    c->cfg = *cfg;
+    c->logS = ilog2(cfg->buffer_slots);
+    c->logH = c->logS + 1;
+    c->list_stride = cfg->max_topk * cfg->max_tokens;
+    const size_t T = cfg->num_tables, S = cfg->buffer_slots;
+    c->kv_host.assign(T, 0); c->kv_dev.assign(T, 0); c->seen.assign(T, 0);
+
+    int max_smem = 0;
+    cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, cfg->device);
+    cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device);
+    const size_t need = stage_one_smem_bytes(cfg->buffer_slots, cfg->max_topk);
+    if (need > (size_t)max_smem) { delete c; return AVSG_EUNSUPPORTED; }
+    if (stage_one_prepare(need) != cudaSuccess) { delete c; return AVSG_ECUDA; }
+
+    const size_t n_ids = T * c->list_stride;
+    bool ok = true;
+    ok = ok && cudaMalloc(&c->d_tok, T * S * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_life, T * S) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_buffer, T * S * cfg->row_bytes) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_stats, T * sizeof(TableStats)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_list, n_ids * sizeof(int2)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_seg, T * sizeof(SegDesc)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_status, 256) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_tok_snap, T * S * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_life_snap, T * S) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_idx_stage, n_ids * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_slots_stage, n_ids * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_hit_stage, n_ids) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_mc_stage, T * cfg->max_tokens * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaHostAlloc(&c->h_seg, T * sizeof(SegDesc), cudaHostAllocDefault) == cudaSuccess;
+    ok = ok && cudaHostAlloc(&c->h_list, n_ids * sizeof(int2), cudaHostAllocDefault) == cudaSuccess;
+    for (auto& e : c->ev) ok = ok && cudaEventCreate(&e) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); free_all(c); delete c; return AVSG_ENOMEM; }
+    if (cudaMemset(c->d_status, 0, 256) != cudaSuccess || cudaMemset(c->d_seg, 0, T * sizeof(SegDesc)) != cudaSuccess ||
+        init_tables(c, 0, (uint32_t)T) != AVSG_OK || cudaDeviceSynchronize() != cudaSuccess) {
+        free_all(c); delete c; return AVSG_ECUDA;
+    }
+    *out = c;
+    return AVSG_OK;
+}
+
+int avsg_destroy(avsg_ctx* c)
+{
+    if (!c) return AVSG_EINVAL;
+    DeviceGuard guard(c->cfg.device);
+    cudaDeviceSynchronize();
+    free_all(c);
+    delete c;
+    return AVSG_OK;
+}
+
+int avsg_reset(avsg_ctx* c, const uint32_t* table_ids, uint32_t n)
+{
+    if (!c || (!table_ids && n)) return AVSG_EINVAL;
+    for (uint32_t i = 0; i < n; ++i) if (table_ids[i] >= c->cfg.num_tables) return AVSG_EINVAL;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return AVSG_ECUDA;
+    CU(cudaDeviceSynchronize());
+    for (uint32_t i = 0; i < n; ++i) {
+        int rc = init_tables(c, table_ids[i], 1);
+        if (rc != AVSG_OK) return rc;
+        c->kv_host[table_ids[i]] = 0; c->kv_dev[table_ids[i]] = 0;
+    }
+    CU(cudaDeviceSynchronize());
+    return AVSG_OK;
+}
+
+int avsg_step(avsg_ctx* c, const avsg_step_args* a, void* stream)
+{
+    return step_impl(c, a, static_cast<cudaStream_t>(stream), false);
+}
+
+int avsg_step_host(avsg_ctx* c, const avsg_step_args* a, void* stream)
+{
+    return step_impl(c, a, static_cast<cudaStream_t>(stream), true);
+}
+
+int avsg_buffer(avsg_ctx* c, uint32_t table_id, void** d_rows)
+{
+    if (!c || !d_rows || table_id >= c->cfg.num_tables) return AVSG_EINVAL;
+    *d_rows = c->d_buffer + (size_t)table_id * c->cfg.buffer_slots * c->cfg.row_bytes;
+    return AVSG_OK;
+}
+
+int avsg_stats(avsg_ctx* c, avsg_stats_t* out)
+{
+    if (!c || !out) return AVSG_EINVAL;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return AVSG_ECUDA;
+    CU(cudaDeviceSynchronize());
+    std::vector<TableStats> h(c->cfg.num_tables);
+    CU(cudaMemcpy(h.data(), c->d_stats, h.size() * sizeof(TableStats), cudaMemcpyDeviceToHost));
+    memset(out, 0, sizeof(*out));
+    for (const TableStats& t : h) {
+        out->steps += t.steps; out->tokens += t.tokens; out->hits += t.hits; out->misses += t.misses;
+        out->rows_copied += t.rows; out->extra_decays += t.extra_decays;
+    }
+    out->bytes_copied = out->rows_copied * c->cfg.row_bytes;
+    if (c->timing && c->events_recorded) {
+        float a = 0.f, b = 0.f;
+        if (cudaEventElapsedTime(&a, c->ev[0], c->ev[1]) == cudaSuccess) out->last_stage_one_us = a * 1000.f;
+        if (cudaEventElapsedTime(&b, c->ev[1], c->ev[2]) == cudaSuccess) out->last_transfer_us = b * 1000.f;
+        cudaGetLastError();
+    }
+    out->last_rows = out->rows_copied - c->last_rows;
+    c->last_rows = out->rows_copied;
+    return read_status(c, nullptr);
+}
+
+int avsg_sync_status(avsg_ctx* c, uint32_t* status_word)
+{
+    if (!c) return AVSG_EINVAL;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return AVSG_ECUDA;
+    CU(cudaDeviceSynchronize());
+    return read_status(c, status_word);
+}
+
+int avsg_export_state(avsg_ctx* c, uint32_t table_id, int32_t* tok, int8_t* life)
+{
+    if (!c || !tok || !life || table_id >= c->cfg.num_tables) return AVSG_EINVAL;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return AVSG_ECUDA;
+    const size_t S = c->cfg.buffer_slots;
+    CU(cudaDeviceSynchronize());
+    CU(cudaMemcpy(tok, c->d_tok + table_id * S, S * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    CU(cudaMemcpy(life, c->d_life + table_id * S, S, cudaMemcpyDeviceToHost));
+    return read_status(c, nullptr);
+}
+
+int avsg_import_state(avsg_ctx* c, uint32_t table_id, const int32_t* tok, const int8_t* life)
+{
+    if (!c || !tok || !life || table_id >= c->cfg.num_tables) return AVSG_EINVAL;
+    const size_t S = c->cfg.buffer_slots;
+    for (size_t j = 0; j < S; ++j)
+        if (life[j] < -1 || life[j] > c->cfg.max_lifetime || tok[j] < -1) return AVSG_EINVAL;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return AVSG_ECUDA;
+    CU(cudaDeviceSynchronize());
+    CU(cudaMemcpy(c->d_tok + table_id * S, tok, S * sizeof(int32_t), cudaMemcpyHostToDevice));
+    CU(cudaMemcpy(c->d_life + table_id * S, life, S, cudaMemcpyHostToDevice));
+    return AVSG_OK;
+}
+
+int avsg_save_state(avsg_ctx* c, void* stream)
+{
+    if (!c) return AVSG_EINVAL;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return AVSG_ECUDA;
+    const size_t n = (size_t)c->cfg.num_tables * c->cfg.buffer_slots;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CU(cudaMemcpyAsync(c->d_tok_snap, c->d_tok, n * sizeof(int32_t), cudaMemcpyDeviceToDevice, s));
+    CU(cudaMemcpyAsync(c->d_life_snap, c->d_life, n, cudaMemcpyDeviceToDevice, s));
+    return AVSG_OK;
+}
+
+int avsg_restore_state(avsg_ctx* c, void* stream)
+{
+    if (!c) return AVSG_EINVAL;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return AVSG_ECUDA;
+    const size_t n = (size_t)c->cfg.num_tables * c->cfg.buffer_slots;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CU(cudaMemcpyAsync(c->d_tok, c->d_tok_snap, n * sizeof(int32_t), cudaMemcpyDeviceToDevice, s));
+    CU(cudaMemcpyAsync(c->d_life, c->d_life_snap, n, cudaMemcpyDeviceToDevice, s));
+    return AVSG_OK;
+}
+
+int avsg_set_transfer_mode(avsg_ctx* c, uint32_t mode)
+{
+    if (!c || mode > AVSG_XFER_ALL_K) return AVSG_EINVAL;
+    c->cfg.transfer_mode = mode;
+    return AVSG_OK;
+}
+
+int avsg_set_timing(avsg_ctx* c, int enable)
+{
+    if (!c) return AVSG_EINVAL;
+    c->timing = enable != 0;
+    c->events_recorded = false;
+    return AVSG_OK;
+}
+
+int avsg_set_transfer_geometry(avsg_ctx* c, uint32_t blocks, uint32_t threads)
+{
+    if (!c || threads < 32 || threads > 1024 || threads % 32 || blocks > 65535) return AVSG_EINVAL;
+    c->xfer_blocks = blocks;
+    c->xfer_threads = threads;
+    return AVSG_OK;
+}
+
+const char* avsg_strerror(int code)
+{
+    switch (code) {
+        case AVSG_OK: return "ok";
+        case AVSG_EINVAL: return "invalid argument";
+        case AVSG_ENOMEM: return "out of memory";
+        case AVSG_ECUDA: return "CUDA runtime error";
+        case AVSG_ECAPACITY: return "buffer_slots < n_tokens * topk (capacity bound violated)";
+        case AVSG_EDEVICE_STATUS: return "a kernel reported a problem in the device status word";
+        case AVSG_EUNSUPPORTED: return "shape not supported by this build";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,86 @@
+// Internal declarations shared by the kernels and the C-ABI host code.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace avsg {
+
+// Device status word: kernels OR one of these in when a bounded loop runs out
+// or an index leaves its range; nothing ever traps.
+enum : uint32_t {
+    ST_PROBE_EXHAUSTED = 1u << 0,   // hash probe visited every bucket
+    ST_NO_DEAD_SLOTS   = 1u << 1,   // fewer reclaimable slots than misses (Eq. 7 violated)
+    ST_BAD_SLOT        = 1u << 2,   // slot / position index out of range
+    ST_BAD_SEGMENT     = 1u << 3,   // transfer kernel could not resolve a miss
+};
+
+// One segment of the step's miss list = the misses of one table, in token
+// order then position order (Alg. 4: "append this token's misses").
+struct SegDesc {
+    uint64_t src_base;    // host KV base of the table (device-visible address)
+    uint64_t src_stride;  // bytes between host rows
+    uint64_t dst_base;    // device buffer base of the table
+    uint32_t count;       // entries in the segment
+    uint32_t pad;
+};
+
+struct TableStats {
+    unsigned long long steps, tokens, hits, misses, rows, extra_decays;
+};
+
+constexpr int S1_MAX_TABLES = 128;   // tables per Stage One launch (kernel parameter space)
+constexpr int MAX_IPT = 8;           // ids per thread
+constexpr int MAX_SPT = 8;           // slots per thread
+constexpr int XFER_MAX_SEG = 2048;   // segments per Stage Two launch (prefix sums live in shared memory)
+
+struct S1Params {
+    int32_t*       tok;          // [num_tables][S]
+    int8_t*        life;         // [num_tables][S]
+    uint8_t*       buffer;       // [num_tables][S * row_bytes]
+    TableStats*    stats;        // [num_tables]
+    int2*          miss_list;    // [segments][list_stride]  (x, slot)
+    SegDesc*       seg;          // [segments]
+    uint32_t*      status;       // mapped host word
+    const int32_t* indices;      // [n][n_q][K]
+    int32_t*       slots;        // [n][n_q][K]
+    uint8_t*       hit;          // [n][n_q][K] or null
+    int32_t*       miss_count;   // [n][n_q] or null
+    uint32_t S, logH, row_bytes, K, n_q, L;
+    uint32_t first;              // index within the call of this launch's first table
+    uint32_t list_stride;        // entries per segment of miss_list
+    uint32_t table_id[S1_MAX_TABLES];
+    int32_t  verified_len[S1_MAX_TABLES];
+    uint64_t kv_base[S1_MAX_TABLES];
+    uint64_t kv_stride[S1_MAX_TABLES];
+};
+
+struct XferParams {
+    const SegDesc* seg;
+    const int2*    miss_list;
+    uint32_t*      status;
+    uint32_t n_seg, list_stride, row_bytes, request_level, S;
+};
+
+struct AllKParams {
+    const int32_t* indices;      // [n][n_q*K]
+    int32_t*       slots;
+    uint8_t*       hit;
+    int32_t*       miss_count;
+    int2*          miss_list;
+    SegDesc*       seg;
+    TableStats*    stats;
+    uint8_t*       buffer;
+    uint32_t S, row_bytes, K, n_q, first, list_stride;
+    uint32_t table_id[S1_MAX_TABLES];
+    uint64_t kv_base[S1_MAX_TABLES];
+    uint64_t kv_stride[S1_MAX_TABLES];
+};
+
+size_t stage_one_smem_bytes(uint32_t S, uint32_t K);
+uint32_t stage_one_threads(uint32_t S, uint32_t K);
+cudaError_t stage_one_prepare(size_t max_smem);
+cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream);
+cudaError_t launch_all_k_prepare(const AllKParams& p, uint32_t n_tables, cudaStream_t stream);
+cudaError_t launch_transfer(const XferParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream);
+
+}  // namespace avsg

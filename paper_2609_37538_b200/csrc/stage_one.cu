@@ -1,0 +1,439 @@
+// Stage One of the AVSG operator: match + reserve, one thread block per table.
+//
+// Follows Algorithm 1 (refresh / classify / allocate) with the lifetime
+// operations of Algorithm 3, for the N_q tokens of one iteration in order
+// (Algorithm 4), and the end-of-step invalidation of Algorithm 4.
+//
+// The whole table lives in shared memory for the step:
+//   s_tok[S]   cached id per slot            s_life[S]  lifetime per slot
+//   s_key[H], s_val[H]  open-addressing index id -> slot, H = 2S buckets,
+//                       rebuilt from s_tok at the start of every step
+// The index is private to this kernel (it is not part of the table state): a
+// hit is "some slot holds the id" (Eq. 1), whatever bucket found it.  Entries
+// are never deleted: when a slot is reclaimed its old key stays behind and is
+// recognised as stale because s_tok[slot] no longer equals the key; a later
+// insert of the same id re-uses that bucket, so a key occupies one bucket at
+// most.  The index is rebuilt when stale keys would push the load above 3/4.
+//
+// The decay loop of Algorithm 1 ("decay all, CollectDead, until enough slots
+// are dead") is evaluated in closed form: d = the smallest number of unit
+// decays after which at least n_g lifetimes are negative, read off a
+// histogram of the S lifetimes; the lifetimes then drop by d at once,
+// saturating at -1.  Dead slots are compacted in increasing slot order and
+// the k-th miss in position order takes the k-th of them (ballot-free packed
+// byte arithmetic + warp/block prefix sums, no atomics, so the assignment is
+// deterministic).
+#include "avsg_kernels.cuh"
+
+namespace avsg {
+namespace {
+
+constexpr int32_t EMPTY = -1;
+
+__device__ __forceinline__ uint32_t hash_id(int32_t x, uint32_t logH)
+{
+    return ((uint32_t)x * 2654435769u) >> (32u - logH);
+}
+
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, uint32_t lane)
+{
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        uint32_t n = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= (uint32_t)o) v += n;
+    }
+    return v;
+}
+
+// Exclusive prefix sum over the block in thread order; s_w holds 33 words.
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* s_w, uint32_t& total)
+{
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const uint32_t incl = warp_incl_scan(v, lane);
+    if (lane == 31) s_w[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = lane < nwarps ? s_w[lane] : 0u;
+        uint32_t wi = warp_incl_scan(w, lane);
+        s_w[lane] = wi - w;
+        if (lane == 31) s_w[32] = wi;
+    }
+    __syncthreads();
+    total = s_w[32];
+    return incl - v + s_w[warp];
+}
+
+struct Index {
+    int32_t*  key;
+    uint16_t* val;
+    const int32_t* tok;
+    uint32_t mask, logH;
+};
+
+// Returns the slot holding x, or -1.  Bounded by the number of buckets.
+__device__ __forceinline__ int32_t index_find(const Index& ix, int32_t x, uint32_t* status)
+{
+    uint32_t b = hash_id(x, ix.logH);
+    for (uint32_t it = 0; it <= ix.mask; ++it) {
+        const int32_t k = ix.key[b];
+        if (k == x) {
+            const uint32_t j = ix.val[b];
+            return ix.tok[j] == x ? (int32_t)j : -1;     // a stale key means the id was reclaimed this step
+        }
+        if (k == EMPTY) return -1;
+        b = (b + 1u) & ix.mask;
+    }
+    atomicOr(status, ST_PROBE_EXHAUSTED);
+    return -1;
+}
+
+// Installs x -> slot; re-uses the bucket that already carries x if there is one.
+__device__ __forceinline__ void index_insert(const Index& ix, int32_t x, uint32_t slot, uint32_t* status)
+{
+    uint32_t b = hash_id(x, ix.logH);
+    for (uint32_t it = 0; it <= ix.mask; ++it) {
+        const int32_t old = atomicCAS(&ix.key[b], EMPTY, x);
+        if (old == EMPTY || old == x) { ix.val[b] = (uint16_t)slot; return; }
+        b = (b + 1u) & ix.mask;
+    }
+    atomicOr(status, ST_PROBE_EXHAUSTED);
+}
+
+// The lifetimes of the slots a thread owns, packed one signed byte each into
+// two words; unused lanes carry 0x7F (never counted, never dead).
+__device__ __forceinline__ void life_load(const int8_t* base, uint32_t j0, uint32_t spt, bool own,
+                                          uint32_t& w0, uint32_t& w1)
+{
+    w0 = w1 = 0x7F7F7F7Fu;
+    if (!own) return;
+    if (spt == 8) { const uint2 v = *reinterpret_cast<const uint2*>(base + j0); w0 = v.x; w1 = v.y; }
+    else if (spt == 4) { w0 = *reinterpret_cast<const uint32_t*>(base + j0); }
+    else if (spt == 2) { w0 = 0x7F7F0000u | *reinterpret_cast<const uint16_t*>(base + j0); }
+    else { w0 = 0x7F7F7F00u | (uint8_t)base[j0]; }
+}
+
+__device__ __forceinline__ void life_store(int8_t* base, uint32_t j0, uint32_t spt, bool own, uint32_t w0, uint32_t w1)
+{
+    if (!own) return;
+    if (spt == 8) { *reinterpret_cast<uint2*>(base + j0) = make_uint2(w0, w1); }
+    else if (spt == 4) { *reinterpret_cast<uint32_t*>(base + j0) = w0; }
+    else if (spt == 2) { *reinterpret_cast<uint16_t*>(base + j0) = (uint16_t)w0; }
+    else { base[j0] = (int8_t)(w0 & 0xFFu); }
+}
+
+// life <- max(life - d, -1) on four packed signed bytes
+__device__ __forceinline__ uint32_t decay4(uint32_t w, uint32_t d)
+{
+    return __vmaxs4(__vsubss4(w, d * 0x01010101u), 0xFFFFFFFFu);
+}
+
+__device__ __forceinline__ void build_index(const Index& ix, const int32_t* s_tok, uint32_t j0, uint32_t spt, bool own,
+                                            uint32_t* s_fill, uint32_t* status)
+{
+    uint32_t live = 0;
+    if (own) {
+#pragma unroll
+        for (uint32_t k = 0; k < (uint32_t)MAX_SPT; ++k) {
+            if (k < spt) {
+                const int32_t x = s_tok[j0 + k];
+                if (x >= 0) { index_insert(ix, x, j0 + k, status); ++live; }
+            }
+        }
+    }
+    live = __reduce_add_sync(0xffffffffu, live);
+    if ((threadIdx.x & 31u) == 0 && live) atomicAdd(s_fill, live);
+}
+
+__global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_constant__ S1Params p)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    const uint32_t S = p.S, K = p.K, H = 1u << p.logH, Kp = (K + 7u) & ~7u;
+    const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31u;
+    const int32_t L = (int32_t)p.L;
+
+    int32_t*  s_tok      = reinterpret_cast<int32_t*>(smem);
+    int32_t*  s_key      = s_tok + S;
+    int32_t*  s_miss_x   = s_key + H;
+    uint16_t* s_val      = reinterpret_cast<uint16_t*>(s_miss_x + Kp);
+    uint16_t* s_miss_pos = s_val + H;
+    uint16_t* s_dead     = s_miss_pos + Kp;
+    int8_t*   s_life     = reinterpret_cast<int8_t*>(s_dead + Kp);
+    uint32_t* s_hist     = reinterpret_cast<uint32_t*>(s_life + S);
+    uint32_t* s_scan_a   = s_hist + 128;
+    uint32_t* s_scan_b   = s_scan_a + 40;
+    uint32_t* s_fill     = s_scan_b + 40;
+
+    const uint32_t ti = p.first + blockIdx.x;            // table index within the call
+    const uint32_t table = p.table_id[blockIdx.x];
+    int32_t* g_tok = p.tok + (size_t)table * S;
+    int8_t*  g_life = p.life + (size_t)table * S;
+
+    const uint32_t spt = S >= nt ? S / nt : 1u;           // slots per thread, power of two <= 8
+    const uint32_t j0 = tid * spt;
+    const bool own = j0 < S;
+    const uint32_t ipt = (K + nt - 1) / nt;               // ids per thread, <= 8
+    const uint32_t i0 = tid * ipt;
+
+    Index ix{s_key, s_val, s_tok, H - 1u, p.logH};
+
+    // ---- load the table; global pre-decay of the iteration's first token (Alg. 1 Pass 1) ----
+    for (uint32_t i = tid; i < H / 4; i += nt) reinterpret_cast<int4*>(s_key)[i] = make_int4(EMPTY, EMPTY, EMPTY, EMPTY);
+    if (tid == 0) *s_fill = 0;
+    if (own) {
+        if ((spt & 3u) == 0) {
+            for (uint32_t q = 0; q < spt / 4; ++q)
+                reinterpret_cast<int4*>(s_tok + j0)[q] = __ldg(reinterpret_cast<const int4*>(g_tok + j0) + q);
+        } else {
+            for (uint32_t k = 0; k < spt; ++k) s_tok[j0 + k] = __ldg(g_tok + j0 + k);
+        }
+    }
+    {
+        uint32_t w0, w1;
+        life_load(g_life, j0, spt, own, w0, w1);
+        life_store(s_life, j0, spt, own, decay4(w0, 1), decay4(w1, 1));
+    }
+    __syncthreads();
+    build_index(ix, s_tok, j0, spt, own, s_fill, p.status);
+    __syncthreads();
+    uint32_t fill_bound = *s_fill;                        // non-empty buckets (upper bound)
+
+    uint32_t list_off = 0, sum_valid = 0, sum_miss = 0, sum_decay = 0;
+    int2* list = p.miss_list + (size_t)ti * p.list_stride;
+
+    for (uint32_t g = 0; g < p.n_q; ++g) {
+        const size_t row = ((size_t)ti * p.n_q + g) * K;
+        const int32_t* X = p.indices + row;
+        int32_t* O = p.slots + row;
+        uint8_t* Hm = p.hit ? p.hit + row : nullptr;
+        if (tid < 128) s_hist[tid] = 0;
+
+        // ---- Probe, refresh hits to L, emit hit slots (Pass 1 + Pass 2) ----
+        int32_t xs[MAX_IPT];
+        uint32_t missmask = 0, nmiss = 0, nvalid = 0;
+#pragma unroll
+        for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {
+            const uint32_t i = i0 + k;
+            if (k < ipt && i < K) {
+                const int32_t x = __ldg(X + i);
+                xs[k] = x;
+                if (x >= 0) {
+                    ++nvalid;
+                    const int32_t j = index_find(ix, x, p.status);
+                    if (j >= 0) {
+                        s_life[j] = (int8_t)L;
+                        O[i] = j;
+                        if (Hm) Hm[i] = 1;
+                    } else {
+                        missmask |= 1u << k;
+                        ++nmiss;
+                    }
+                } else {
+                    O[i] = -1;
+                    if (Hm) Hm[i] = 0;
+                }
+            }
+        }
+        // order-preserving compaction of the misses: t = x[not m]
+        uint32_t total;
+        uint32_t off = block_excl_scan(nmiss | (nvalid << 16), s_scan_a, total) & 0xFFFFu;
+        const uint32_t n_g = total & 0xFFFFu;
+        sum_valid += total >> 16;
+        sum_miss += n_g;
+#pragma unroll
+        for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {
+            if (missmask & (1u << k)) {
+                s_miss_x[off] = xs[k];
+                s_miss_pos[off] = (uint16_t)(i0 + k);
+                ++off;
+            }
+        }
+        if (tid == 0 && p.miss_count) p.miss_count[(size_t)ti * p.n_q + g] = (int32_t)n_g;
+        if (n_g == 0) { __syncthreads(); continue; }
+        __syncthreads();
+
+        // ---- Pass 3: how many unit decays until n_g slots are dead ----
+        uint32_t w0, w1;
+        life_load(s_life, j0, spt, own, w0, w1);
+        for (int32_t v = -1; v <= L; ++v) {
+            const uint32_t vv = (uint32_t)(v & 0xFF) * 0x01010101u;
+            uint32_t c = (__popc(__vcmpeq4(w0, vv)) + __popc(__vcmpeq4(w1, vv))) >> 3;
+            c = __reduce_add_sync(0xffffffffu, c);
+            if (lane == 0 && c) atomicAdd(&s_hist[v + 1], c);
+        }
+        __syncthreads();
+        uint32_t d = (uint32_t)L + 1u, cum = 0;
+        bool found = false;
+        for (uint32_t b = 0; b <= (uint32_t)L + 1u; ++b) {   // bin b counts lifetime b-1; dead after d = b decays
+            cum += s_hist[b];
+            if (cum >= n_g) { d = b; found = true; break; }
+        }
+        if (!found && tid == 0) atomicOr(p.status, ST_NO_DEAD_SLOTS);
+        if (d > 0) {
+            w0 = decay4(w0, d);
+            w1 = decay4(w1, d);
+            life_store(s_life, j0, spt, own, w0, w1);
+        }
+        // CollectDead: dead slots in increasing order; keep the first n_g
+        const uint32_t sg0 = w0 & 0x80808080u, sg1 = w1 & 0x80808080u;
+        uint32_t dtotal;
+        uint32_t doff = block_excl_scan(__popc(sg0) + __popc(sg1), s_scan_b, dtotal);
+#pragma unroll
+        for (uint32_t k = 0; k < (uint32_t)MAX_SPT; ++k) {
+            const uint32_t bit = k < 4 ? (sg0 >> (8 * k + 7)) & 1u : (sg1 >> (8 * (k - 4) + 7)) & 1u;
+            if (bit) {
+                if (doff < n_g) s_dead[doff] = (uint16_t)(j0 + k);
+                ++doff;
+            }
+        }
+        __syncthreads();
+
+        // ---- install the misses: k-th miss takes the k-th dead slot ----
+        const bool rebuild = fill_bound + n_g > (H / 4u) * 3u;
+        const uint32_t n_take = n_g < dtotal ? n_g : dtotal;
+        for (uint32_t k = tid; k < n_take; k += nt) {
+            const uint32_t j = s_dead[k];
+            const int32_t x = s_miss_x[k];
+            const uint32_t i = s_miss_pos[k];
+            if (j < S && i < K) {
+                s_tok[j] = x;
+                s_life[j] = (int8_t)L;
+                O[i] = (int32_t)j;
+                if (Hm) Hm[i] = 0;
+                list[list_off + k] = make_int2(x, (int32_t)j);
+                if (!rebuild) index_insert(ix, x, j, p.status);
+            } else {
+                atomicOr(p.status, ST_BAD_SLOT);
+            }
+        }
+        list_off += n_take;
+        sum_decay += d;
+        if (!rebuild) {
+            fill_bound += n_g;
+            __syncthreads();
+        } else {
+            __syncthreads();
+            for (uint32_t i = tid; i < H / 4; i += nt)
+                reinterpret_cast<int4*>(s_key)[i] = make_int4(EMPTY, EMPTY, EMPTY, EMPTY);
+            if (tid == 0) *s_fill = 0;
+            __syncthreads();
+            build_index(ix, s_tok, j0, spt, own, s_fill, p.status);
+            __syncthreads();
+            fill_bound = *s_fill;
+        }
+    }
+
+    // ---- write the table back; speculative entries (id >= N) become empty (Alg. 4) ----
+    const int32_t N = p.verified_len[blockIdx.x];
+    if (own) {
+        if ((spt & 3u) == 0) {
+            for (uint32_t q = 0; q < spt / 4; ++q) {
+                int4 v = reinterpret_cast<const int4*>(s_tok + j0)[q];
+                v.x = v.x >= N ? -1 : v.x; v.y = v.y >= N ? -1 : v.y;
+                v.z = v.z >= N ? -1 : v.z; v.w = v.w >= N ? -1 : v.w;
+                reinterpret_cast<int4*>(g_tok + j0)[q] = v;
+            }
+        } else {
+            for (uint32_t k = 0; k < spt; ++k) {
+                const int32_t v = s_tok[j0 + k];
+                g_tok[j0 + k] = v >= N ? -1 : v;
+            }
+        }
+        uint32_t w0, w1;
+        life_load(s_life, j0, spt, own, w0, w1);
+        life_store(g_life, j0, spt, own, w0, w1);
+    }
+    if (tid == 0) {
+        SegDesc sd;
+        sd.src_base = p.kv_base[blockIdx.x];
+        sd.src_stride = p.kv_stride[blockIdx.x];
+        sd.dst_base = reinterpret_cast<uint64_t>(p.buffer + (size_t)table * S * p.row_bytes);
+        sd.count = list_off;
+        sd.pad = 0;
+        p.seg[ti] = sd;
+        TableStats* st = p.stats + table;
+        st->steps += 1;
+        st->tokens += p.n_q;
+        st->hits += sum_valid - sum_miss;
+        st->misses += sum_miss;
+        st->rows += list_off;
+        st->extra_decays += sum_decay;
+    }
+}
+
+// "KV offload" comparator: every selected row moves, position (g, i) -> slot g*K + i.
+__global__ void __launch_bounds__(256) avsg_all_k_prepare_kernel(const __grid_constant__ AllKParams p)
+{
+    __shared__ uint32_t s_valid;
+    const uint32_t g = blockIdx.x, b = blockIdx.y, ti = p.first + b, K = p.K;
+    const uint32_t table = p.table_id[b];
+    if (threadIdx.x == 0) s_valid = 0;
+    __syncthreads();
+    const size_t row = ((size_t)ti * p.n_q + g) * K;
+    int2* list = p.miss_list + (size_t)ti * p.list_stride + (size_t)g * K;
+    uint32_t valid = 0;
+    for (uint32_t i = threadIdx.x; i < K; i += blockDim.x) {
+        const int32_t x = __ldg(p.indices + row + i);
+        const int32_t o = x >= 0 ? (int32_t)(g * K + i) : -1;
+        p.slots[row + i] = o;
+        if (p.hit) p.hit[row + i] = 0;
+        list[i] = make_int2(x, o);
+        valid += x >= 0;
+    }
+    valid = __reduce_add_sync(0xffffffffu, valid);
+    if ((threadIdx.x & 31u) == 0 && valid) atomicAdd(&s_valid, valid);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (p.miss_count) p.miss_count[(size_t)ti * p.n_q + g] = (int32_t)s_valid;
+        TableStats* st = p.stats + table;
+        atomicAdd(&st->tokens, 1ull);
+        atomicAdd(&st->misses, (unsigned long long)s_valid);
+        atomicAdd(&st->rows, (unsigned long long)s_valid);
+        if (g == 0) {
+            SegDesc sd;
+            sd.src_base = p.kv_base[b];
+            sd.src_stride = p.kv_stride[b];
+            sd.dst_base = reinterpret_cast<uint64_t>(p.buffer + (size_t)table * p.S * p.row_bytes);
+            sd.count = p.n_q * K;
+            sd.pad = 0;
+            p.seg[ti] = sd;
+            atomicAdd(&st->steps, 1ull);
+        }
+    }
+}
+
+}  // namespace
+
+size_t stage_one_smem_bytes(uint32_t S, uint32_t K)
+{
+    const size_t H = 2ull * S, Kp = (K + 7u) & ~7u;
+    return S * 4 + H * 4 + Kp * 4 + H * 2 + Kp * 2 + Kp * 2 + S + (128 + 40 + 40 + 8) * 4;
+}
+
+uint32_t stage_one_threads(uint32_t S, uint32_t K)
+{
+    (void)K;
+    uint32_t t = S / 2;
+    if (t < 128) t = 128;
+    if (t > 1024) t = 1024;
+    return t;
+}
+
+cudaError_t stage_one_prepare(size_t max_smem)
+{
+    return cudaFuncSetAttribute(avsg_stage_one_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+}
+
+cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream)
+{
+    const uint32_t threads = stage_one_threads(p.S, p.K);
+    avsg_stage_one_kernel<<<n_tables, threads, stage_one_smem_bytes(p.S, p.K), stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_all_k_prepare(const AllKParams& p, uint32_t n_tables, cudaStream_t stream)
+{
+    avsg_all_k_prepare_kernel<<<dim3(p.n_q, n_tables), 256, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace avsg

@@ -1,0 +1,224 @@
+"""Bit-exact parity of the CUDA path (through the C ABI) with the CPU oracle, on a B200."""
+import ctypes
+
+import numpy as np
+import pytest
+
+import avsg_traces as tr
+from oracle import OracleTable
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def avsg():
+    import torch
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    import paper_2609_37538_b200 as m
+    m.load_library()
+    return m
+
+
+def _parity(*a, **kw):
+    from harness import run_parity
+    return run_parity(*a, **kw)
+
+
+# ---- the five configurations at full size ---------------------------------------------------------------
+def test_c1_full(avsg):
+    r = _parity(tr.workload("C1"))
+    assert r["gpu"]["tokens"] == 16 and r["gpu"]["extra_decays"] == 0
+
+
+def test_c2_full(avsg):
+    r = _parity(tr.workload("C2"), buffer_every=8)
+    g = r["gpu"]
+    assert g["tokens"] == 256 and g["hits"] + g["misses"] == 256 * 2048
+
+
+def test_c3_full(avsg):
+    # 128 tables (32 requests x 4 layers), 11 GB of pinned host KV; every table checked after every step
+    r = _parity(tr.workload("C3"), buffer_every=16)
+    g = r["gpu"]
+    assert g["tokens"] == 128 * 64 * 2 and g["hits"] + g["misses"] == g["tokens"] * 2048
+
+
+def test_c4_full(avsg):
+    r = _parity(tr.workload("C4"), buffer_every=16)
+    assert r["gpu"]["tokens"] == 16 * 64 * 2
+
+
+def test_c5_full_balanced(avsg):
+    r = _parity(tr.workload("C5"), buffer_every=8)
+    assert r["gpu"]["tokens"] == 64 * 33
+
+
+@pytest.mark.parametrize("mode_name", ["XFER_REQUEST_LEVEL", "XFER_ALL_K"])
+def test_c5_comparators(avsg, mode_name):
+    r = _parity(tr.workload("C5", n_iters=6), mode=getattr(avsg, mode_name), buffer_every=2)
+    assert r["gpu"]["rows_copied"] == r["oracle"]["rows_copied"]
+
+
+def test_copy_engine_comparator(avsg):
+    _parity(tr.workload("C3", requests=4, layers=2, n_iters=6, context=32768), mode=avsg.XFER_COPY_ENGINE)
+
+
+# ---- shapes that span several tiles, ragged tails and the degenerate cases ---------------------------------
+SHAPES = [
+    # name, overrides
+    ("C2", dict(topk=37, buffer_slots=128, n_iters=40, context=4096, recent_window=128)),      # odd K
+    ("C2", dict(topk=16, buffer_slots=32, n_iters=60, context=512, recent_window=64)),         # smallest S = N_q K
+    ("C2", dict(topk=1000, buffer_slots=2048, n_iters=30, context=65536, recent_window=2048)),  # K not a power of two
+    ("C2", dict(topk=4096, buffer_slots=8192, n_iters=10, context=65536, recent_window=8192)),  # S = N_q K at max S
+    ("C2", dict(topk=2048, buffer_slots=4096, n_iters=24, context=65536, max_lifetime=1)),      # L = 1, S = N_q K
+    ("C2", dict(topk=512, buffer_slots=4096, n_iters=40, context=65536, max_lifetime=126)),     # largest L
+    ("C4", dict(topk=300, buffer_slots=1024, n_iters=40, context=1 << 16, requests=5, hot_size=64, hot_range=1024)),
+    ("C5", dict(topk=256, buffer_slots=256, n_iters=20, requests=7, ctx_lo=512, ctx_hi=8192)),   # S = K, one token
+    ("C5", dict(topk=8192, buffer_slots=8192, n_iters=5, requests=2, ctx_lo=20000, ctx_hi=60000)),  # K = S = max
+]
+
+
+@pytest.mark.parametrize("name,kw", SHAPES)
+def test_shapes(avsg, name, kw):
+    _parity(tr.workload(name, **kw))
+
+
+def test_more_tables_than_one_launch_takes(avsg):
+    w = tr.workload("C5", topk=64, buffer_slots=128, n_iters=6, requests=300, ctx_lo=256, ctx_hi=2048)
+    _parity(w, buffer_every=3)
+
+
+def test_padding_when_context_is_shorter_than_k(avsg):
+    w = tr.workload("C5", topk=128, buffer_slots=256, n_iters=6, requests=4, ctx_lo=40, ctx_hi=100)
+    r = _parity(w)
+    assert r["gpu"]["hits"] + r["gpu"]["misses"] < 4 * 6 * 128
+
+
+def test_strided_host_rows_and_host_io(avsg):
+    w = tr.workload("C4", topk=256, buffer_slots=1024, n_iters=12, context=1 << 15, requests=3, hot_size=64,
+                    hot_range=1024)
+    _parity(w, row_stride=1024)
+    _parity(w, host_io=True)
+
+
+def test_other_row_sizes(avsg):
+    for rb in (16, 1152, 4096):
+        _parity(tr.workload("C2", topk=128, buffer_slots=512, n_iters=10, context=8192, row_bytes=rb))
+
+
+def test_transfer_geometries(avsg):
+    w = tr.workload("C5", topk=512, buffer_slots=1024, n_iters=5, requests=9, ctx_lo=1024, ctx_hi=8192)
+    for geo in [(1, 32), (7, 1024), (148, 128), (600, 256)]:
+        _parity(w, xfer_geometry=geo)
+
+
+# ---- behaviours ---------------------------------------------------------------------------------------------
+def test_regenerated_speculative_row_is_fetched_again(avsg):
+    import torch
+    rb, S, K, N = 656, 64, 4, 100
+    kv = avsg.pinned_empty((N + 4) * rb)
+    tr.fill_kv(kv.data_ptr(), 1, 0, N + 4, rb)
+    ctx = avsg.Context(1, S, rb, K, 1, 16)
+    orc = OracleTable(S, rb, 16)
+    X = np.array([[[5, 50, 99, 100]]], dtype=np.int32)
+    out = ctx.step([0], torch.from_numpy(X).cuda(), [kv], [N])
+    r = orc.step(X[0], N, kv.numpy())
+    assert (out.slots.cpu().numpy()[0] == r.O).all()
+    tok, life = ctx.export_state(0)
+    assert tok[r.O[0, 3]] == -1 and life[r.O[0, 3]] == 16
+    tr.fill_kv(kv.data_ptr() + 100 * rb, 1, 0, 1, rb, first_row=100, version=1)    # host regenerates the row
+    out = ctx.step([0], torch.from_numpy(X).cuda(), [kv], [N + 1])
+    r = orc.step(X[0], N + 1, kv.numpy())
+    assert out.hit.cpu().numpy()[0, 0].tolist() == [1, 1, 1, 0] == r.M[0].tolist()
+    assert (ctx.buffer(0).cpu().numpy() == orc.rows()).all()
+    new_slot = int(out.slots.cpu().numpy()[0, 0, 3])
+    assert (ctx.buffer(0).cpu().numpy()[new_slot] == kv.numpy()[100 * rb:101 * rb]).all()
+
+
+def test_device_resident_kv_and_reset_import_export(avsg):
+    import torch
+    rb, S, K = 64, 128, 16
+    host = np.empty(1000 * rb, np.uint8)
+    tr.fill_kv(host, 2, 0, 1000, rb)
+    dkv = torch.from_numpy(host).cuda()
+    ctx = avsg.Context(2, S, rb, K, 2, 4)
+    orc = OracleTable(S, rb, 4)
+    rng = np.random.default_rng(0)
+    for step in range(10):
+        X = np.stack([np.sort(rng.choice(1000, K, replace=False)) for _ in range(2)]).astype(np.int32)
+        out = ctx.step([1], torch.from_numpy(X[None]).cuda(), [dkv], [1000])
+        r = orc.step(X, 1000, host)
+        assert (out.slots.cpu().numpy()[0] == r.O).all()
+    assert (ctx.buffer(1).cpu().numpy() == orc.rows()).all()
+    assert (ctx.export_state(0)[0] == -1).all()                      # the other table was never touched
+    tok, life = ctx.export_state(1)
+    ctx.import_state(0, tok, life)                                   # checkpoint / resume into table 0
+    X = np.sort(rng.choice(1000, (1, K), replace=False), axis=1).astype(np.int32)
+    a = ctx.step([0], torch.from_numpy(X[None]).cuda(), [dkv], [1000])
+    b = ctx.step([1], torch.from_numpy(X[None]).cuda(), [dkv], [1000])
+    assert (a.slots.cpu() == b.slots.cpu()).all() and (a.hit.cpu() == b.hit.cpu()).all()
+    ctx.reset([1])
+    tok, life = ctx.export_state(1)
+    assert (tok == -1).all() and (life == -1).all() and (ctx.buffer(1).cpu().numpy() == 0).all()
+    c = ctx.step([1], torch.from_numpy(X[None]).cuda(), [dkv], [1000])
+    assert c.hit.cpu().numpy().sum() == 0 and c.slots.cpu().numpy()[0, 0].tolist() == list(range(K))
+
+
+def test_save_restore_replays_a_step(avsg):
+    import torch
+    w = tr.workload("C2", topk=256, buffer_slots=1024, n_iters=8, context=16384, recent_window=512)
+    X, N = tr.generate(w.tables[0])
+    kv = avsg.pinned_empty(w.tables[0].context * w.row_bytes)
+    tr.fill_kv(kv.data_ptr(), w.seed, 0, w.tables[0].context, w.row_bytes)
+    ctx = avsg.Context(1, w.buffer_slots, w.row_bytes, w.topk, 2, 16)
+    for t in range(6):
+        ctx.step([0], torch.from_numpy(X[t][None]).cuda(), [kv], [int(N[t])])
+    ctx.save_state()
+    first = ctx.step([0], torch.from_numpy(X[6][None]).cuda(), [kv], [int(N[6])])
+    state = ctx.export_state(0)
+    for _ in range(3):
+        ctx.restore_state()
+        again = ctx.step([0], torch.from_numpy(X[6][None]).cuda(), [kv], [int(N[6])])
+        assert (again.slots.cpu() == first.slots.cpu()).all() and (again.hit.cpu() == first.hit.cpu()).all()
+        s2 = ctx.export_state(0)
+        assert (s2[0] == state[0]).all() and (s2[1] == state[1]).all()
+
+
+def test_timing_and_stats(avsg):
+    import torch
+    w = tr.workload("C2", topk=512, buffer_slots=2048, n_iters=4, context=16384, recent_window=512)
+    X, N = tr.generate(w.tables[0])
+    kv = avsg.pinned_empty(w.tables[0].context * w.row_bytes)
+    tr.fill_kv(kv.data_ptr(), w.seed, 0, w.tables[0].context, w.row_bytes)
+    ctx = avsg.Context(1, w.buffer_slots, w.row_bytes, w.topk, 2, 16)
+    ctx.set_timing(True)
+    for t in range(4):
+        ctx.step([0], torch.from_numpy(X[t][None]).cuda(), [kv], [int(N[t])])
+    st = ctx.stats()
+    assert st["last_stage_one_us"] > 0 and st["last_transfer_us"] > 0
+    assert st["steps"] == 4 and st["tokens"] == 8 and st["hits"] + st["misses"] == 8 * 512
+    assert st["bytes_copied"] == st["rows_copied"] * w.row_bytes == st["misses"] * w.row_bytes
+
+
+def test_argument_errors(avsg):
+    import torch
+    ctx = avsg.Context(4, 64, 32, 16, 2, 4)
+    kv = avsg.pinned_empty(100 * 32)
+    idx = torch.zeros((1, 2, 16), dtype=torch.int32, device="cuda")
+    with pytest.raises(avsg.AvsgError) as e:
+        ctx.step([4], idx, [kv], [100])                                  # table id out of range
+    assert e.value.code == avsg.EINVAL
+    with pytest.raises(avsg.AvsgError) as e:
+        ctx.step([1, 1], torch.zeros((2, 2, 16), dtype=torch.int32, device="cuda"), [kv, kv], [100, 100])
+    assert e.value.code == avsg.EINVAL                                   # duplicate table
+    with pytest.raises(avsg.AvsgError) as e:
+        ctx.step([0], torch.zeros((1, 2, 40), dtype=torch.int32, device="cuda"), [kv], [100])
+    assert e.value.code == avsg.EINVAL                                   # K above max_topk
+    pageable = np.zeros(100 * 32, np.uint8)
+    with pytest.raises(avsg.AvsgError) as e:
+        ctx.step([0], idx, [pageable], [100])                            # host KV that the GPU cannot read
+    assert e.value.code == avsg.EINVAL
+    with pytest.raises(avsg.AvsgError) as e:
+        avsg.Context(1, 64, 32, 40, 2, 4)                                # Eq. 7 at create
+    assert e.value.code == avsg.ECAPACITY
+    assert ctx.sync_status() == 0
