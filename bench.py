@@ -1,0 +1,419 @@
+#!/usr/bin/env python
+"""Benchmark of the AVSG per-decode-step operator on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Workload: configuration C3 (32 requests x 4 layers = 128 tables, context 131072, top-K 2048, 8192-slot
+buffers, 2 query tokens per iteration, 656-byte rows, ~11 GB of pinned host KV).  One "step" is one decode
+iteration of the whole batch: four operator calls (one per layer, 32 tables each), every call running
+match + reserve (Stage One) and the balanced miss-only host->device gather (Stage Two).
+
+Prints ONE JSON line (rank 0).  value = miss bytes the step needed / device time of the step (GB/s, whole job).
+roofline = Stage Two alone against the pinned-copy bandwidth measured in the same run (the host link bounds it);
+roofline_stage_one = Stage One against the measured HBM copy bandwidth.
+
+--impl reference times the CPU oracle (plain C, one thread per table over the host cores) on the same
+workload; it is a deliberately slow checker, reported as a baseline.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "miss-only H2D gather GB/s (% of link peak); match+reserve us per decode step"
+PAPER_CONTEXT = {
+    "hardware": "Ascend 910B NPU (paper), not comparable",
+    "hash_vs_dual_pointer_speedup": 2.80, "stage_one_us_K2048_S2048": 53.7,
+    "max_h2d_gain_over_request_level": 34.44, "hit_rate_8k_buffer_pct": 94.83,
+}
+
+
+def _measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()          # the exact process started above
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def _workload(rank: int, n_iters: int, args=None):
+    import avsg_traces as tr
+    kw = {}
+    if args is not None:
+        kw = {"requests": args.requests, "layers": args.layers}
+    return tr.workload("C3", seed=3 + 1000 * rank, n_iters=n_iters, **kw)
+
+
+def _gen_traces(w, threads):
+    import avsg_traces as tr
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        return list(ex.map(lambda c: tr.generate(c), w.tables))
+
+
+# ------------------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle on the host cores
+# ------------------------------------------------------------------------------------------------------------
+def oracle_run(w, traces, kv_np, tables, warmup, steps, threads):
+    """Steps the oracle over `tables` for warmup+steps iterations, one thread per table; times the last `steps`.
+    Returns (seconds per step list, miss rows per step list, hits, misses)."""
+    from oracle import OracleTable
+    orc = {ti: OracleTable(w.buffer_slots, w.row_bytes, w.max_lifetime) for ti in tables}
+
+    def one(ti, t):
+        X, N = traces[ti]
+        r = orc[ti].step(X[t], int(N[t]), kv_np[ti])
+        return int(r.n.sum()), int(r.M.sum())
+
+    secs, rows, hits, misses = [], [], 0, 0
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        for t in range(warmup + steps):
+            t0 = time.perf_counter()
+            res = list(ex.map(lambda ti: one(ti, t), tables))
+            dt = time.perf_counter() - t0
+            if t >= warmup:
+                secs.append(dt)
+                rows.append(sum(r[0] for r in res))
+                misses += sum(r[0] for r in res)
+                hits += sum(r[1] for r in res)
+    return secs, rows, hits, misses
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import __graft_entry__
+    import avsg_traces as tr
+    import oracle
+    tr.build_library(); oracle.build_library()
+    cores = os.cpu_count() or 1
+    n_iters = max(64, args.warmup + args.steps)
+    w = _workload(0, n_iters, args)
+    traces = _gen_traces(w, cores)
+    kv_np = []
+    for ti, cfg in enumerate(w.tables):
+        a = np.empty(cfg.context * w.row_bytes, np.uint8)
+        tr.fill_kv(a, w.seed, ti, cfg.context, w.row_bytes)
+        kv_np.append(a)
+    tables = list(range(w.num_tables))
+    secs, rows, hits, misses = oracle_run(w, traces, kv_np, tables, args.warmup, args.steps, cores)
+    total_bytes = sum(rows) * w.row_bytes
+    value = total_bytes / 1e9 / sum(secs)
+    sample = "all %d tables, %d iterations after %d warm-up, one thread per table over %d threads" % (
+        w.num_tables, args.steps, args.warmup, cores)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(secs) / len(secs),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32/u8",
+        "data": "synthetic", "config": _config(w),
+        "hit_rate": hits / max(1, hits + misses),
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def _config(w):
+    return {"workload": "C3: %d tables (%d requests x %d layers), context 131072, top-K %d, %d-slot buffers, "
+                        "%d query tokens per iteration, %d-byte rows, Beta(18,2) overlap; one step = %d calls of %d tables"
+                        % (w.num_tables, len(w.calls[0]), len(w.calls), w.topk, w.buffer_slots, w.n_q, w.row_bytes,
+                           len(w.calls), len(w.calls[0])),
+            "tables": w.num_tables, "topk": w.topk, "buffer_slots": w.buffer_slots, "n_tokens": w.n_q,
+            "row_bytes": w.row_bytes, "max_lifetime": w.max_lifetime,
+            "host_kv_gb": round(w.host_kv_bytes() / 1e9, 2),
+            "l2": "flushed between timed steps (256 MiB write); host KV (11 GB) is far larger than L2"}
+
+
+# ------------------------------------------------------------------------------------------------------------
+# the CUDA arm
+# ------------------------------------------------------------------------------------------------------------
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    import __graft_entry__
+    import avsg_traces as tr
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        __graft_entry__.build()
+    if world > 1:
+        dist.barrier()
+    import paper_2609_37538_b200 as avsg
+    avsg.load_library()
+
+    cores = os.cpu_count() or 1
+    threads = max(1, cores // world)
+    W, K = args.warmup, args.steps
+    n_iters = max(64, W + K)
+    w = _workload(rank, n_iters, args)
+    traces = _gen_traces(w, threads)
+    kv = []
+    for ti, cfg in enumerate(w.tables):
+        buf = avsg.pinned_empty(cfg.context * w.row_bytes)
+        tr.fill_kv(buf.data_ptr(), w.seed, ti, cfg.context, w.row_bytes)
+        kv.append(buf)
+
+    ctx = avsg.Context(num_tables=w.num_tables, buffer_slots=w.buffer_slots, row_bytes=w.row_bytes,
+                       max_topk=w.topk, max_tokens=w.n_q, max_lifetime=w.max_lifetime, device=local)
+    ncalls = len(w.calls)
+    calls = [ctx.prepare(grp, [kv[t] for t in grp], w.n_q, w.topk) for grp in w.calls]
+    # inputs resident in HBM: every iteration's ids, per call [n, n_q, K]
+    Xh = [[np.stack([traces[ti][0][t] for ti in grp]) for grp in w.calls] for t in range(n_iters)]
+    vlen = [[[int(traces[ti][1][t]) for ti in grp] for grp in w.calls] for t in range(n_iters)]
+    Xd = [[torch.from_numpy(x).cuda() for x in row] for row in Xh]
+    slots_d = [torch.empty_like(Xd[0][c]) for c in range(ncalls)]
+    mc_d = [torch.empty((len(w.calls[c]), w.n_q), dtype=torch.int32, device="cuda") for c in range(ncalls)]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def device_step(t):
+        for c in range(ncalls):
+            calls[c].run(Xd[t][c], vlen[t][c], slots_d[c], None, mc_d[c], stream)
+
+    # ---- host-link peak: large pinned copy on this machine, this run ----
+    big_h = torch.empty(1 << 30, dtype=torch.uint8, pin_memory=True)
+    big_d = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
+    big_d.copy_(big_h, non_blocking=True)
+    torch.cuda.synchronize()
+    best = 0.0
+    for _ in range(4):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); big_d.copy_(big_h, non_blocking=True); e1.record()
+        torch.cuda.synchronize()
+        best = max(best, (1 << 30) / 1e9 / (e0.elapsed_time(e1) / 1e3))
+    link_peak = best
+    del big_h, big_d
+
+    # ---- warm-up (cold start + W-1 iterations), then the timed steps ----
+    for t in range(W):
+        device_step(t)
+    torch.cuda.synchronize()
+    st0 = ctx.stats()
+    ctx.save_state()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    torch.cuda.synchronize()
+    for k in range(K):
+        flush.fill_(k & 0xFF)
+        ev[k][0].record()
+        device_step(W + k)
+        ev[k][1].record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    st1 = ctx.stats()
+    clocks = sampler.stop()
+    rows_timed = st1["rows_copied"] - st0["rows_copied"]
+    hits_timed, miss_timed = st1["hits"] - st0["hits"], st1["misses"] - st0["misses"]
+    total_ms = sum(step_ms)
+
+    # ---- end to end: ids from pinned host memory, slot table back to pinned host memory ----
+    Xp = [[torch.from_numpy(x).pin_memory() for x in row] for row in Xh[W:W + K]]
+    slots_h = [torch.empty(Xd[0][c].shape, dtype=torch.int32, pin_memory=True) for c in range(ncalls)]
+    mc_h = [torch.empty((len(w.calls[c]), w.n_q), dtype=torch.int32, pin_memory=True) for c in range(ncalls)]
+    ctx.restore_state()
+    torch.cuda.synchronize()
+    ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for k in range(K):
+        flush.fill_(k & 0xFF)
+        ev2[k][0].record()
+        for c in range(ncalls):
+            calls[c].run(Xp[k][c], vlen[W + k][c], slots_h[c], None, mc_h[c], stream, host=True)
+        ev2[k][1].record()
+    torch.cuda.synchronize()
+    e2e_ms = sum(a.elapsed_time(b) for a, b in ev2)
+    ids_bytes = sum(x.numel() * 4 for x in Xp[0])
+    mc_bytes = sum(m.numel() * 4 for m in mc_h)
+
+    # ---- per-kernel times (events inside the library around Stage One / Stage Two), L2 flushed per call ----
+    ctx.restore_state()
+    ctx.set_timing(True)
+    torch.cuda.synchronize()
+    ctx.stats()
+    s1_us, x_us, x_rows = [], [], []
+    for k in range(K):
+        for c in range(ncalls):
+            flush.fill_(c)
+            calls[c].run(Xd[W + k][c], vlen[W + k][c], slots_d[c], None, mc_d[c], stream)
+            s = ctx.stats()
+            s1_us.append(s["last_stage_one_us"]); x_us.append(s["last_transfer_us"]); x_rows.append(s["last_rows"])
+    # ---- replay of one recorded steady-state call, 1000 times (L2-warm), the paper's Stage One protocol ----
+    rep = []
+    ctx.save_state()
+    for _ in range(args.replays):
+        ctx.restore_state()
+        calls[0].run(Xd[W + K - 1][0], vlen[W + K - 1][0], slots_d[0], None, mc_d[0], stream)
+        rep.append(ctx.stats()["last_stage_one_us"])
+    ctx.set_timing(False)
+
+    # ---- aggregate over ranks: device time = max over ranks, work = sum over ranks ----
+    if world > 1:
+        tmax = torch.tensor([total_ms, e2e_ms, sum(x_us)], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        tsum = torch.tensor([rows_timed, sum(x_rows), hits_timed, miss_timed], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
+        total_ms_j, e2e_ms_j, xus_j = tmax.tolist()
+        rows_j, xrows_j, hits_j, miss_j = tsum.tolist()
+    else:
+        total_ms_j, e2e_ms_j, xus_j = total_ms, e2e_ms, sum(x_us)
+        rows_j, xrows_j, hits_j, miss_j = rows_timed, sum(x_rows), hits_timed, miss_timed
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    rb = w.row_bytes
+    value = rows_j * rb / 1e9 / (total_ms_j / 1e3)
+    e2e_value = rows_j * rb / 1e9 / (e2e_ms_j / 1e3)
+    hbm_peak, peak_kind = _measured_peaks()
+    n_launch = len(x_us)
+    x_bytes_per_launch = sum(x_rows) * rb / n_launch
+    x_avg_us = sum(x_us) / n_launch
+    x_gbs = x_bytes_per_launch / 1e3 / x_avg_us
+    # Stage One algorithmic bytes per call: state read + write, ids in, slots out, miss counts, miss list
+    n_tab = len(w.calls[0])
+    s1_bytes = n_tab * (2 * w.buffer_slots * 5 + 2 * w.n_q * w.topk * 4 + w.n_q * 4 + 32) + 8 * sum(x_rows) / n_launch
+    s1_avg_us = sum(s1_us) / len(s1_us)
+    s1_gbs = s1_bytes / 1e3 / s1_avg_us
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": total_ms_j / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int32/u8", "data": "synthetic", "config": _config(w),
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "GB/s",
+                "h2d_bytes_per_step": int(ids_bytes + rows_timed * rb / K), "d2h_bytes_per_step": int(ids_bytes + mc_bytes),
+                "ms_per_step": e2e_ms_j / K,
+                "note": "avsg_step_host: ids uploaded from pinned host memory, slot table and miss counts "
+                        "downloaded; h2d bytes = ids + missed KV rows"},
+        "gpu_launches": 2 * ncalls * K,
+        "hit_rate": hits_j / max(1.0, hits_j + miss_j),
+        "miss_rows_per_step": rows_j / K / world,
+        "link_peak_gbs": link_peak, "link": "PCIe Gen5 x16 (nominal 63 GB/s per direction); peak = best 1 GiB pinned cudaMemcpyAsync H2D in this run",
+        "pct_of_link_peak": 100.0 * x_gbs / link_peak,
+        "match_reserve_us": {"per_call_mean": s1_avg_us, "per_call_median": statistics.median(s1_us),
+                             "per_call_min": min(s1_us), "per_call_max": max(s1_us),
+                             "replay_median": statistics.median(rep) if rep else None, "replays": len(rep),
+                             "tables_per_call": n_tab,
+                             "note": "per_call_*: L2 flushed before each call; replay_*: one recorded call re-run from a restored state (L2-warm)"},
+        "transfer_us": {"per_call_mean": x_avg_us, "per_call_median": statistics.median(x_us),
+                        "rows_per_call_mean": sum(x_rows) / n_launch},
+        "roofline": {"bound": "host_link", "kernel": "avsg_transfer_kernel", "achieved": x_gbs, "peak": link_peak,
+                     "unit": "GB/s", "frac": x_gbs / link_peak, "traffic": None,
+                     "peak_kind": "measured in this run (pinned cudaMemcpyAsync H2D)",
+                     "note": "algorithmic bytes = row_bytes x missed rows per launch; the rows cross the host link, not HBM reads"},
+        "roofline_stage_one": {"bound": "hbm", "kernel": "avsg_stage_one_kernel", "achieved": s1_gbs, "peak": hbm_peak,
+                               "unit": "GB/s", "frac": s1_gbs / hbm_peak, "traffic": None, "peak_kind": peak_kind,
+                               "bytes_per_launch": s1_bytes},
+        "paper_context": PAPER_CONTEXT,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        kv_np = [k.numpy() for k in kv]
+        cb_steps = min(16, K)
+        tables = list(range(w.num_tables))
+        secs, rows, _, _ = oracle_run(w, traces, kv_np, tables, W, cb_steps, cores)
+        line["cpu_baseline"] = {
+            "value": sum(rows) * rb / 1e9 / sum(secs), "unit": "GB/s", "cores": cores, "kind": "oracle",
+            "ms_per_step": 1e3 * sum(secs) / len(secs),
+            "sample": "all %d tables, %d iterations after %d warm-up, one thread per table over %d threads"
+                      % (w.num_tables, cb_steps, W, cores)}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--replays", type=int, default=1000)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--requests", type=int, default=32, help="requests per layer (32 = the full configuration)")
+    ap.add_argument("--layers", type=int, default=4, help="layers (4 = the full configuration)")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()
