@@ -267,7 +267,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     int max_smem = 0;
     cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, cfg->device);
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device);
-    const size_t need = stage_one_smem_bytes(cfg->buffer_slots, cfg->max_topk);
+    const size_t need = stage_one_smem_bytes(cfg->buffer_slots, cfg->max_topk, (uint32_t)cfg->max_lifetime);
     if (need > (size_t)max_smem) { delete c; return AVSG_EUNSUPPORTED; }
     if (stage_one_prepare(need) != cudaSuccess) { delete c; return AVSG_ECUDA; }
 

@@ -76,7 +76,7 @@ struct AllKParams {
     uint64_t kv_stride[S1_MAX_TABLES];
 };
 
-size_t stage_one_smem_bytes(uint32_t S, uint32_t K);
+size_t stage_one_smem_bytes(uint32_t S, uint32_t K, uint32_t L);
 uint32_t stage_one_threads(uint32_t S, uint32_t K);
 cudaError_t stage_one_prepare(size_t max_smem);
 cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream);

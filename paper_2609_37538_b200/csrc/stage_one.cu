@@ -19,7 +19,9 @@
 // are dead") is evaluated in closed form: d = the smallest number of unit
 // decays after which at least n_g lifetimes are negative, read off a
 // histogram of the S lifetimes; the lifetimes then drop by d at once,
-// saturating at -1.  Dead slots are compacted in increasing slot order and
+// saturating at -1.  For L <= 30 the histogram is counted without atomics:
+// every thread bumps private byte counters (one column per thread, one row
+// per lifetime value) and one warp per value sums its row with dp4a.  Dead slots are compacted in increasing slot order and
 // the k-th miss in position order takes the k-th of them (ballot-free packed
 // byte arithmetic + warp/block prefix sums, no atomics, so the assignment is
 // deterministic).
@@ -29,6 +31,7 @@ namespace avsg {
 namespace {
 
 constexpr int32_t EMPTY = -1;
+constexpr int32_t PRIV_HIST_MAX_L = 30;   // private byte-counter histogram up to this L (32 rows)
 
 __device__ __forceinline__ uint32_t hash_id(int32_t x, uint32_t logH)
 {
@@ -127,16 +130,37 @@ __device__ __forceinline__ uint32_t decay4(uint32_t w, uint32_t d)
     return __vmaxs4(__vsubss4(w, d * 0x01010101u), 0xFFFFFFFFu);
 }
 
+// Inserts the ids of the slots a thread owns.  The first compare-and-swap of every id is issued
+// before any result is inspected, so that a thread keeps up to eight shared-memory atomics in flight.
 __device__ __forceinline__ void build_index(const Index& ix, const int32_t* s_tok, uint32_t j0, uint32_t spt, bool own,
                                             uint32_t* s_fill, uint32_t* status)
 {
     uint32_t live = 0;
-    if (own) {
+    int32_t x[MAX_SPT], old[MAX_SPT];
+    uint32_t b[MAX_SPT];
 #pragma unroll
-        for (uint32_t k = 0; k < (uint32_t)MAX_SPT; ++k) {
-            if (k < spt) {
-                const int32_t x = s_tok[j0 + k];
-                if (x >= 0) { index_insert(ix, x, j0 + k, status); ++live; }
+    for (uint32_t k = 0; k < (uint32_t)MAX_SPT; ++k) {
+        x[k] = (own && k < spt) ? s_tok[j0 + k] : -1;
+        if (x[k] >= 0) {
+            b[k] = hash_id(x[k], ix.logH);
+            old[k] = atomicCAS(&ix.key[b[k]], EMPTY, x[k]);
+            ++live;
+        }
+    }
+#pragma unroll
+    for (uint32_t k = 0; k < (uint32_t)MAX_SPT; ++k) {
+        if (x[k] >= 0) {
+            if (old[k] == EMPTY || old[k] == x[k]) {
+                ix.val[b[k]] = (uint16_t)(j0 + k);
+            } else {
+                uint32_t bb = (b[k] + 1u) & ix.mask;
+                bool done = false;
+                for (uint32_t it = 0; it < ix.mask; ++it) {
+                    const int32_t o = atomicCAS(&ix.key[bb], EMPTY, x[k]);
+                    if (o == EMPTY || o == x[k]) { ix.val[bb] = (uint16_t)(j0 + k); done = true; break; }
+                    bb = (bb + 1u) & ix.mask;
+                }
+                if (!done) atomicOr(status, ST_PROBE_EXHAUSTED);
             }
         }
     }
@@ -144,11 +168,74 @@ __device__ __forceinline__ void build_index(const Index& ix, const int32_t* s_to
     if ((threadIdx.x & 31u) == 0 && live) atomicAdd(s_fill, live);
 }
 
+// The ids a thread handles for one token: positions i0 .. i0+ipt-1.
+__device__ __forceinline__ void load_ids(const int32_t* X, uint32_t i0, uint32_t ipt, uint32_t K, int32_t (&xs)[MAX_IPT])
+{
+    if ((ipt & 3u) == 0 && (K & 3u) == 0 && ((reinterpret_cast<uintptr_t>(X) & 15u) == 0)) {
+#pragma unroll
+        for (uint32_t q = 0; q < (uint32_t)MAX_IPT / 4; ++q) {
+            if (4 * q < ipt && i0 + 4 * q < K) {
+                const int4 v = __ldg(reinterpret_cast<const int4*>(X + i0) + q);
+                xs[4 * q] = v.x; xs[4 * q + 1] = v.y; xs[4 * q + 2] = v.z; xs[4 * q + 3] = v.w;
+            }
+        }
+    } else if (ipt == 2 && (K & 1u) == 0 && ((reinterpret_cast<uintptr_t>(X) & 7u) == 0)) {
+        if (i0 < K) {
+            const int2 v = __ldg(reinterpret_cast<const int2*>(X + i0));
+            xs[0] = v.x; xs[1] = v.y;
+        }
+    } else {
+#pragma unroll
+        for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k)
+            if (k < ipt && i0 + k < K) xs[k] = __ldg(X + i0 + k);
+    }
+}
+
+// Lifetime histogram of the table: s_hist[v + 1] = number of slots with lifetime v, v = -1 .. L.
+// s_hist must be zero on entry.  w0/w1 are the thread's packed lifetimes (life_load).
+__device__ __forceinline__ void count_lifetimes(uint32_t w0, uint32_t w1, uint32_t spt, bool own, int32_t L,
+                                                uint8_t* s_priv, uint32_t priv_stride, uint32_t* s_hist)
+{
+    const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31u;
+    if (s_priv) {
+        // private byte counters: row = lifetime value + 1, column = thread; no atomics
+        if (own) {
+#pragma unroll
+            for (uint32_t k = 0; k < (uint32_t)MAX_SPT; ++k) {
+                if (k < spt) {
+                    const uint32_t byte = ((k < 4 ? w0 >> (8 * k) : w1 >> (8 * (k - 4))) + 1u) & 0xFFu;   // value + 1
+                    s_priv[byte * priv_stride + tid] += 1;
+                }
+            }
+        }
+        __syncthreads();
+        // one warp per row: sum nt byte counters with dp4a and clear them for the next use
+        const uint32_t words = nt >> 2;
+        for (uint32_t row = tid >> 5; row <= (uint32_t)L + 1u; row += nt >> 5) {
+            uint32_t* r = reinterpret_cast<uint32_t*>(s_priv + row * priv_stride);
+            uint32_t acc = 0;
+            for (uint32_t i = lane; i < words; i += 32u) {
+                acc = __dp4a(r[i], 0x01010101u, acc);
+                r[i] = 0;
+            }
+            acc = __reduce_add_sync(0xffffffffu, acc);
+            if (lane == 0) s_hist[row] = acc;
+        }
+    } else {
+        for (int32_t v = -1; v <= L; ++v) {
+            const uint32_t vv = (uint32_t)(v & 0xFF) * 0x01010101u;
+            uint32_t c = (__popc(__vcmpeq4(w0, vv)) + __popc(__vcmpeq4(w1, vv))) >> 3;
+            c = __reduce_add_sync(0xffffffffu, c);
+            if (lane == 0 && c) atomicAdd(&s_hist[v + 1], c);
+        }
+    }
+}
+
 __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_constant__ S1Params p)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     const uint32_t S = p.S, K = p.K, H = 1u << p.logH, Kp = (K + 7u) & ~7u;
-    const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31u;
+    const uint32_t tid = threadIdx.x, nt = blockDim.x;
     const int32_t L = (int32_t)p.L;
 
     int32_t*  s_tok      = reinterpret_cast<int32_t*>(smem);
@@ -162,6 +249,8 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
     uint32_t* s_scan_a   = s_hist + 128;
     uint32_t* s_scan_b   = s_scan_a + 40;
     uint32_t* s_fill     = s_scan_b + 40;
+    const uint32_t priv_stride = nt + 4u;                 // +4: rows start in different banks
+    uint8_t*  s_priv     = L <= PRIV_HIST_MAX_L ? reinterpret_cast<uint8_t*>(s_fill + 8) : nullptr;
 
     const uint32_t ti = p.first + blockIdx.x;            // table index within the call
     const uint32_t table = p.table_id[blockIdx.x];
@@ -176,22 +265,43 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
 
     Index ix{s_key, s_val, s_tok, H - 1u, p.logH};
 
-    // ---- load the table; global pre-decay of the iteration's first token (Alg. 1 Pass 1) ----
+    // ---- issue every global load first: table state and the first token's ids ----
+    int4 t4[MAX_SPT / 4];
+    int32_t t1[3];
+    uint32_t lw0, lw1;
+    if (own) {
+        if ((spt & 3u) == 0) {
+#pragma unroll
+            for (uint32_t q = 0; q < (uint32_t)MAX_SPT / 4; ++q)
+                if (q < spt / 4) t4[q] = __ldg(reinterpret_cast<const int4*>(g_tok + j0) + q);
+        } else {
+#pragma unroll
+            for (uint32_t k = 0; k < 3; ++k)
+                if (k < spt) t1[k] = __ldg(g_tok + j0 + k);
+        }
+    }
+    life_load(g_life, j0, spt, own, lw0, lw1);
+    int32_t xs[MAX_IPT];
+    load_ids(p.indices + (size_t)ti * p.n_q * K, i0, ipt, K, xs);
+
     for (uint32_t i = tid; i < H / 4; i += nt) reinterpret_cast<int4*>(s_key)[i] = make_int4(EMPTY, EMPTY, EMPTY, EMPTY);
+    if (s_priv)
+        for (uint32_t i = tid; i < ((uint32_t)(L + 2) * priv_stride + 15u) / 16u; i += nt)
+            reinterpret_cast<int4*>(s_priv)[i] = make_int4(0, 0, 0, 0);
     if (tid == 0) *s_fill = 0;
     if (own) {
         if ((spt & 3u) == 0) {
-            for (uint32_t q = 0; q < spt / 4; ++q)
-                reinterpret_cast<int4*>(s_tok + j0)[q] = __ldg(reinterpret_cast<const int4*>(g_tok + j0) + q);
+#pragma unroll
+            for (uint32_t q = 0; q < (uint32_t)MAX_SPT / 4; ++q)
+                if (q < spt / 4) reinterpret_cast<int4*>(s_tok + j0)[q] = t4[q];
         } else {
-            for (uint32_t k = 0; k < spt; ++k) s_tok[j0 + k] = __ldg(g_tok + j0 + k);
+#pragma unroll
+            for (uint32_t k = 0; k < 3; ++k)
+                if (k < spt) s_tok[j0 + k] = t1[k];
         }
     }
-    {
-        uint32_t w0, w1;
-        life_load(g_life, j0, spt, own, w0, w1);
-        life_store(s_life, j0, spt, own, decay4(w0, 1), decay4(w1, 1));
-    }
+    // global pre-decay of the iteration's first token (Alg. 1 Pass 1)
+    life_store(s_life, j0, spt, own, decay4(lw0, 1), decay4(lw1, 1));
     __syncthreads();
     build_index(ix, s_tok, j0, spt, own, s_fill, p.status);
     __syncthreads();
@@ -202,20 +312,17 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
 
     for (uint32_t g = 0; g < p.n_q; ++g) {
         const size_t row = ((size_t)ti * p.n_q + g) * K;
-        const int32_t* X = p.indices + row;
         int32_t* O = p.slots + row;
         uint8_t* Hm = p.hit ? p.hit + row : nullptr;
         if (tid < 128) s_hist[tid] = 0;
 
         // ---- Probe, refresh hits to L, emit hit slots (Pass 1 + Pass 2) ----
-        int32_t xs[MAX_IPT];
         uint32_t missmask = 0, nmiss = 0, nvalid = 0;
 #pragma unroll
         for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {
             const uint32_t i = i0 + k;
             if (k < ipt && i < K) {
-                const int32_t x = __ldg(X + i);
-                xs[k] = x;
+                const int32_t x = xs[k];
                 if (x >= 0) {
                     ++nvalid;
                     const int32_t j = index_find(ix, x, p.status);
@@ -247,6 +354,8 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
                 ++off;
             }
         }
+        // the next token's ids travel while this token's misses are placed
+        if (g + 1 < p.n_q) load_ids(p.indices + row + K, i0, ipt, K, xs);
         if (tid == 0 && p.miss_count) p.miss_count[(size_t)ti * p.n_q + g] = (int32_t)n_g;
         if (n_g == 0) { __syncthreads(); continue; }
         __syncthreads();
@@ -254,12 +363,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
         // ---- Pass 3: how many unit decays until n_g slots are dead ----
         uint32_t w0, w1;
         life_load(s_life, j0, spt, own, w0, w1);
-        for (int32_t v = -1; v <= L; ++v) {
-            const uint32_t vv = (uint32_t)(v & 0xFF) * 0x01010101u;
-            uint32_t c = (__popc(__vcmpeq4(w0, vv)) + __popc(__vcmpeq4(w1, vv))) >> 3;
-            c = __reduce_add_sync(0xffffffffu, c);
-            if (lane == 0 && c) atomicAdd(&s_hist[v + 1], c);
-        }
+        count_lifetimes(w0, w1, spt, own, L, s_priv, priv_stride, s_hist);
         __syncthreads();
         uint32_t d = (uint32_t)L + 1u, cum = 0;
         bool found = false;
@@ -403,10 +507,12 @@ __global__ void __launch_bounds__(256) avsg_all_k_prepare_kernel(const __grid_co
 
 }  // namespace
 
-size_t stage_one_smem_bytes(uint32_t S, uint32_t K)
+size_t stage_one_smem_bytes(uint32_t S, uint32_t K, uint32_t L)
 {
     const size_t H = 2ull * S, Kp = (K + 7u) & ~7u;
-    return S * 4 + H * 4 + Kp * 4 + H * 2 + Kp * 2 + Kp * 2 + S + (128 + 40 + 40 + 8) * 4;
+    size_t n = S * 4 + H * 4 + Kp * 4 + H * 2 + Kp * 2 + Kp * 2 + S + (128 + 40 + 40 + 8) * 4;
+    if ((int32_t)L <= PRIV_HIST_MAX_L) n += ((size_t)(L + 2) * (stage_one_threads(S, K) + 4) + 15) / 16 * 16;
+    return n;
 }
 
 uint32_t stage_one_threads(uint32_t S, uint32_t K)
@@ -426,7 +532,7 @@ cudaError_t stage_one_prepare(size_t max_smem)
 cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream)
 {
     const uint32_t threads = stage_one_threads(p.S, p.K);
-    avsg_stage_one_kernel<<<n_tables, threads, stage_one_smem_bytes(p.S, p.K), stream>>>(p);
+    avsg_stage_one_kernel<<<n_tables, threads, stage_one_smem_bytes(p.S, p.K, p.L), stream>>>(p);
     return cudaGetLastError();
 }
 
