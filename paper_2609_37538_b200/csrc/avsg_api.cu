@@ -269,7 +269,9 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device);
     const size_t need = stage_one_smem_bytes(cfg->buffer_slots, cfg->max_topk, (uint32_t)cfg->max_lifetime);
     if (need > (size_t)max_smem) { delete c; return AVSG_EUNSUPPORTED; }
-    if (stage_one_prepare(need) != cudaSuccess) { delete c; return AVSG_ECUDA; }
+    // always raise the kernel's dynamic shared-memory limit to the device maximum: the attribute is
+    // per function, so a context with a small table must not lower it under a context with a large one
+    if (stage_one_prepare((size_t)max_smem) != cudaSuccess) { delete c; return AVSG_ECUDA; }
 
     const size_t n_ids = T * c->list_stride;
     bool ok = true;

@@ -222,3 +222,18 @@ def test_argument_errors(avsg):
         avsg.Context(1, 64, 32, 40, 2, 4)                                # Eq. 7 at create
     assert e.value.code == avsg.ECAPACITY
     assert ctx.sync_status() == 0
+
+
+def test_small_context_created_after_a_large_one_does_not_break_it(avsg):
+    import torch
+    rb = 32
+    kv = avsg.pinned_empty(20000 * rb)
+    tr.fill_kv(kv.data_ptr(), 5, 0, 20000, rb)
+    big = avsg.Context(1, 8192, rb, 2048, 2, 16)
+    small = avsg.Context(1, 64, rb, 16, 1, 16)
+    Xs = torch.arange(16, dtype=torch.int32, device="cuda").reshape(1, 1, 16)
+    small.step([0], Xs, [kv], [20000])
+    Xb = torch.arange(4096, dtype=torch.int32, device="cuda").reshape(1, 2, 2048) * 3
+    out = big.step([0], Xb, [kv], [20000])                   # must still launch with its large shared memory
+    torch.cuda.synchronize()
+    assert out.miss_count.cpu().numpy().sum() == 4096 and big.sync_status() == 0
