@@ -149,6 +149,64 @@ int avsg_set_timing(avsg_ctx *ctx, int enable);
 /* Stage Two geometry: thread blocks (0 = one per SM) and threads per block. */
 int avsg_set_transfer_geometry(avsg_ctx *ctx, uint32_t blocks, uint32_t threads);
 
+/*
+ * avsg_step_noalloc - the same decode iteration for callers that cannot
+ * allocate.  (The paper has no counterpart; this is a deployment aid.)
+ *
+ * Who needs it: a serving engine that hands all free device memory to its own
+ * pool at start-up, so that any later cudaMalloc fails, or a caller on a
+ * latency-critical path where an allocation (which may synchronise the whole
+ * device) is not acceptable.  There is no context object: the caller owns the
+ * table state and passes it in on every call, and the library allocates
+ * nothing - no cudaMalloc, cudaFree or allocating library routine is called.
+ * The scratch the step needs (miss list, per-table segment descriptors,
+ * counters, status word) is a fixed array of about 1 MiB inside the library
+ * image; every GPU that loads the library holds it until the process exits.
+ *
+ * Limits (AVSG_EUNSUPPORTED beyond them): n <= AVSG_NOALLOC_MAX_TABLES,
+ * n * n_tokens * topk <= AVSG_NOALLOC_MAX_IDS, buffer_slots <= 8192.
+ * buffer_slots < n_tokens * topk returns AVSG_ECAPACITY.
+ *
+ * Runs on the CURRENT device, asynchronously on cuda_stream.  The first call
+ * on a device also looks up the device address of the scratch array and sets
+ * the kernel's shared-memory limit; make that first call outside any stream
+ * capture.  All calls on a device share the one scratch array: calls that
+ * overlap on the GPU (two streams, or two host threads) race on it, so keep
+ * them on one stream or order them yourself.  The array keeps the previous
+ * call's contents; the library clears what has to start at zero.
+ *
+ * State layout (caller-owned DEVICE memory, table i at index i):
+ *   tok    int32 [n][buffer_slots]  cached id per slot; a new table is all -1
+ *   life   int8  [n][buffer_slots]  lifetime per slot;  a new table is all -1
+ *   buffer bytes [n][buffer_slots * row_bytes]  the KV rows attention reads
+ * Results are the same, bit for bit, as avsg_step on a context in the same
+ * state.
+ */
+#define AVSG_NOALLOC_MAX_TABLES 32u
+#define AVSG_NOALLOC_MAX_IDS    131072u   /* n * n_tokens * topk of one call */
+
+typedef struct {
+    uint32_t        n;             /* tables in this call                                */
+    uint32_t        n_tokens;      /* N_q                                                */
+    uint32_t        topk;          /* K                                                  */
+    uint32_t        buffer_slots;  /* S: power of two, 32 .. 8192                        */
+    uint32_t        row_bytes;     /* multiple of 16                                     */
+    int32_t         max_lifetime;  /* L in 1 .. 126                                      */
+    int32_t        *tok;           /* DEVICE in/out [n][S]                               */
+    int8_t         *life;          /* DEVICE in/out [n][S]                               */
+    void           *buffer;        /* DEVICE in/out [n][S * row_bytes]                   */
+    const int32_t  *indices;       /* DEVICE [n][n_tokens][topk]                         */
+    const void *const *kv_base;    /* HOST [n]: pinned host KV base per table            */
+    const uint64_t *row_stride;    /* HOST [n] or NULL (= row_bytes)                     */
+    const int32_t  *verified_len;  /* HOST [n]                                           */
+    int32_t        *slots;         /* DEVICE out [n][n_tokens][topk]                     */
+    uint8_t        *hit;           /* DEVICE out or NULL                                 */
+    int32_t        *miss_count;    /* DEVICE out [n][n_tokens] or NULL                   */
+    uint32_t       *status;        /* DEVICE out or NULL: 0, or the kernels' status bits */
+} avsg_noalloc_args;
+
+int avsg_step_noalloc(const avsg_noalloc_args *args, void *cuda_stream);
+
 const char *avsg_strerror(int code);
 
 #ifdef __cplusplus

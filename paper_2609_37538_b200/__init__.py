@@ -4,4 +4,5 @@ from .binding import (  # noqa: F401
     XFER_ALL_K, XFER_COPY_ENGINE, XFER_REQUEST_LEVEL, XFER_SM_BALANCED,
     AvsgConfig, AvsgError, AvsgStats, AvsgStepArgs, Context, PreparedCall, StepOutput,
     load_library, pinned_empty,
+    AvsgNoAllocArgs, NOALLOC_MAX_IDS, NOALLOC_MAX_TABLES, step_noalloc,
 )

@@ -22,6 +22,7 @@ EXPORTS = (
     "avsg_create", "avsg_destroy", "avsg_reset", "avsg_step", "avsg_step_host", "avsg_buffer", "avsg_stats",
     "avsg_sync_status", "avsg_export_state", "avsg_import_state", "avsg_save_state", "avsg_restore_state",
     "avsg_set_transfer_mode", "avsg_set_timing", "avsg_set_transfer_geometry", "avsg_strerror",
+    "avsg_step_noalloc",
 )
 
 
@@ -43,6 +44,18 @@ class AvsgStats(ctypes.Structure):
                 ("misses", ctypes.c_uint64), ("rows_copied", ctypes.c_uint64), ("bytes_copied", ctypes.c_uint64),
                 ("extra_decays", ctypes.c_uint64), ("last_stage_one_us", ctypes.c_float),
                 ("last_transfer_us", ctypes.c_float), ("last_rows", ctypes.c_uint64)]
+
+
+class AvsgNoAllocArgs(ctypes.Structure):
+    _fields_ = [("n", ctypes.c_uint32), ("n_tokens", ctypes.c_uint32), ("topk", ctypes.c_uint32),
+                ("buffer_slots", ctypes.c_uint32), ("row_bytes", ctypes.c_uint32), ("max_lifetime", ctypes.c_int32),
+                ("tok", ctypes.c_void_p), ("life", ctypes.c_void_p), ("buffer", ctypes.c_void_p),
+                ("indices", ctypes.c_void_p), ("kv_base", ctypes.c_void_p), ("row_stride", ctypes.c_void_p),
+                ("verified_len", ctypes.c_void_p), ("slots", ctypes.c_void_p), ("hit", ctypes.c_void_p),
+                ("miss_count", ctypes.c_void_p), ("status", ctypes.c_void_p)]
+
+
+NOALLOC_MAX_TABLES, NOALLOC_MAX_IDS = 32, 131072
 
 
 class AvsgError(RuntimeError):
@@ -80,6 +93,7 @@ def load_library():
     lib.avsg_set_timing.argtypes, lib.avsg_set_timing.restype = [vp, i32], i32
     lib.avsg_set_transfer_geometry.argtypes, lib.avsg_set_transfer_geometry.restype = [vp, u32, u32], i32
     lib.avsg_strerror.argtypes, lib.avsg_strerror.restype = [i32], ctypes.c_char_p
+    lib.avsg_step_noalloc.argtypes, lib.avsg_step_noalloc.restype = [ctypes.POINTER(AvsgNoAllocArgs), vp], i32
     _lib = lib
     return lib
 
@@ -269,3 +283,33 @@ class Context:
         s = AvsgStats()
         _check(self._lib.avsg_stats(self._h, ctypes.byref(s)), "avsg_stats")
         return {name: getattr(s, name) for name, _ in AvsgStats._fields_}
+
+
+def step_noalloc(tok, life, buffer, indices, kv, verified_len, *, max_lifetime: int = 16, slots, hit=None,
+                 miss_count=None, status=None, row_stride=None, stream=None) -> None:
+    """avsg_step_noalloc: one decode iteration on caller-owned state, for callers that cannot allocate
+    (an engine whose own pool holds all device memory, or a path where an allocation's device-wide
+    synchronisation is not acceptable).  Every tensor is the caller's; the library allocates nothing and
+    keeps its scratch in a fixed array inside the library image.
+
+    tok int32 [n, S], life int8 [n, S], buffer uint8 [n, S, row_bytes], indices int32 [n, n_tokens, topk],
+    slots int32 like indices: CUDA tensors on the current device.  kv: one pinned host tensor (or address) per
+    table.  Calls that overlap on the GPU race on the shared scratch: keep them on one stream.
+    """
+    n, S = tok.shape
+    _, n_q, K = indices.shape
+    kv_arr = (ctypes.c_void_p * n)(*[_addr(k) for k in kv])
+    vlen = (ctypes.c_int32 * n)(*[int(v) for v in verified_len])
+    stride = (ctypes.c_uint64 * n)(*[int(s) for s in row_stride]) if row_stride is not None else None
+    a = AvsgNoAllocArgs()
+    a.n, a.n_tokens, a.topk, a.buffer_slots = n, n_q, K, S
+    a.row_bytes, a.max_lifetime = buffer.shape[-1], max_lifetime
+    a.tok, a.life, a.buffer, a.indices = _addr(tok), _addr(life), _addr(buffer), _addr(indices)
+    a.kv_base = ctypes.addressof(kv_arr)
+    a.row_stride = ctypes.addressof(stride) if stride is not None else None
+    a.verified_len = ctypes.addressof(vlen)
+    a.slots = _addr(slots)
+    a.hit = _addr(hit) if hit is not None else None
+    a.miss_count = _addr(miss_count) if miss_count is not None else None
+    a.status = _addr(status) if status is not None else None
+    _check(load_library().avsg_step_noalloc(ctypes.byref(a), _stream_handle(stream)), "avsg_step_noalloc")
