@@ -406,6 +406,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
                 list[list_off + k] = make_int2(x, (int32_t)j);
                 if (!rebuild) index_insert(ix, x, j, p.status);
             } else {
+                list[list_off + k] = make_int2(-1, -1);          // Stage Two skips it
                 atomicOr(p.status, ST_BAD_SLOT);
             }
         }
