@@ -219,15 +219,17 @@ def run_cuda(args):
     w = _workload(rank, n_iters, args)
     traces = _gen_traces(w, threads)
     kv = []
+    stride = args.row_stride or w.row_bytes
     for ti, cfg in enumerate(w.tables):
-        buf = avsg.pinned_empty(cfg.context * w.row_bytes)
-        tr.fill_kv(buf.data_ptr(), w.seed, ti, cfg.context, w.row_bytes)
+        buf = avsg.pinned_empty(cfg.context * stride)
+        tr.fill_kv(buf.data_ptr(), w.seed, ti, cfg.context, w.row_bytes, row_stride=stride)
         kv.append(buf)
 
     ctx = avsg.Context(num_tables=w.num_tables, buffer_slots=w.buffer_slots, row_bytes=w.row_bytes,
                        max_topk=w.topk, max_tokens=w.n_q, max_lifetime=w.max_lifetime, device=local)
     ncalls = len(w.calls)
-    calls = [ctx.prepare(grp, [kv[t] for t in grp], w.n_q, w.topk) for grp in w.calls]
+    calls = [ctx.prepare(grp, [kv[t] for t in grp], w.n_q, w.topk,
+                         [stride] * len(grp) if args.row_stride else None) for grp in w.calls]
     # inputs resident in HBM: every iteration's ids, per call [n, n_q, K]
     Xh = [[np.stack([traces[ti][0][t] for ti in grp]) for grp in w.calls] for t in range(n_iters)]
     vlen = [[[int(traces[ti][1][t]) for ti in grp] for grp in w.calls] for t in range(n_iters)]
@@ -357,7 +359,7 @@ def run_cuda(args):
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms_j / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int32/u8", "data": "synthetic", "config": _config(w),
+        "dtype": "int32/u8", "data": "synthetic", "config": dict(_config(w), host_row_stride=stride),
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "GB/s",
                 "h2d_bytes_per_step": int(ids_bytes + rows_timed * rb / K), "d2h_bytes_per_step": int(ids_bytes + mc_bytes),
@@ -493,6 +495,67 @@ def run_suite(args):
             print(json.dumps(r2), flush=True)
 
 
+# ------------------------------------------------------------------------------------------------------------
+# --table3: the Stage Two strategies of App. D on the paper's grid (B x reuse, K = 2048, N_mtp = 0, 1152-byte rows)
+# ------------------------------------------------------------------------------------------------------------
+def run_table3(args):
+    import torch
+    import __graft_entry__
+    import avsg_traces as tr
+    __graft_entry__.build()
+    import paper_2609_37538_b200 as avsg
+    torch.cuda.set_device(0)
+    K, S, RB, CTX, B_MAX = 2048, 8192, 1152, 131072, 32
+    rng = np.random.default_rng(20260937)
+    kv = []
+    for ti in range(B_MAX):
+        buf = avsg.pinned_empty(CTX * RB)
+        tr.fill_kv(buf.data_ptr(), 33, ti, CTX, RB)
+        kv.append(buf)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    modes = (("S1_request_level", avsg.XFER_REQUEST_LEVEL), ("S2_position_level", avsg.XFER_POSITION_LEVEL),
+             ("S3_miss_level", avsg.XFER_SM_BALANCED))
+    for B in (1, 2, 4, 8, 16, 32):
+        ctx = avsg.Context(num_tables=B, buffer_slots=S, row_bytes=RB, max_topk=K, max_tokens=1, max_lifetime=16)
+        ctx.set_timing(True)
+        call = ctx.prepare(list(range(B)), kv[:B], 1, K)
+        first = np.stack([np.sort(rng.choice(CTX, K, replace=False)) for _ in range(B)]).astype(np.int32)
+        Xa = torch.from_numpy(first[:, None, :]).cuda()
+        slots = torch.empty_like(Xa)
+        call.run(Xa, [CTX] * B, slots, None, None, stream)          # cold step: the first selection becomes resident
+        ctx.save_state()
+        torch.cuda.synchronize()
+        for reuse in (0.0, 0.25, 0.5, 0.75):
+            keep = int(round(reuse * K))
+            sel = []
+            for b in range(B):
+                kept = rng.choice(first[b], keep, replace=False)
+                pool = np.setdiff1d(np.arange(CTX, dtype=np.int32), first[b])
+                sel.append(np.sort(np.concatenate([kept, rng.choice(pool, K - keep, replace=False)])))
+            Xb = torch.from_numpy(np.stack(sel).astype(np.int32)[:, None, :]).cuda()
+            row = {"table3": True, "B": B, "reuse_pct": int(reuse * 100), "rows": B * (K - keep),
+                   "bytes": B * (K - keep) * RB}
+            for name, mode in modes:
+                ctx.set_transfer_mode(mode)
+                us = []
+                for rep in range(args.replays_table3 + 2):
+                    ctx.restore_state()
+                    flush.fill_(rep)
+                    call.run(Xb, [CTX] * B, slots, None, None, stream)
+                    st = ctx.stats()
+                    if rep >= 2:
+                        us.append(st["last_transfer_us"])
+                    assert st["last_rows"] == B * (K - keep) or rep == 0
+                med = statistics.median(us)
+                row[name + "_us"] = med
+                row[name + "_gbs"] = row["bytes"] / 1e3 / med
+            row["S3_over_S1"] = row["S3_miss_level_gbs"] / row["S1_request_level_gbs"]
+            row["S3_over_S2"] = row["S3_miss_level_gbs"] / row["S2_position_level_gbs"]
+            print(json.dumps(row), flush=True)
+        ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -503,12 +566,19 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--requests", type=int, default=32, help="requests per layer (32 = the full configuration)")
     ap.add_argument("--layers", type=int, default=4, help="layers (4 = the full configuration)")
+    ap.add_argument("--row-stride", type=int, default=0,
+                    help="bytes between host KV rows (0 = packed, 656); e.g. 768 pads rows to 128-byte lines")
+    ap.add_argument("--table3", action="store_true",
+                    help="extra report: Stage Two strategies S1/S2/S3 on the paper's B x reuse grid (1 GPU)")
+    ap.add_argument("--replays-table3", type=int, default=9)
     ap.add_argument("--suite", action="store_true",
                     help="extra report: C1..C5 hit rates, per-call times and the Stage Two comparators (1 GPU)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.suite:
+    if args.table3:
+        run_table3(args)
+    elif args.suite:
         run_suite(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -51,6 +51,10 @@ extern "C" {
 #define AVSG_XFER_REQUEST_LEVEL 2u  /* comparator S1: one thread block per request       */
 #define AVSG_XFER_ALL_K         3u  /* comparator "KV offload": no reuse, all n_tokens*K
                                        rows move; position (g,i) -> slot g*K+i           */
+#define AVSG_XFER_POSITION_LEVEL 4u /* comparator S2 (Eq. 14): all top-K positions of the
+                                       call are cut into equal ranges, one per thread
+                                       block, which walks its range and copies the misses;
+                                       hit positions are visited for nothing             */
 
 typedef struct avsg_ctx avsg_ctx;   /* opaque */
 

@@ -53,6 +53,8 @@ def _load():
     lib.orc_partition.argtypes = [u64, u32, u32, vp, vp]
     lib.orc_partition.restype = None
     lib.orc_requests_of_core.argtypes, lib.orc_requests_of_core.restype = [u32, u32, u32], u32
+    lib.orc_position_range.argtypes, lib.orc_position_range.restype = [u64, u32, u32, vp, vp], None
+    lib.orc_workload.argtypes, lib.orc_workload.restype = [vp, vp, u64, u64], u64
     lib.orc_export.argtypes, lib.orc_export.restype = [vp, vp, vp], None
     lib.orc_import.argtypes, lib.orc_import.restype = [vp, vp, vp], None
     lib.orc_rows.argtypes, lib.orc_rows.restype = [vp], vp
@@ -188,3 +190,17 @@ def partition(n_miss: int, C: int, c: int) -> Tuple[int, int]:
 def requests_of_core(B: int, C: int, c: int) -> int:
     """Eq. 13: number of requests core c serves under request-level assignment."""
     return _load().orc_requests_of_core(B, C, c)
+
+
+def position_range(n_positions: int, C: int, c: int) -> Tuple[int, int]:
+    """Eq. 14: the [begin, end) range of flattened top-K positions that core c walks (hits included)."""
+    b, e = ctypes.c_uint64(0), ctypes.c_uint64(0)
+    _load().orc_position_range(n_positions, C, c, ctypes.byref(b), ctypes.byref(e))
+    return b.value, e.value
+
+
+def workload(M: np.ndarray, X: np.ndarray, begin: int, end: int) -> int:
+    """Eq. 5: number of rows a core moves for the flattened positions [begin, end)."""
+    M = np.ascontiguousarray(M, dtype=np.uint8).ravel()
+    X = np.ascontiguousarray(X, dtype=np.int32).ravel()
+    return int(_load().orc_workload(M.ctypes.data, X.ctypes.data, begin, end))

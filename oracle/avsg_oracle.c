@@ -14,6 +14,7 @@
  *   - MTP sequencing + invalidation .... Algorithm 4
  *   - balanced miss partition .......... Eq. 6, Sec. 3.4
  *   - request-level assignment ......... Eq. 13 (comparator S1)
+ *   - equal top-K position partition ... Eq. 14 (comparator S2)
  *
  * Readings taken where the paper is silent or ambiguous (all listed in the
  * design notes of the repository):
@@ -249,6 +250,24 @@ void orc_partition(uint64_t n_miss, uint32_t C, uint32_t c, uint64_t *begin, uin
 uint32_t orc_requests_of_core(uint32_t B, uint32_t C, uint32_t c)
 {
     return B / C + (c < B % C ? 1u : 0u);
+}
+
+/* Eq. 14: equal top-K position partitioning; core c takes the flattened
+ * positions floor(c*NgK/C) <= gK+i < floor((c+1)*NgK/C), hits included. */
+void orc_position_range(uint64_t n_positions, uint32_t C, uint32_t c, uint64_t *begin, uint64_t *end)
+{
+    *begin = (uint64_t)c * n_positions / C;
+    *end = (uint64_t)(c + 1) * n_positions / C;
+}
+
+/* Eq. 5: transfer workload of a set of positions = the misses among them.
+ * m[] is the hit mask over the flattened positions; padding counts as no work. */
+uint64_t orc_workload(const uint8_t *m, const int32_t *x, uint64_t begin, uint64_t end)
+{
+    uint64_t w = 0;
+    for (uint64_t p = begin; p < end; ++p)
+        if (x[p] >= 0) w += 1u - m[p];
+    return w;
 }
 
 /* accessors for the Python test harness */

@@ -16,7 +16,7 @@ import numpy as np
 from . import build as _build
 
 OK, EINVAL, ENOMEM, ECUDA, ECAPACITY, EDEVICE_STATUS, EUNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
-XFER_SM_BALANCED, XFER_COPY_ENGINE, XFER_REQUEST_LEVEL, XFER_ALL_K = 0, 1, 2, 3
+XFER_SM_BALANCED, XFER_COPY_ENGINE, XFER_REQUEST_LEVEL, XFER_ALL_K, XFER_POSITION_LEVEL = 0, 1, 2, 3, 4
 
 EXPORTS = (
     "avsg_create", "avsg_destroy", "avsg_reset", "avsg_step", "avsg_step_host", "avsg_buffer", "avsg_stats",

@@ -170,9 +170,11 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         hit = a->hit ? c->d_hit_stage : nullptr;
         miss_count = a->miss_count ? c->d_mc_stage : nullptr;
     }
+    const uint32_t mode = c->cfg.transfer_mode;
+    // the position-level comparator reads the hit mask: use the library's own buffer if the caller wants none
+    if (mode == AVSG_XFER_POSITION_LEVEL && !hit) hit = c->d_hit_stage;
     if (c->timing) CU(cudaEventRecord(c->ev[0], stream));
 
-    const uint32_t mode = c->cfg.transfer_mode;
     c->call_kv_host.assign(a->kv_base, a->kv_base + n);
     for (uint32_t first = 0; first < n; first += S1_MAX_TABLES) {
         const uint32_t cnt = n - first < (uint32_t)S1_MAX_TABLES ? n - first : (uint32_t)S1_MAX_TABLES;
@@ -209,6 +211,11 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
 
     if (mode == AVSG_XFER_COPY_ENGINE) {
         if ((rc = copy_engine_transfer(c, a, stream)) != AVSG_OK) return rc;
+    } else if (mode == AVSG_XFER_POSITION_LEVEL) {
+        PosParams q;
+        q.seg = c->d_seg; q.indices = indices; q.slots = slots; q.hit = hit; q.status = c->d_status;
+        q.n = n; q.per_table = n_q * K; q.row_bytes = c->cfg.row_bytes; q.S = c->cfg.buffer_slots;
+        CU(launch_transfer_positions(q, c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count, c->xfer_threads, stream));
     } else {
         XferParams x;
         x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
@@ -248,7 +255,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     if (cfg->row_bytes == 0 || cfg->row_bytes % 16) return AVSG_EINVAL;
     if (cfg->max_topk == 0 || cfg->max_tokens == 0) return AVSG_EINVAL;
     if (cfg->max_lifetime < 1 || cfg->max_lifetime > 126) return AVSG_EINVAL;
-    if (cfg->transfer_mode > AVSG_XFER_ALL_K) return AVSG_EINVAL;
+    if (cfg->transfer_mode > AVSG_XFER_POSITION_LEVEL) return AVSG_EINVAL;
     if ((uint64_t)cfg->max_topk * cfg->max_tokens > cfg->buffer_slots) return AVSG_ECAPACITY;   // Eq. 7
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device < 0 || cfg->device >= ndev) return AVSG_ECUDA;
@@ -429,7 +436,7 @@ int avsg_restore_state(avsg_ctx* c, void* stream)
 
 int avsg_set_transfer_mode(avsg_ctx* c, uint32_t mode)
 {
-    if (!c || mode > AVSG_XFER_ALL_K) return AVSG_EINVAL;
+    if (!c || mode > AVSG_XFER_POSITION_LEVEL) return AVSG_EINVAL;
     c->cfg.transfer_mode = mode;
     return AVSG_OK;
 }

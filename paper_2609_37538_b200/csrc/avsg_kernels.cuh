@@ -61,6 +61,15 @@ struct XferParams {
     uint32_t n_seg, list_stride, row_bytes, request_level, S;
 };
 
+struct PosParams {               // comparator S2: equal top-K position partition
+    const SegDesc* seg;          // per table: host base, stride, buffer base
+    const int32_t* indices;      // [n][n_q*K]
+    const int32_t* slots;        // [n][n_q*K] (written by Stage One)
+    const uint8_t* hit;          // [n][n_q*K] (written by Stage One)
+    uint32_t*      status;
+    uint32_t n, per_table, row_bytes, S;     // per_table = n_q * K positions
+};
+
 struct AllKParams {
     const int32_t* indices;      // [n][n_q*K]
     int32_t*       slots;
@@ -82,5 +91,6 @@ cudaError_t stage_one_prepare(size_t max_smem);
 cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream);
 cudaError_t launch_all_k_prepare(const AllKParams& p, uint32_t n_tables, cudaStream_t stream);
 cudaError_t launch_transfer(const XferParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream);
+cudaError_t launch_transfer_positions(const PosParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream);
 
 }  // namespace avsg

@@ -115,7 +115,49 @@ __global__ void __launch_bounds__(1024) avsg_transfer_kernel(const __grid_consta
     }
 }
 
+// Comparator S2 (App. D, Eq. 14): the n * N_q * K selected positions of the call are flattened and cut into
+// gridDim.x near-equal contiguous ranges regardless of hit or miss; a block walks its range, one warp per
+// position, and copies the row of every position that missed.  Work per block = misses in its range (Eq. 15).
+__global__ void __launch_bounds__(1024) avsg_transfer_positions_kernel(const __grid_constant__ PosParams p)
+{
+    const uint32_t lane = threadIdx.x & 31u, warps = blockDim.x >> 5;
+    const uint64_t P = (uint64_t)p.n * p.per_table, C = gridDim.x, c = blockIdx.x;
+    const uint64_t begin = c * P / C, end = (c + 1) * P / C;
+    const uint32_t cpr = p.row_bytes >> 4;
+    for (uint64_t q = begin + (threadIdx.x >> 5); q < end; q += warps) {
+        const int32_t x = __ldg(p.indices + q);
+        if (x < 0 || __ldg(p.hit + q)) continue;                 // padding or hit: nothing to move
+        const int32_t o = __ldg(p.slots + q);
+        if (o < 0 || (uint32_t)o >= p.S) {
+            if (lane == 0) atomicOr(p.status, ST_BAD_SLOT);
+            continue;
+        }
+        const uint32_t ti = (uint32_t)(q / p.per_table);
+        const uint64_t src = __ldg(&p.seg[ti].src_base) + (uint64_t)(uint32_t)x * __ldg(&p.seg[ti].src_stride);
+        const uint64_t dst = __ldg(&p.seg[ti].dst_base) + (uint64_t)(uint32_t)o * p.row_bytes;
+        for (uint32_t c0 = lane; c0 < cpr; c0 += 32u * CHUNKS_PER_PASS) {
+            int4 v[CHUNKS_PER_PASS];
+#pragma unroll
+            for (int k = 0; k < CHUNKS_PER_PASS; ++k) {
+                const uint32_t cc = c0 + 32u * k;
+                if (cc < cpr) v[k] = *reinterpret_cast<const int4*>(src + 16ull * cc);
+            }
+#pragma unroll
+            for (int k = 0; k < CHUNKS_PER_PASS; ++k) {
+                const uint32_t cc = c0 + 32u * k;
+                if (cc < cpr) *reinterpret_cast<int4*>(dst + 16ull * cc) = v[k];
+            }
+        }
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_transfer_positions(const PosParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream)
+{
+    avsg_transfer_positions_kernel<<<blocks, threads, 0, stream>>>(p);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_transfer(const XferParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream)
 {

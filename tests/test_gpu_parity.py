@@ -53,10 +53,18 @@ def test_c5_full_balanced(avsg):
     assert r["gpu"]["tokens"] == 64 * 33
 
 
-@pytest.mark.parametrize("mode_name", ["XFER_REQUEST_LEVEL", "XFER_ALL_K"])
+@pytest.mark.parametrize("mode_name", ["XFER_REQUEST_LEVEL", "XFER_ALL_K", "XFER_POSITION_LEVEL"])
 def test_c5_comparators(avsg, mode_name):
     r = _parity(tr.workload("C5", n_iters=6), mode=getattr(avsg, mode_name), buffer_every=2)
     assert r["gpu"]["rows_copied"] == r["oracle"]["rows_copied"]
+
+
+def test_position_level_comparator_with_mtp_padding_and_host_io(avsg):
+    w = tr.workload("C3", requests=5, layers=2, n_iters=8, context=32768)
+    _parity(w, mode=avsg.XFER_POSITION_LEVEL, buffer_every=2)
+    _parity(w, mode=avsg.XFER_POSITION_LEVEL, host_io=True, buffer_every=4)
+    w = tr.workload("C5", topk=128, buffer_slots=256, n_iters=6, requests=4, ctx_lo=40, ctx_hi=100)
+    _parity(w, mode=avsg.XFER_POSITION_LEVEL)
 
 
 def test_copy_engine_comparator(avsg):

@@ -10,7 +10,8 @@ import numpy as np
 import pytest
 
 import avsg_traces as tr
-from oracle import ORC_ECAPACITY, OracleError, OracleTable, partition, requests_of_core
+from oracle import (ORC_ECAPACITY, OracleError, OracleTable, partition, position_range, requests_of_core,
+                    workload)
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -397,3 +398,32 @@ def test_all_k_comparator():
     assert O.ravel().tolist() == list(range(64))
     assert (t.rows() == kv.reshape(500, rb)[X.ravel()]).all()
     assert t.counters()["rows_copied"] == 64
+
+
+# ----------------------------------------------------------------------------
+# Eq. 14 / Eq. 15: equal top-K position partitioning covers every position once, sizes differ by at most
+# one, and the work of a core is the number of misses in its range - so two cores with equal shares of
+# positions can have very different work, down to none at all for an all-hit range.
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("P,C", [(2048, 148), (65536, 148), (100, 7), (5, 8)])
+def test_position_partition(P, C):
+    ranges = [position_range(P, C, c) for c in range(C)]
+    assert ranges[0][0] == 0 and ranges[-1][1] == P
+    assert all(ranges[i][1] == ranges[i + 1][0] for i in range(C - 1))
+    sizes = [e - b for b, e in ranges]
+    assert max(sizes) - min(sizes) <= 1
+    assert [b for b, _ in ranges] == [c * P // C for c in range(C)]            # the floor formula itself
+
+
+def test_position_partition_work_is_hit_dependent():
+    K, C = 64, 4
+    X = np.arange(K, dtype=np.int32)
+    M = np.zeros(K, np.uint8)
+    M[:16] = 1                                      # the first core's whole range hits
+    work = [workload(M, X, *position_range(K, C, c)) for c in range(C)]
+    assert work == [0, 16, 16, 16] and sum(work) == int((1 - M).sum())
+    # Eq. 15: W_c - W_d = hits(d) - hits(c) for equal-sized ranges
+    hits = [int(M[slice(*position_range(K, C, c))].sum()) for c in range(C)]
+    assert all(work[c] - work[d] == hits[d] - hits[c] for c in range(C) for d in range(C))
+    Xp = X.copy(); Xp[60:] = -1                     # padding is neither work nor a hit
+    assert workload(M, Xp, *position_range(K, C, 3)) == 12
