@@ -119,7 +119,7 @@ def _gen_traces(w, threads):
 # ------------------------------------------------------------------------------------------------------------
 # reference arm: the CPU oracle on the host cores
 # ------------------------------------------------------------------------------------------------------------
-def oracle_run(w, traces, kv_np, tables, warmup, steps, threads):
+def oracle_run(w, traces, kv_np, tables, warmup, steps, threads, row_stride=None):
     """Steps the oracle over `tables` for warmup+steps iterations, one thread per table; times the last `steps`.
     Returns (seconds per step list, miss rows per step list, hits, misses)."""
     from oracle import OracleTable
@@ -127,7 +127,7 @@ def oracle_run(w, traces, kv_np, tables, warmup, steps, threads):
 
     def one(ti, t):
         X, N = traces[ti]
-        r = orc[ti].step(X[t], int(N[t]), kv_np[ti])
+        r = orc[ti].step(X[t], int(N[t]), kv_np[ti], row_stride)
         return int(r.n.sum()), int(r.M.sum())
 
     secs, rows, hits, misses = [], [], 0, 0
@@ -326,16 +326,11 @@ def run_cuda(args):
     ctx.set_timing(False)
 
     # ---- aggregate over ranks: device time = max over ranks, work = sum over ranks ----
-    if world > 1:
-        tmax = torch.tensor([total_ms, e2e_ms, sum(x_us)], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        tsum = torch.tensor([rows_timed, sum(x_rows), hits_timed, miss_timed], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
-        total_ms_j, e2e_ms_j, xus_j = tmax.tolist()
-        rows_j, xrows_j, hits_j, miss_j = tsum.tolist()
-    else:
-        total_ms_j, e2e_ms_j, xus_j = total_ms, e2e_ms, sum(x_us)
-        rows_j, xrows_j, hits_j, miss_j = rows_timed, sum(x_rows), hits_timed, miss_timed
+    from paper_2609_37538_b200.sharding import aggregate
+    tmax, tsum = aggregate({"total_ms": total_ms, "e2e_ms": e2e_ms, "xus": sum(x_us)},
+                           {"rows": rows_timed, "xrows": sum(x_rows), "hits": hits_timed, "misses": miss_timed})
+    total_ms_j, e2e_ms_j, xus_j = tmax["total_ms"], tmax["e2e_ms"], tmax["xus"]
+    rows_j, xrows_j, hits_j, miss_j = tsum["rows"], tsum["xrows"], tsum["hits"], tsum["misses"]
 
     if rank != 0:
         if world > 1:
@@ -394,7 +389,7 @@ def run_cuda(args):
         kv_np = [k.numpy() for k in kv]
         cb_steps = min(16, K)
         tables = list(range(w.num_tables))
-        secs, rows, _, _ = oracle_run(w, traces, kv_np, tables, W, cb_steps, cores)
+        secs, rows, _, _ = oracle_run(w, traces, kv_np, tables, W, cb_steps, cores, stride)
         line["cpu_baseline"] = {
             "value": sum(rows) * rb / 1e9 / sum(secs), "unit": "GB/s", "cores": cores, "kind": "oracle",
             "ms_per_step": 1e3 * sum(secs) / len(secs),
