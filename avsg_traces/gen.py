@@ -51,6 +51,8 @@ class _TgConfig(ctypes.Structure):
         ("p_hot", ctypes.c_double),
         ("hot_size", ctypes.c_uint32),
         ("hot_range", ctypes.c_uint32),
+        ("p_hist", ctypes.c_double),
+        ("hist_sigma", ctypes.c_double),
     ]
 
 
@@ -94,6 +96,8 @@ class TraceConfig:
     p_hot: float = 0.0
     hot_size: int = 0
     hot_range: int = 0
+    p_hist: float = 0.0          # share of new ids re-drawn from earlier selections ("historical recall")
+    hist_sigma: float = 0.0      # per-token jitter of p_hist (normal, clipped to [0, 1])
 
     def _c(self) -> _TgConfig:
         c = _TgConfig()
@@ -106,6 +110,7 @@ class TraceConfig:
             c.rho_fixed = 0.0 if self.rho_fixed is None else float(self.rho_fixed)
         c.p_recent, c.recent_window = self.p_recent, self.recent_window
         c.p_hot, c.hot_size, c.hot_range = self.p_hot, self.hot_size, self.hot_range
+        c.p_hist, c.hist_sigma = self.p_hist, self.hist_sigma
         return c
 
 

@@ -16,7 +16,8 @@
  *   q  > 0 : keep = floor(rho*K) ids drawn without replacement from the
  *            selection of token q-1, the remaining K-keep ids drawn by
  *            rejection (distinct from everything already chosen) from a
- *            mixture of {recent window, fixed hot set, uniform};
+ *            mixture of {recent window, fixed hot set, history of earlier
+ *            selections, uniform};
  *   every selection is emitted sorted ascending, padded with -1 when the
  *   drawable range holds fewer than K ids.
  *   lim(q) = verified_len(t) + g, with verified_len(t) = context -
@@ -44,6 +45,10 @@ typedef struct {
     double   p_hot;         /* share of new ids drawn from the hot set       */
     uint32_t hot_size;      /* ids in the per-table hot set                  */
     uint32_t hot_range;     /* hot ids are distinct draws from [0,hot_range) */
+    double   p_hist;        /* share of new ids drawn from ids selected at any
+                               earlier step ("historical recall")            */
+    double   hist_sigma;    /* p_hist is redrawn per token as N(p_hist, sigma^2)
+                               clipped to [0,1] when sigma > 0               */
 } tg_config;
 
 static inline uint64_t sm64_next(uint64_t *s)
@@ -121,8 +126,13 @@ int tg_generate(const tg_config *c, int32_t *X, int32_t *verified_len)
     int32_t *prev = (int32_t *)malloc(sizeof(int32_t) * K);
     int32_t *cur = (int32_t *)malloc(sizeof(int32_t) * K);
     int32_t *hot = c->hot_size ? (int32_t *)malloc(sizeof(int32_t) * c->hot_size) : NULL;
-    if (!mark || !prev || !cur || (c->hot_size && !hot)) {
-        free(mark); free(prev); free(cur); free(hot);
+    /* history: every id selected so far, each once (seen[] marks membership) */
+    const int use_hist = c->p_hist > 0.0;
+    int32_t *hist = use_hist ? (int32_t *)malloc(sizeof(int32_t) * ((size_t)c->context + c->n_q + 1)) : NULL;
+    uint8_t *seen = use_hist ? (uint8_t *)calloc((size_t)c->context + c->n_q + 1, 1) : NULL;
+    size_t n_hist = 0;
+    if (!mark || !prev || !cur || (c->hot_size && !hot) || (use_hist && (!hist || !seen))) {
+        free(mark); free(prev); free(cur); free(hot); free(hist); free(seen);
         return -1;
     }
 
@@ -160,10 +170,27 @@ int tg_generate(const tg_config *c, int32_t *X, int32_t *verified_len)
                     mark[prev[i]] = 1;
                 }
             }
+            double p_hist = c->p_hist;
+            if (use_hist && c->hist_sigma > 0.0) {      /* Box-Muller normal, clipped to [0,1] */
+                double u1 = u01(&s), u2 = u01(&s);
+                if (u1 < 1e-300) u1 = 1e-300;
+                p_hist += c->hist_sigma * sqrt(-2.0 * log(u1)) * cos(6.283185307179586 * u2);
+                if (p_hist < 0.0) p_hist = 0.0;
+                if (p_hist > 1.0) p_hist = 1.0;
+            }
             while (n_cur < want) {
                 int32_t id = -1;
                 double comp = u01(&s);
-                if (comp < c->p_recent && c->recent_window) {
+                if (use_hist && comp < p_hist && n_hist) {
+                    for (int tries = 0; tries < 64; ++tries) {
+                        int32_t cand = hist[below(&s, n_hist)];
+                        if (cand < lim && !mark[cand]) { id = cand; break; }
+                    }
+                    comp = 2.0;                          /* the other restricted components are skipped */
+                }
+                if (id >= 0) {
+                    /* drawn from history */
+                } else if (comp < c->p_recent && c->recent_window) {
                     int64_t w = c->recent_window < lim ? c->recent_window : lim;
                     for (int tries = 0; tries < 64; ++tries) {
                         int32_t cand = (int32_t)(lim - 1 - (int64_t)below(&s, (uint64_t)w));
@@ -183,6 +210,9 @@ int tg_generate(const tg_config *c, int32_t *X, int32_t *verified_len)
                 cur[n_cur++] = id;
             }
             for (uint32_t i = 0; i < n_cur; ++i) mark[cur[i]] = 0;
+            if (use_hist)
+                for (uint32_t i = 0; i < n_cur; ++i)
+                    if (!seen[cur[i]]) { seen[cur[i]] = 1; hist[n_hist++] = cur[i]; }
             qsort(cur, n_cur, sizeof(int32_t), cmp_i32);
 
             int32_t *out = X + ((size_t)t * c->n_q + g) * K;
@@ -192,7 +222,7 @@ int tg_generate(const tg_config *c, int32_t *X, int32_t *verified_len)
             n_prev = n_cur;
         }
     }
-    free(mark); free(prev); free(cur); free(hot);
+    free(mark); free(prev); free(cur); free(hot); free(hist); free(seen);
     return 0;
 }
 

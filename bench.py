@@ -281,7 +281,6 @@ def run_cuda(args):
         dist.barrier()
     step_ms = [a.elapsed_time(b) for a, b in ev]
     st1 = ctx.stats()
-    clocks = sampler.stop()
     rows_timed = st1["rows_copied"] - st0["rows_copied"]
     hits_timed, miss_timed = st1["hits"] - st0["hits"], st1["misses"] - st0["misses"]
     total_ms = sum(step_ms)
@@ -324,6 +323,7 @@ def run_cuda(args):
         calls[0].run(Xd[W + K - 1][0], vlen[W + K - 1][0], slots_d[0], None, mc_d[0], stream)
         rep.append(ctx.stats()["last_stage_one_us"])
     ctx.set_timing(False)
+    clocks = sampler.stop()       # sampled from the first timed step to the last replay
 
     # ---- aggregate over ranks: device time = max over ranks, work = sum over ranks ----
     from paper_2609_37538_b200.sharding import aggregate
@@ -551,6 +551,93 @@ def run_table3(args):
         ctx.close()
 
 
+# ------------------------------------------------------------------------------------------------------------
+# --sweeps: Stage One latency over K and S (the shapes of the paper's Fig. 3), lifetime ablation (App. A),
+# capacity study (App. E protocol) and MTP cold-start reuse (App. E), all on synthetic traces, 1 GPU
+# ------------------------------------------------------------------------------------------------------------
+def _run_tables(avsg, torch, tr, cfgs, S, L, rb=656, replay=0, warm=None):
+    """Steps the given per-table trace recipes through one context (one call per iteration).
+    Returns (per-iteration (hits, misses), median Stage One us of `replay` replays of the last step)."""
+    n, K, n_q, T = len(cfgs), cfgs[0].topk, cfgs[0].n_q, cfgs[0].n_iters
+    traces = [tr.generate(c) for c in cfgs]
+    ctxlen = max(c.context for c in cfgs)
+    kv = avsg.pinned_empty(ctxlen * rb)                     # the bytes do not matter here: all tables share one
+    ctx = avsg.Context(num_tables=n, buffer_slots=S, row_bytes=rb, max_topk=K, max_tokens=n_q, max_lifetime=L)
+    call = ctx.prepare(list(range(n)), [kv] * n, n_q, K)
+    stream = torch.cuda.current_stream()
+    per_iter, prev = [], ctx.stats()
+    slots = None
+    for t in range(T):
+        X = torch.from_numpy(np.stack([traces[i][0][t] for i in range(n)])).cuda()
+        slots = torch.empty_like(X)
+        vlen = [int(traces[i][1][t]) for i in range(n)]
+        if replay and t == T - 1:
+            ctx.save_state()
+        call.run(X, vlen, slots, None, None, stream)
+        st = ctx.stats()
+        per_iter.append((st["hits"] - prev["hits"], st["misses"] - prev["misses"]))
+        prev = st
+    med = None
+    if replay:
+        ctx.set_timing(True)
+        us = []
+        for _ in range(replay):
+            ctx.restore_state()
+            call.run(X, vlen, slots, None, None, stream)
+            us.append(ctx.stats()["last_stage_one_us"])
+        med = statistics.median(us)
+    ctx.close()
+    return per_iter, med
+
+
+def run_sweeps(args):
+    import torch
+    import __graft_entry__
+    import avsg_traces as tr
+    __graft_entry__.build()
+    import paper_2609_37538_b200 as avsg
+    torch.cuda.set_device(0)
+
+    def recipe(table, K, n_q, T, ctx=131072, seed=77, **kw):
+        base = dict(beta=(18, 2), p_recent=0.5, recent_window=4096)
+        base.update(kw)
+        return tr.TraceConfig(seed=seed, table=table, topk=K, n_q=n_q, n_iters=T, context=ctx, **base)
+
+    # (a) Stage One latency: S = K = N; K at S = 4096; S at K = 512.  Median of 300 replays of a steady step.
+    shapes = [("S=K=N", k, k) for k in (256, 512, 1024, 2048)]
+    shapes += [("K at S=4096", k, 4096) for k in (256, 512, 1024, 2048)]
+    shapes += [("S at K=512", 512, sz) for sz in (512, 1024, 2048, 4096, 8192)]
+    for label, K, S in shapes:
+        for B in (1, 32):
+            _, med = _run_tables(avsg, torch, tr, [recipe(i, K, 1, 24) for i in range(B)], S, 16, replay=300)
+            print(json.dumps({"sweep": "stage_one_latency", "series": label, "K": K, "S": S, "tables": B,
+                              "match_reserve_us_median": med}), flush=True)
+    # (b) lifetime ablation: K = 2048, 8K pool, MTP-0, 16 tables, 200 steps, steady steps only
+    for L in (1, 2, 4, 8, 16, 32):
+        per, med = _run_tables(avsg, torch, tr, [recipe(i, 2048, 1, 200) for i in range(16)], 8192, L, replay=100)
+        h = sum(a for a, _ in per[40:]); m = sum(b for _, b in per[40:])
+        print(json.dumps({"sweep": "lifetime", "L": L, "hit_rate": h / (h + m), "match_reserve_us_median": med}),
+              flush=True)
+    # (c) capacity study: max KV 16K, K = 2048, L = 8, MTP-0, adjacent-step similarity gamma fixed, historical
+    #     recall ~ N(mu, 0.01^2); 4K and 8K pools; 5 seeds (one table each); 300 steps, the first 60 not counted
+    for gamma in (0.5, 0.7, 0.9):
+        for mu in (0.5, 0.7, 0.9):
+            row = {"sweep": "capacity", "gamma": gamma, "mu_hist": mu}
+            for S in (4096, 8192):
+                cfgs = [tr.TraceConfig(seed=900 + sd, table=sd, topk=2048, n_q=1, n_iters=300, context=16384,
+                                       rho_fixed=gamma, p_hist=mu, hist_sigma=0.01) for sd in range(5)]
+                per, _ = _run_tables(avsg, torch, tr, cfgs, S, 8)
+                h = sum(a for a, _ in per[60:]); m = sum(b for _, b in per[60:])
+                row["hit_rate_%dK" % (S // 1024)] = h / (h + m)
+            print(json.dumps(row), flush=True)
+    # (d) MTP cold start: reuse inside the first iteration from an empty buffer, degrees 0..3, 32 tables
+    for deg in range(4):
+        per, _ = _run_tables(avsg, torch, tr, [recipe(i, 2048, deg + 1, 1) for i in range(32)], 8192, 16)
+        h, m = per[0]
+        print(json.dumps({"sweep": "mtp_cold_start", "n_mtp": deg, "reuse": h / (h + m),
+                          "rows_copied_per_request": m / 32}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -566,12 +653,16 @@ def main():
     ap.add_argument("--table3", action="store_true",
                     help="extra report: Stage Two strategies S1/S2/S3 on the paper's B x reuse grid (1 GPU)")
     ap.add_argument("--replays-table3", type=int, default=9)
+    ap.add_argument("--sweeps", action="store_true",
+                    help="extra report: Stage One K/S latency sweep, lifetime ablation, capacity study, MTP cold start")
     ap.add_argument("--suite", action="store_true",
                     help="extra report: C1..C5 hit rates, per-call times and the Stage Two comparators (1 GPU)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.table3:
+    if args.sweeps:
+        run_sweeps(args)
+    elif args.table3:
         run_table3(args)
     elif args.suite:
         run_suite(args)
