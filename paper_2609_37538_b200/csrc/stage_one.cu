@@ -360,27 +360,32 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
         if (n_g == 0) { __syncthreads(); continue; }
         __syncthreads();
 
-        // ---- Pass 3: how many unit decays until n_g slots are dead ----
+        // ---- Pass 3: CollectDead; if fewer than n_g slots are dead, decay until enough are ----
         uint32_t w0, w1;
         life_load(s_life, j0, spt, own, w0, w1);
-        count_lifetimes(w0, w1, spt, own, L, s_priv, priv_stride, s_hist);
-        __syncthreads();
-        uint32_t d = (uint32_t)L + 1u, cum = 0;
-        bool found = false;
-        for (uint32_t b = 0; b <= (uint32_t)L + 1u; ++b) {   // bin b counts lifetime b-1; dead after d = b decays
-            cum += s_hist[b];
-            if (cum >= n_g) { d = b; found = true; break; }
-        }
-        if (!found && tid == 0) atomicOr(p.status, ST_NO_DEAD_SLOTS);
-        if (d > 0) {
+        uint32_t sg0 = w0 & 0x80808080u, sg1 = w1 & 0x80808080u;       // sign bits = dead slots
+        uint32_t dtotal, d = 0;
+        uint32_t doff = block_excl_scan(__popc(sg0) + __popc(sg1), s_scan_b, dtotal);
+        if (dtotal < n_g) {
+            // the while-loop of Alg. 1 in closed form: d = fewest unit decays after which n_g slots are dead,
+            // read off the histogram of the lifetimes (only needed on this, the rarer, path)
+            count_lifetimes(w0, w1, spt, own, L, s_priv, priv_stride, s_hist);
+            __syncthreads();
+            uint32_t cum = 0;
+            bool found = false;
+            d = (uint32_t)L + 1u;
+            for (uint32_t b = 0; b <= (uint32_t)L + 1u; ++b) {   // bin b counts lifetime b-1; dead after b decays
+                cum += s_hist[b];
+                if (cum >= n_g) { d = b; found = true; break; }
+            }
+            if (!found && tid == 0) atomicOr(p.status, ST_NO_DEAD_SLOTS);
             w0 = decay4(w0, d);
             w1 = decay4(w1, d);
             life_store(s_life, j0, spt, own, w0, w1);
+            sg0 = w0 & 0x80808080u; sg1 = w1 & 0x80808080u;
+            doff = block_excl_scan(__popc(sg0) + __popc(sg1), s_scan_b, dtotal);
         }
-        // CollectDead: dead slots in increasing order; keep the first n_g
-        const uint32_t sg0 = w0 & 0x80808080u, sg1 = w1 & 0x80808080u;
-        uint32_t dtotal;
-        uint32_t doff = block_excl_scan(__popc(sg0) + __popc(sg1), s_scan_b, dtotal);
+        // dead slots in increasing order; the first n_g are handed out
 #pragma unroll
         for (uint32_t k = 0; k < (uint32_t)MAX_SPT; ++k) {
             const uint32_t bit = k < 4 ? (sg0 >> (8 * k + 7)) & 1u : (sg1 >> (8 * (k - 4) + 7)) & 1u;
