@@ -265,6 +265,12 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
 
     Index ix{s_key, s_val, s_tok, H - 1u, p.logH};
 
+    // Programmatic dependent launch: this grid may have been started while the previous kernel of the stream
+    // was still running; nothing is read before that kernel has completed.  The next kernel (Stage Two) is
+    // allowed to start its own prologue right away - it waits the same way before it reads the miss list.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     // ---- issue every global load first: table state and the first token's ids ----
     int4 t4[MAX_SPT / 4];
     int32_t t1[3];
@@ -537,9 +543,17 @@ cudaError_t stage_one_prepare(size_t max_smem)
 
 cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream)
 {
-    const uint32_t threads = stage_one_threads(p.S, p.K);
-    avsg_stage_one_kernel<<<n_tables, threads, stage_one_smem_bytes(p.S, p.K, p.L), stream>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_tables);
+    cfg.blockDim = dim3(stage_one_threads(p.S, p.K));
+    cfg.dynamicSmemBytes = stage_one_smem_bytes(p.S, p.K, p.L);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel, p);
 }
 
 cudaError_t launch_all_k_prepare(const AllKParams& p, uint32_t n_tables, cudaStream_t stream)

@@ -55,6 +55,11 @@ __global__ void __launch_bounds__(1024) avsg_transfer_kernel(const __grid_consta
     const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31u;
     const uint32_t n_seg = p.n_seg;
 
+    // Programmatic dependent launch: the blocks may already be resident while Stage One still runs; the miss
+    // list is read only after that grid has completed.  The kernel after this one may start its prologue.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     // global miss prefix sum (every block computes the same one)
     uint32_t running = 0;
     for (uint32_t base = 0; base < n_seg; base += nt) {
@@ -161,8 +166,17 @@ cudaError_t launch_transfer_positions(const PosParams& p, uint32_t blocks, uint3
 
 cudaError_t launch_transfer(const XferParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream)
 {
-    avsg_transfer_kernel<<<blocks, threads, 0, stream>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, avsg_transfer_kernel, p);
 }
 
 }  // namespace avsg
