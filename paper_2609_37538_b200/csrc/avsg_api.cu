@@ -41,6 +41,9 @@ struct avsg_ctx {
     uint32_t epoch = 0;
     std::vector<const void*> call_kv_host;     // host pointers of the current call (copy-engine mode)
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+    // avsg_step_host: the outputs go back on a side stream while Stage Two runs
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_outputs_ready = nullptr, ev_outputs_copied = nullptr;
     uint64_t last_rows = 0;
 };
 
@@ -71,6 +74,9 @@ void free_all(avsg_ctx* c)
     if (c->h_seg) cudaFreeHost(c->h_seg);
     if (c->h_list) cudaFreeHost(c->h_list);
     for (auto& e : c->ev) if (e) cudaEventDestroy(e);
+    if (c->ev_outputs_ready) cudaEventDestroy(c->ev_outputs_ready);
+    if (c->ev_outputs_copied) cudaEventDestroy(c->ev_outputs_copied);
+    if (c->side) cudaStreamDestroy(c->side);
 }
 
 int init_tables(avsg_ctx* c, uint32_t first, uint32_t n)
@@ -209,6 +215,18 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
     }
     if (c->timing) CU(cudaEventRecord(c->ev[1], stream));
 
+    if (host_io) {
+        // The slot table, hit mask and miss counts are final once Stage One has run.  They travel device -> host
+        // on a side stream while Stage Two pulls rows host -> device: the two directions of the link overlap.
+        CU(cudaEventRecord(c->ev_outputs_ready, stream));
+        CU(cudaStreamWaitEvent(c->side, c->ev_outputs_ready, 0));
+        CU(cudaMemcpyAsync(a->slots, c->d_slots_stage, n_ids * sizeof(int32_t), cudaMemcpyDeviceToHost, c->side));
+        if (a->hit) CU(cudaMemcpyAsync(a->hit, c->d_hit_stage, n_ids, cudaMemcpyDeviceToHost, c->side));
+        if (a->miss_count)
+            CU(cudaMemcpyAsync(a->miss_count, c->d_mc_stage, (size_t)n * n_q * sizeof(int32_t), cudaMemcpyDeviceToHost, c->side));
+        CU(cudaEventRecord(c->ev_outputs_copied, c->side));
+    }
+
     if (mode == AVSG_XFER_COPY_ENGINE) {
         if ((rc = copy_engine_transfer(c, a, stream)) != AVSG_OK) return rc;
     } else if (mode == AVSG_XFER_POSITION_LEVEL) {
@@ -226,12 +244,7 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
     }
     if (c->timing) { CU(cudaEventRecord(c->ev[2], stream)); c->events_recorded = true; }
 
-    if (host_io) {
-        CU(cudaMemcpyAsync(a->slots, c->d_slots_stage, n_ids * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
-        if (a->hit) CU(cudaMemcpyAsync(a->hit, c->d_hit_stage, n_ids, cudaMemcpyDeviceToHost, stream));
-        if (a->miss_count)
-            CU(cudaMemcpyAsync(a->miss_count, c->d_mc_stage, (size_t)n * n_q * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
-    }
+    if (host_io) CU(cudaStreamWaitEvent(stream, c->ev_outputs_copied, 0));     // the call ends when the outputs are home
     return AVSG_OK;
 }
 
@@ -298,6 +311,9 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaHostAlloc(&c->h_seg, T * sizeof(SegDesc), cudaHostAllocDefault) == cudaSuccess;
     ok = ok && cudaHostAlloc(&c->h_list, n_ids * sizeof(int2), cudaHostAllocDefault) == cudaSuccess;
     for (auto& e : c->ev) ok = ok && cudaEventCreate(&e) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_ready, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_copied, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { cudaGetLastError(); free_all(c); delete c; return AVSG_ENOMEM; }
     if (cudaMemset(c->d_status, 0, 256) != cudaSuccess || cudaMemset(c->d_seg, 0, T * sizeof(SegDesc)) != cudaSuccess ||
         init_tables(c, 0, (uint32_t)T) != AVSG_OK || cudaDeviceSynchronize() != cudaSuccess) {
