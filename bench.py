@@ -225,8 +225,11 @@ def run_cuda(args):
         tr.fill_kv(buf.data_ptr(), w.seed, ti, cfg.context, w.row_bytes, row_stride=stride)
         kv.append(buf)
 
+    direct = args.index == "direct"
     ctx = avsg.Context(num_tables=w.num_tables, buffer_slots=w.buffer_slots, row_bytes=w.row_bytes,
-                       max_topk=w.topk, max_tokens=w.n_q, max_lifetime=w.max_lifetime, device=local)
+                       max_topk=w.topk, max_tokens=w.n_q, max_lifetime=w.max_lifetime, device=local,
+                       index_mode=avsg.INDEX_DIRECT if direct else avsg.INDEX_HASH,
+                       max_context=max(c.context for c in w.tables) + w.n_q)
     ncalls = len(w.calls)
     calls = [ctx.prepare(grp, [kv[t] for t in grp], w.n_q, w.topk,
                          [stride] * len(grp) if args.row_stride else None) for grp in w.calls]
@@ -354,7 +357,7 @@ def run_cuda(args):
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms_j / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int32/u8", "data": "synthetic", "config": dict(_config(w), host_row_stride=stride),
+        "dtype": "int32/u8", "data": "synthetic", "config": dict(_config(w), host_row_stride=stride, stage_one_index=args.index),
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "GB/s",
                 "h2d_bytes_per_step": int(ids_bytes + rows_timed * rb / K), "d2h_bytes_per_step": int(ids_bytes + mc_bytes),
@@ -648,6 +651,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--requests", type=int, default=32, help="requests per layer (32 = the full configuration)")
     ap.add_argument("--layers", type=int, default=4, help="layers (4 = the full configuration)")
+    ap.add_argument("--index", default="direct", choices=["hash", "direct"],
+                    help="Stage One index: direct-address table in device memory (default) or shared-memory hash table")
     ap.add_argument("--row-stride", type=int, default=0,
                     help="bytes between host KV rows (0 = packed, 656); e.g. 768 pads rows to 128-byte lines")
     ap.add_argument("--table3", action="store_true",

@@ -56,6 +56,12 @@ extern "C" {
                                        block, which walks its range and copies the misses;
                                        hit positions are visited for nothing             */
 
+/* How Stage One finds the slot that holds an id (same results either way). */
+#define AVSG_INDEX_HASH   0u  /* open-addressing table in shared memory, rebuilt every step     */
+#define AVSG_INDEX_DIRECT 1u  /* one 16-bit entry per context position in device memory
+                                 (2 bytes x max_context per table, L2-resident); needs every
+                                 id < max_context                                              */
+
 typedef struct avsg_ctx avsg_ctx;   /* opaque */
 
 typedef struct {
@@ -67,6 +73,9 @@ typedef struct {
     int32_t  max_lifetime;   /* L in 1 .. 126 (paper default 16)                        */
     uint32_t transfer_mode;  /* AVSG_XFER_*                                             */
     int32_t  device;         /* CUDA device ordinal                                     */
+    uint32_t index_mode;     /* AVSG_INDEX_*                                            */
+    uint32_t max_context;    /* AVSG_INDEX_DIRECT: ids are < max_context (count the
+                                speculative positions too); ignored for AVSG_INDEX_HASH  */
 } avsg_config;
 
 typedef struct {

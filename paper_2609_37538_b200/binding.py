@@ -17,6 +17,7 @@ from . import build as _build
 
 OK, EINVAL, ENOMEM, ECUDA, ECAPACITY, EDEVICE_STATUS, EUNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
 XFER_SM_BALANCED, XFER_COPY_ENGINE, XFER_REQUEST_LEVEL, XFER_ALL_K, XFER_POSITION_LEVEL = 0, 1, 2, 3, 4
+INDEX_HASH, INDEX_DIRECT = 0, 1
 
 EXPORTS = (
     "avsg_create", "avsg_destroy", "avsg_reset", "avsg_step", "avsg_step_host", "avsg_buffer", "avsg_stats",
@@ -29,7 +30,8 @@ EXPORTS = (
 class AvsgConfig(ctypes.Structure):
     _fields_ = [("num_tables", ctypes.c_uint32), ("buffer_slots", ctypes.c_uint32), ("row_bytes", ctypes.c_uint32),
                 ("max_topk", ctypes.c_uint32), ("max_tokens", ctypes.c_uint32), ("max_lifetime", ctypes.c_int32),
-                ("transfer_mode", ctypes.c_uint32), ("device", ctypes.c_int32)]
+                ("transfer_mode", ctypes.c_uint32), ("device", ctypes.c_int32), ("index_mode", ctypes.c_uint32),
+                ("max_context", ctypes.c_uint32)]
 
 
 class AvsgStepArgs(ctypes.Structure):
@@ -183,11 +185,12 @@ class Context:
     """Owns the device state of num_tables tables (see avsg_create)."""
 
     def __init__(self, num_tables: int, buffer_slots: int, row_bytes: int, max_topk: int, max_tokens: int = 1,
-                 max_lifetime: int = 16, transfer_mode: int = XFER_SM_BALANCED, device: int = 0):
+                 max_lifetime: int = 16, transfer_mode: int = XFER_SM_BALANCED, device: int = 0,
+                 index_mode: int = INDEX_HASH, max_context: int = 0):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         cfg = AvsgConfig(num_tables, buffer_slots, row_bytes, max_topk, max_tokens, max_lifetime, transfer_mode,
-                         device)
+                         device, index_mode, max_context)
         _check(self._lib.avsg_create(ctypes.byref(cfg), ctypes.byref(self._h)), "avsg_create")
         self.num_tables, self.S, self.row_bytes = num_tables, buffer_slots, row_bytes
         self.max_topk, self.max_tokens, self.L, self.device = max_topk, max_tokens, max_lifetime, device
@@ -275,8 +278,11 @@ class Context:
         _check(self._lib.avsg_set_transfer_geometry(self._h, blocks, threads), "avsg_set_transfer_geometry")
 
     def sync_status(self) -> int:
+        """Waits for the device and returns the kernels' status word (0 = no problem was flagged)."""
         w = ctypes.c_uint32(0)
-        _check(self._lib.avsg_sync_status(self._h, ctypes.byref(w)), "avsg_sync_status")
+        rc = self._lib.avsg_sync_status(self._h, ctypes.byref(w))
+        if rc != EDEVICE_STATUS:
+            _check(rc, "avsg_sync_status")
         return w.value
 
     def stats(self) -> dict:

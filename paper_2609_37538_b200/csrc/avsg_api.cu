@@ -25,6 +25,7 @@ struct avsg_ctx {
     int2* d_list = nullptr;
     SegDesc* d_seg = nullptr;
     uint32_t* d_status = nullptr;
+    uint16_t* d_where = nullptr;       // direct index, or null
     int32_t* d_tok_snap = nullptr;
     int8_t* d_life_snap = nullptr;
     // staging of avsg_step_host
@@ -68,7 +69,7 @@ uint32_t ilog2(uint32_t v) { uint32_t l = 0; while ((1u << l) < v) ++l; return l
 void free_all(avsg_ctx* c)
 {
     cudaFree(c->d_tok); cudaFree(c->d_life); cudaFree(c->d_buffer); cudaFree(c->d_stats);
-    cudaFree(c->d_list); cudaFree(c->d_seg); cudaFree(c->d_status);
+    cudaFree(c->d_list); cudaFree(c->d_seg); cudaFree(c->d_status); cudaFree(c->d_where);
     cudaFree(c->d_tok_snap); cudaFree(c->d_life_snap);
     cudaFree(c->d_idx_stage); cudaFree(c->d_slots_stage); cudaFree(c->d_hit_stage); cudaFree(c->d_mc_stage);
     if (c->h_seg) cudaFreeHost(c->h_seg);
@@ -204,6 +205,7 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
             p.S = c->cfg.buffer_slots; p.logH = c->logH; p.row_bytes = c->cfg.row_bytes;
             p.K = K; p.n_q = n_q; p.L = (uint32_t)c->cfg.max_lifetime;
             p.first = first; p.list_stride = c->list_stride;
+            p.where = c->d_where; p.max_context = c->cfg.max_context;
             for (uint32_t i = 0; i < cnt; ++i) {
                 p.table_id[i] = a->table_ids[first + i];
                 p.verified_len[i] = a->verified_len[first + i];
@@ -268,7 +270,8 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     if (cfg->row_bytes == 0 || cfg->row_bytes % 16) return AVSG_EINVAL;
     if (cfg->max_topk == 0 || cfg->max_tokens == 0) return AVSG_EINVAL;
     if (cfg->max_lifetime < 1 || cfg->max_lifetime > 126) return AVSG_EINVAL;
-    if (cfg->transfer_mode > AVSG_XFER_POSITION_LEVEL) return AVSG_EINVAL;
+    if (cfg->transfer_mode > AVSG_XFER_POSITION_LEVEL || cfg->index_mode > AVSG_INDEX_DIRECT) return AVSG_EINVAL;
+    if (cfg->index_mode == AVSG_INDEX_DIRECT && cfg->max_context == 0) return AVSG_EINVAL;
     if ((uint64_t)cfg->max_topk * cfg->max_tokens > cfg->buffer_slots) return AVSG_ECAPACITY;   // Eq. 7
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || cfg->device < 0 || cfg->device >= ndev) return AVSG_ECUDA;
@@ -287,7 +290,8 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     int max_smem = 0;
     cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, cfg->device);
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device);
-    const size_t need = stage_one_smem_bytes(cfg->buffer_slots, cfg->max_topk, (uint32_t)cfg->max_lifetime);
+    const size_t need = stage_one_smem_bytes(cfg->buffer_slots, cfg->max_topk, (uint32_t)cfg->max_lifetime,
+                                             cfg->index_mode == AVSG_INDEX_DIRECT);
     if (need > (size_t)max_smem) { delete c; return AVSG_EUNSUPPORTED; }
     // always raise the kernel's dynamic shared-memory limit to the device maximum: the attribute is
     // per function, so a context with a small table must not lower it under a context with a large one
@@ -302,6 +306,8 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaMalloc(&c->d_list, n_ids * sizeof(int2)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_seg, T * sizeof(SegDesc)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_status, 256) == cudaSuccess;
+    if (cfg->index_mode == AVSG_INDEX_DIRECT)
+        ok = ok && cudaMalloc(&c->d_where, T * (size_t)cfg->max_context * sizeof(uint16_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_tok_snap, T * S * sizeof(int32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_life_snap, T * S) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_idx_stage, n_ids * sizeof(int32_t)) == cudaSuccess;
@@ -315,7 +321,8 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_ready, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_copied, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { cudaGetLastError(); free_all(c); delete c; return AVSG_ENOMEM; }
-    if (cudaMemset(c->d_status, 0, 256) != cudaSuccess || cudaMemset(c->d_seg, 0, T * sizeof(SegDesc)) != cudaSuccess ||
+    if ((c->d_where && cudaMemset(c->d_where, 0xFF, T * (size_t)cfg->max_context * sizeof(uint16_t)) != cudaSuccess) ||
+        cudaMemset(c->d_status, 0, 256) != cudaSuccess || cudaMemset(c->d_seg, 0, T * sizeof(SegDesc)) != cudaSuccess ||
         init_tables(c, 0, (uint32_t)T) != AVSG_OK || cudaDeviceSynchronize() != cudaSuccess) {
         free_all(c); delete c; return AVSG_ECUDA;
     }
@@ -423,6 +430,10 @@ int avsg_import_state(avsg_ctx* c, uint32_t table_id, const int32_t* tok, const 
     CU(cudaDeviceSynchronize());
     CU(cudaMemcpy(c->d_tok + table_id * S, tok, S * sizeof(int32_t), cudaMemcpyHostToDevice));
     CU(cudaMemcpy(c->d_life + table_id * S, life, S, cudaMemcpyHostToDevice));
+    if (c->d_where) {
+        CU(launch_direct_index_from_state(c->d_tok, c->d_where, table_id, 1, c->cfg.buffer_slots, c->cfg.max_context, nullptr));
+        CU(cudaDeviceSynchronize());
+    }
     return AVSG_OK;
 }
 
@@ -447,6 +458,9 @@ int avsg_restore_state(avsg_ctx* c, void* stream)
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     CU(cudaMemcpyAsync(c->d_tok, c->d_tok_snap, n * sizeof(int32_t), cudaMemcpyDeviceToDevice, s));
     CU(cudaMemcpyAsync(c->d_life, c->d_life_snap, n, cudaMemcpyDeviceToDevice, s));
+    if (c->d_where)
+        CU(launch_direct_index_from_state(c->d_tok, c->d_where, 0, c->cfg.num_tables, c->cfg.buffer_slots,
+                                          c->cfg.max_context, s));
     return AVSG_OK;
 }
 

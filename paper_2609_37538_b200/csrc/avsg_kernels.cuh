@@ -12,6 +12,7 @@ enum : uint32_t {
     ST_NO_DEAD_SLOTS   = 1u << 1,   // fewer reclaimable slots than misses (Eq. 7 violated)
     ST_BAD_SLOT        = 1u << 2,   // slot / position index out of range
     ST_BAD_SEGMENT     = 1u << 3,   // transfer kernel could not resolve a miss
+    ST_BAD_ID          = 1u << 4,   // direct index: an id beyond max_context (treated as padding)
 };
 
 // One segment of the step's miss list = the misses of one table, in token
@@ -48,6 +49,8 @@ struct S1Params {
     uint32_t S, logH, row_bytes, K, n_q, L;
     uint32_t first;              // index within the call of this launch's first table
     uint32_t list_stride;        // entries per segment of miss_list
+    uint32_t max_context;        // direct index: entries per table
+    uint16_t* where;             // direct index [num_tables][max_context], or null for the hash index
     uint32_t table_id[S1_MAX_TABLES];
     int32_t  verified_len[S1_MAX_TABLES];
     uint64_t kv_base[S1_MAX_TABLES];
@@ -85,10 +88,12 @@ struct AllKParams {
     uint64_t kv_stride[S1_MAX_TABLES];
 };
 
-size_t stage_one_smem_bytes(uint32_t S, uint32_t K, uint32_t L);
+size_t stage_one_smem_bytes(uint32_t S, uint32_t K, uint32_t L, bool direct = false);
 uint32_t stage_one_threads(uint32_t S, uint32_t K);
 cudaError_t stage_one_prepare(size_t max_smem);
 cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream);
+cudaError_t launch_direct_index_from_state(const int32_t* tok, uint16_t* where, uint32_t first_table, uint32_t n_tables,
+                                           uint32_t S, uint32_t max_context, cudaStream_t stream);
 cudaError_t launch_all_k_prepare(const AllKParams& p, uint32_t n_tables, cudaStream_t stream);
 cudaError_t launch_transfer(const XferParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream);
 cudaError_t launch_transfer_positions(const PosParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream);

@@ -4,6 +4,13 @@
 // operations of Algorithm 3, for the N_q tokens of one iteration in order
 // (Algorithm 4), and the end-of-step invalidation of Algorithm 4.
 //
+// Two interchangeable id -> slot indexes (template parameter DIRECT):
+//   hash   (default) an open-addressing table in shared memory, rebuilt every step (described below);
+//   direct           one 16-bit slot number per context position in global memory (it stays L2-resident:
+//                    2 bytes x context per table).  An entry is only ever written when an id is installed
+//                    and is never cleared: a lookup masks it to a valid slot number and then compares the
+//                    slot's cached id, so stale or uninitialised entries simply miss.  No build, no probing.
+//
 // The whole table lives in shared memory for the step:
 //   s_tok[S]   cached id per slot            s_life[S]  lifetime per slot
 //   s_key[H], s_val[H]  open-addressing index id -> slot, H = 2S buckets,
@@ -231,10 +238,11 @@ __device__ __forceinline__ void count_lifetimes(uint32_t w0, uint32_t w1, uint32
     }
 }
 
+template <bool DIRECT>
 __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_constant__ S1Params p)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    const uint32_t S = p.S, K = p.K, H = 1u << p.logH, Kp = (K + 7u) & ~7u;
+    const uint32_t S = p.S, K = p.K, H = DIRECT ? 0u : 1u << p.logH, Kp = (K + 7u) & ~7u;
     const uint32_t tid = threadIdx.x, nt = blockDim.x;
     const int32_t L = (int32_t)p.L;
 
@@ -264,6 +272,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
     const uint32_t i0 = tid * ipt;
 
     Index ix{s_key, s_val, s_tok, H - 1u, p.logH};
+    uint16_t* where = DIRECT ? p.where + (size_t)table * p.max_context : nullptr;
 
     // Programmatic dependent launch: this grid may have been started while the previous kernel of the stream
     // was still running; nothing is read before that kernel has completed.  The next kernel (Stage Two) is
@@ -290,7 +299,9 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
     int32_t xs[MAX_IPT];
     load_ids(p.indices + (size_t)ti * p.n_q * K, i0, ipt, K, xs);
 
-    for (uint32_t i = tid; i < H / 4; i += nt) reinterpret_cast<int4*>(s_key)[i] = make_int4(EMPTY, EMPTY, EMPTY, EMPTY);
+    if (!DIRECT)
+        for (uint32_t i = tid; i < H / 4; i += nt)
+            reinterpret_cast<int4*>(s_key)[i] = make_int4(EMPTY, EMPTY, EMPTY, EMPTY);
     if (s_priv)
         for (uint32_t i = tid; i < ((uint32_t)(L + 2) * priv_stride + 15u) / 16u; i += nt)
             reinterpret_cast<int4*>(s_priv)[i] = make_int4(0, 0, 0, 0);
@@ -309,9 +320,12 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
     // global pre-decay of the iteration's first token (Alg. 1 Pass 1)
     life_store(s_life, j0, spt, own, decay4(lw0, 1), decay4(lw1, 1));
     __syncthreads();
-    build_index(ix, s_tok, j0, spt, own, s_fill, p.status);
-    __syncthreads();
-    uint32_t fill_bound = *s_fill;                        // non-empty buckets (upper bound)
+    uint32_t fill_bound = 0;                              // hash index: non-empty buckets (upper bound)
+    if (!DIRECT) {
+        build_index(ix, s_tok, j0, spt, own, s_fill, p.status);
+        __syncthreads();
+        fill_bound = *s_fill;
+    }
 
     uint32_t list_off = 0, sum_valid = 0, sum_miss = 0, sum_decay = 0;
     int2* list = p.miss_list + (size_t)ti * p.list_stride;
@@ -324,14 +338,27 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
 
         // ---- Probe, refresh hits to L, emit hit slots (Pass 1 + Pass 2) ----
         uint32_t missmask = 0, nmiss = 0, nvalid = 0;
+        uint32_t cand[MAX_IPT];                             // direct index: candidate slot per id
+        if (DIRECT) {
+#pragma unroll
+            for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {   // all loads are issued before any is used
+                cand[k] = 0xFFFFFFFFu;
+                if (k < ipt && i0 + k < K && xs[k] >= 0) {
+                    if ((uint32_t)xs[k] < p.max_context) cand[k] = __ldcg(where + xs[k]) & (S - 1u);
+                    else atomicOr(p.status, ST_BAD_ID);
+                }
+            }
+        }
 #pragma unroll
         for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {
             const uint32_t i = i0 + k;
             if (k < ipt && i < K) {
                 const int32_t x = xs[k];
-                if (x >= 0) {
+                if (x >= 0 && (!DIRECT || cand[k] != 0xFFFFFFFFu)) {
                     ++nvalid;
-                    const int32_t j = index_find(ix, x, p.status);
+                    int32_t j;
+                    if (DIRECT) j = s_tok[cand[k]] == x ? (int32_t)cand[k] : -1;
+                    else j = index_find(ix, x, p.status);
                     if (j >= 0) {
                         s_life[j] = (int8_t)L;
                         O[i] = j;
@@ -403,7 +430,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
         __syncthreads();
 
         // ---- install the misses: k-th miss takes the k-th dead slot ----
-        const bool rebuild = fill_bound + n_g > (H / 4u) * 3u;
+        const bool rebuild = !DIRECT && fill_bound + n_g > (H / 4u) * 3u;
         const uint32_t n_take = n_g < dtotal ? n_g : dtotal;
         for (uint32_t k = tid; k < n_take; k += nt) {
             const uint32_t j = s_dead[k];
@@ -415,7 +442,8 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
                 O[i] = (int32_t)j;
                 if (Hm) Hm[i] = 0;
                 list[list_off + k] = make_int2(x, (int32_t)j);
-                if (!rebuild) index_insert(ix, x, j, p.status);
+                if (DIRECT) __stcg(where + x, (uint16_t)j);
+                else if (!rebuild) index_insert(ix, x, j, p.status);
             } else {
                 list[list_off + k] = make_int2(-1, -1);          // Stage Two skips it
                 atomicOr(p.status, ST_BAD_SLOT);
@@ -476,6 +504,20 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
     }
 }
 
+// Direct index: points every resident id at its slot again, after the table state was replaced from outside
+// (import, restore of a snapshot).  One thread per slot; ids are unique within a table.
+__global__ void avsg_direct_index_from_state_kernel(const int32_t* __restrict__ tok, uint16_t* where,
+                                                    uint32_t first_table, uint32_t n_tables, uint32_t S,
+                                                    uint32_t max_context)
+{
+    const size_t n = (size_t)n_tables * S;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const uint32_t t = first_table + (uint32_t)(i / S), j = (uint32_t)(i % S);
+        const int32_t x = tok[(size_t)t * S + j];
+        if (x >= 0 && (uint32_t)x < max_context) where[(size_t)t * max_context + x] = (uint16_t)j;
+    }
+}
+
 // "KV offload" comparator: every selected row moves, position (g, i) -> slot g*K + i.
 __global__ void __launch_bounds__(256) avsg_all_k_prepare_kernel(const __grid_constant__ AllKParams p)
 {
@@ -519,11 +561,12 @@ __global__ void __launch_bounds__(256) avsg_all_k_prepare_kernel(const __grid_co
 
 }  // namespace
 
-size_t stage_one_smem_bytes(uint32_t S, uint32_t K, uint32_t L)
+size_t stage_one_smem_bytes(uint32_t S, uint32_t K, uint32_t L, bool direct)
 {
-    const size_t H = 2ull * S, Kp = (K + 7u) & ~7u;
+    const size_t H = direct ? 0 : 2ull * S, Kp = (K + 7u) & ~7u;
     size_t n = S * 4 + H * 4 + Kp * 4 + H * 2 + Kp * 2 + Kp * 2 + S + (128 + 40 + 40 + 8) * 4;
     if ((int32_t)L <= PRIV_HIST_MAX_L) n += ((size_t)(L + 2) * (stage_one_threads(S, K) + 4) + 15) / 16 * 16;
+    (void)direct;
     return n;
 }
 
@@ -538,7 +581,9 @@ uint32_t stage_one_threads(uint32_t S, uint32_t K)
 
 cudaError_t stage_one_prepare(size_t max_smem)
 {
-    return cudaFuncSetAttribute(avsg_stage_one_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    cudaError_t e = cudaFuncSetAttribute(avsg_stage_one_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(avsg_stage_one_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
 }
 
 cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream)
@@ -546,14 +591,25 @@ cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_tables);
     cfg.blockDim = dim3(stage_one_threads(p.S, p.K));
-    cfg.dynamicSmemBytes = stage_one_smem_bytes(p.S, p.K, p.L);
+    const bool direct = p.where != nullptr;
+    cfg.dynamicSmemBytes = stage_one_smem_bytes(p.S, p.K, p.L, direct);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel, p);
+    return direct ? cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel<true>, p)
+                  : cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel<false>, p);
+}
+
+cudaError_t launch_direct_index_from_state(const int32_t* tok, uint16_t* where, uint32_t first_table, uint32_t n_tables,
+                                           uint32_t S, uint32_t max_context, cudaStream_t stream)
+{
+    const size_t n = (size_t)n_tables * S;
+    const uint32_t blocks = (uint32_t)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184);
+    avsg_direct_index_from_state_kernel<<<blocks, 256, 0, stream>>>(tok, where, first_table, n_tables, S, max_context);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_all_k_prepare(const AllKParams& p, uint32_t n_tables, cudaStream_t stream)

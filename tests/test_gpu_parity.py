@@ -245,3 +245,56 @@ def test_small_context_created_after_a_large_one_does_not_break_it(avsg):
     out = big.step([0], Xb, [kv], [20000])                   # must still launch with its large shared memory
     torch.cuda.synchronize()
     assert out.miss_count.cpu().numpy().sum() == 4096 and big.sync_status() == 0
+
+
+# ---- the direct-address index gives the same results as the shared-memory hash index ---------------------------
+@pytest.mark.parametrize("name,kw,every", [
+    ("C1", {}, 1), ("C2", {}, 16), ("C3", {}, 32), ("C4", {}, 32), ("C5", {}, 16),
+])
+def test_direct_index_full(avsg, name, kw, every):
+    _parity(tr.workload(name, **kw), index_mode=avsg.INDEX_DIRECT, buffer_every=every)
+
+
+@pytest.mark.parametrize("name,kw", SHAPES)
+def test_direct_index_shapes(avsg, name, kw):
+    _parity(tr.workload(name, **kw), index_mode=avsg.INDEX_DIRECT)
+
+
+def test_direct_index_import_restore_and_bad_ids(avsg):
+    import torch
+    rb, S, K, ctxlen = 32, 128, 16, 2000
+    host = np.empty(ctxlen * rb, np.uint8)
+    tr.fill_kv(host, 2, 0, ctxlen, rb)
+    dkv = torch.from_numpy(host).cuda()
+    ctx = avsg.Context(2, S, rb, K, 1, 4, index_mode=avsg.INDEX_DIRECT, max_context=ctxlen)
+    orc = OracleTable(S, rb, 4)
+    rng = np.random.default_rng(1)
+    sels = [np.sort(rng.choice(ctxlen, K, replace=False)).astype(np.int32) for _ in range(40)]
+    for t in range(20):
+        ctx.step([0], torch.from_numpy(sels[t][None, None]).cuda(), [dkv], [ctxlen])
+        orc.step(sels[t][None], ctxlen, host)
+    tok, life = ctx.export_state(0)
+    ctx.import_state(1, tok, life)                         # resume into a table whose index has never seen these ids
+    ctx.save_state()
+    for t in range(20, 30):
+        a = ctx.step([1], torch.from_numpy(sels[t][None, None]).cuda(), [dkv], [ctxlen])
+        r = orc.step(sels[t][None], ctxlen, host)
+        assert (a.slots.cpu().numpy()[0] == r.O).all() and (a.hit.cpu().numpy()[0] == r.M).all()
+    first = ctx.export_state(1)
+    ctx.restore_state()                                    # back to the snapshot: the same ten steps replay identically
+    orc2 = OracleTable(S, rb, 4)
+    orc2.import_state(tok, life)
+    for t in range(20, 30):
+        a = ctx.step([1], torch.from_numpy(sels[t][None, None]).cuda(), [dkv], [ctxlen])
+        r = orc2.step(sels[t][None], ctxlen, host)
+        assert (a.slots.cpu().numpy()[0] == r.O).all() and (a.hit.cpu().numpy()[0] == r.M).all()
+    again = ctx.export_state(1)
+    assert (first[0] == again[0]).all() and (first[1] == again[1]).all()
+    assert ctx.sync_status() == 0
+    bad = np.sort(rng.choice(ctxlen, K, replace=False)).astype(np.int32)
+    bad[-1] = ctxlen + 5                                   # an id the direct index cannot hold
+    out = ctx.step([0], torch.from_numpy(bad[None, None]).cuda(), [dkv], [ctxlen + 10])
+    assert out.slots.cpu().numpy()[0, 0, -1] == -1
+    assert ctx.sync_status() != 0                          # reported, not faulted
+    with pytest.raises(avsg.AvsgError):
+        avsg.Context(1, S, rb, K, 1, 4, index_mode=avsg.INDEX_DIRECT, max_context=0)
