@@ -35,7 +35,8 @@ METRIC = "miss-only H2D gather GB/s (% of link peak); match+reserve us per decod
 # DRAM traffic per unit from the ncu capture summarised under profiles/ (dram__bytes_read + dram__bytes_write
 # per launch of the one-layer case, divided by the units of that launch); scaled by the units of a launch here.
 NCU_XFER_DRAM_BYTES_PER_ROW = 91.0          # 0.94 MB per launch of 10.3 k rows: the written rows stay in L2
-NCU_S1_DRAM_BYTES_PER_TABLE = 59300.0       # 1.90 MB per launch of 32 tables
+NCU_S1_DRAM_BYTES_PER_TABLE = {"hash": 59400.0,     # 1.90 MB per launch of 32 tables
+                               "direct": 174000.0}  # 5.57 MB: the 2-byte index entries arrive as 32-byte sectors
 PAPER_CONTEXT = {
     "hardware": "Ascend 910B NPU (paper), not comparable",
     "hash_vs_dual_pointer_speedup": 2.80, "stage_one_us_K2048_S2048": 53.7,
@@ -351,6 +352,8 @@ def run_cuda(args):
     # Stage One algorithmic bytes per call: state read + write, ids in, slots out, miss counts, miss list
     n_tab = len(w.calls[0])
     s1_bytes = n_tab * (2 * w.buffer_slots * 5 + 2 * w.n_q * w.topk * 4 + w.n_q * 4 + 32) + 8 * sum(x_rows) / n_launch
+    if direct:      # direct index: one 2-byte entry read per id, one written per miss
+        s1_bytes += n_tab * w.n_q * w.topk * 2 + 2 * sum(x_rows) / n_launch
     s1_avg_us = sum(s1_us) / len(s1_us)
     s1_gbs = s1_bytes / 1e3 / s1_avg_us
 
@@ -382,8 +385,8 @@ def run_cuda(args):
                      "peak_kind": "measured in this run (pinned cudaMemcpyAsync H2D)",
                      "note": "algorithmic bytes = row_bytes x missed rows per launch; the rows cross the host link and stay "
                              "in L2 after the write, so DRAM traffic (scaled from the ncu capture of the one-layer case) is small"},
-        "roofline_stage_one": {"bound": "hbm", "kernel": "avsg_stage_one_kernel", "achieved": s1_gbs, "peak": hbm_peak,
-                               "unit": "GB/s", "frac": s1_gbs / hbm_peak, "traffic": NCU_S1_DRAM_BYTES_PER_TABLE * n_tab,
+        "roofline_stage_one": {"bound": "hbm", "kernel": "avsg_stage_one_kernel<%s>" % args.index, "achieved": s1_gbs, "peak": hbm_peak,
+                               "unit": "GB/s", "frac": s1_gbs / hbm_peak, "traffic": NCU_S1_DRAM_BYTES_PER_TABLE[args.index] * n_tab,
                                "peak_kind": peak_kind,
                                "bytes_per_launch": s1_bytes},
         "paper_context": PAPER_CONTEXT,
