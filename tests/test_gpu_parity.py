@@ -298,3 +298,32 @@ def test_direct_index_import_restore_and_bad_ids(avsg):
     assert ctx.sync_status() != 0                          # reported, not faulted
     with pytest.raises(avsg.AvsgError):
         avsg.Context(1, S, rb, K, 1, 4, index_mode=avsg.INDEX_DIRECT, max_context=0)
+
+
+# ---- degenerate selections --------------------------------------------------------------------------------------
+@pytest.mark.parametrize("index_mode", [0, 1])
+def test_degenerate_selections(avsg, index_mode):
+    import torch
+    rb, S, ctxlen = 32, 32, 500
+    host = np.empty(ctxlen * rb, np.uint8)
+    tr.fill_kv(host, 4, 0, ctxlen, rb)
+    kv = avsg.pinned_empty(ctxlen * rb)
+    kv.numpy()[:] = host
+    rng = np.random.default_rng(index_mode)
+    for K, n_q in [(1, 1), (1, 8), (4, 8), (32, 1), (7, 3)]:
+        ctx = avsg.Context(1, S, rb, K, n_q, 2, index_mode=index_mode, max_context=ctxlen)
+        orc = OracleTable(S, rb, 2)
+        for t in range(30):
+            X = np.stack([np.sort(rng.choice(ctxlen, K, replace=False)) for _ in range(n_q)]).astype(np.int32)
+            if t % 5 == 4:
+                X[n_q - 1, :] = -1                                   # a token made of padding only
+            if t % 7 == 6 and K > 1:
+                X[0, K // 2:] = -1                                   # a half-padded token
+            out = ctx.step([0], torch.from_numpy(X[None]).cuda(), [kv], [ctxlen])
+            r = orc.step(X, ctxlen, host)
+            assert (out.slots.cpu().numpy()[0] == r.O).all(), (K, n_q, t)
+            assert (out.hit.cpu().numpy()[0] == r.M).all() and (out.miss_count.cpu().numpy()[0] == r.n).all()
+            tok, life = ctx.export_state(0)
+            c, l = orc.export_state()
+            assert (tok == c).all() and (life == l).all()
+        assert (ctx.buffer(0).cpu().numpy() == orc.rows()).all() and ctx.sync_status() == 0
