@@ -561,14 +561,15 @@ def run_table3(args):
 # --sweeps: Stage One latency over K and S (the shapes of the paper's Fig. 3), lifetime ablation (App. A),
 # capacity study (App. E protocol) and MTP cold-start reuse (App. E), all on synthetic traces, 1 GPU
 # ------------------------------------------------------------------------------------------------------------
-def _run_tables(avsg, torch, tr, cfgs, S, L, rb=656, replay=0, warm=None):
+def _run_tables(avsg, torch, tr, cfgs, S, L, rb=656, replay=0, warm=None, index_mode=0, probe_retries=0):
     """Steps the given per-table trace recipes through one context (one call per iteration).
     Returns (per-iteration (hits, misses), median Stage One us of `replay` replays of the last step)."""
     n, K, n_q, T = len(cfgs), cfgs[0].topk, cfgs[0].n_q, cfgs[0].n_iters
     traces = [tr.generate(c) for c in cfgs]
     ctxlen = max(c.context for c in cfgs)
     kv = avsg.pinned_empty(ctxlen * rb)                     # the bytes do not matter here: all tables share one
-    ctx = avsg.Context(num_tables=n, buffer_slots=S, row_bytes=rb, max_topk=K, max_tokens=n_q, max_lifetime=L)
+    ctx = avsg.Context(num_tables=n, buffer_slots=S, row_bytes=rb, max_topk=K, max_tokens=n_q, max_lifetime=L,
+                       index_mode=index_mode, max_context=ctxlen + n_q, probe_retries=probe_retries)
     call = ctx.prepare(list(range(n)), [kv] * n, n_q, K)
     stream = torch.cuda.current_stream()
     per_iter, prev = [], ctx.stats()
@@ -636,6 +637,16 @@ def run_sweeps(args):
                 h = sum(a for a, _ in per[60:]); m = sum(b for _, b in per[60:])
                 row["hit_rate_%dK" % (S // 1024)] = h / (h + m)
             print(json.dumps(row), flush=True)
+    # (e) the paper's Hash-State table as printed (bounded probing, lossy) against the exact indexes
+    for n_q in (1, 2):
+        cfgs = [recipe(i, 2048, n_q, 200) for i in range(16)]
+        for label, mode, R in (("exact_hash", avsg.INDEX_HASH, 0), ("exact_direct", avsg.INDEX_DIRECT, 0),
+                               ("paper_R1", avsg.INDEX_PAPER, 1), ("paper_R3", avsg.INDEX_PAPER, 3),
+                               ("paper_R7", avsg.INDEX_PAPER, 7)):
+            per, med = _run_tables(avsg, torch, tr, cfgs, 8192, 16, replay=100, index_mode=mode, probe_retries=R)
+            h = sum(a for a, _ in per[40:]); m = sum(b for _, b in per[40:])
+            print(json.dumps({"sweep": "index_mode", "n_tokens": n_q, "index": label, "hit_rate": h / (h + m),
+                              "rows_copied_per_table_iter": m / 16 / 160, "match_reserve_us_median": med}), flush=True)
     # (d) MTP cold start: reuse inside the first iteration from an empty buffer, degrees 0..3, 32 tables
     for deg in range(4):
         per, _ = _run_tables(avsg, torch, tr, [recipe(i, 2048, deg + 1, 1) for i in range(32)], 8192, 16)

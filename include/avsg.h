@@ -61,6 +61,12 @@ extern "C" {
 #define AVSG_INDEX_DIRECT 1u  /* one 16-bit entry per context position in device memory
                                  (2 bytes x max_context per table, L2-resident); needs every
                                  id < max_context                                              */
+#define AVSG_INDEX_PAPER  2u  /* the paper's Hash-State table as printed (Eq. 2-4, Eq. 8-11,
+                                 Alg. 2): packed 64-bit entries, double hashing with a retry
+                                 budget, fingerprints, lazy reclamation.  LOSSY: a resident id
+                                 whose bucket word was overwritten is missed and fetched again,
+                                 so hit rates are lower than with the two exact indexes.  For
+                                 studying the paper's table, not for production use.           */
 
 typedef struct avsg_ctx avsg_ctx;   /* opaque */
 
@@ -75,7 +81,11 @@ typedef struct {
     int32_t  device;         /* CUDA device ordinal                                     */
     uint32_t index_mode;     /* AVSG_INDEX_*                                            */
     uint32_t max_context;    /* AVSG_INDEX_DIRECT: ids are < max_context (count the
-                                speculative positions too); ignored for AVSG_INDEX_HASH  */
+                                speculative positions too); ignored otherwise            */
+    uint32_t probe_retries;  /* AVSG_INDEX_PAPER: R, buckets per id = R + 1 (0 = the
+                                paper's default 3)                                       */
+    uint32_t hash_a1;        /* AVSG_INDEX_PAPER: the two distinct odd primes of Eq. 9   */
+    uint32_t hash_a2;        /*   (0 = 1000003 and 998244353; the paper names none)      */
 } avsg_config;
 
 typedef struct {
@@ -146,6 +156,11 @@ int avsg_sync_status(avsg_ctx *ctx, uint32_t *status_word);
  * slot, -1 empty) and life[S] (lifetime, -1 dead).  Synchronous. */
 int avsg_export_state(avsg_ctx *ctx, uint32_t table_id, int32_t *tok, int8_t *life);
 int avsg_import_state(avsg_ctx *ctx, uint32_t table_id, const int32_t *tok, const int8_t *life);
+
+/* AVSG_INDEX_PAPER only: the packed words q[S] (Eq. 2) next to the ids c[S] = tok[S].  avsg_import_state
+ * in that mode keeps ids and lifetimes but marks every bucket mapping invalid. */
+int avsg_export_hash_state(avsg_ctx *ctx, uint32_t table_id, int32_t *c, uint32_t *q);
+int avsg_import_hash_state(avsg_ctx *ctx, uint32_t table_id, const int32_t *c, const uint32_t *q);
 
 /* Device-side snapshot of every table's (tok, life) and its restore, both
  * asynchronous on the stream: lets a measurement replay one step many times. */

@@ -59,6 +59,14 @@ def _load():
     lib.orc_import.argtypes, lib.orc_import.restype = [vp, vp, vp], None
     lib.orc_rows.argtypes, lib.orc_rows.restype = [vp], vp
     lib.orc_counters.argtypes, lib.orc_counters.restype = [vp, vp], None
+    lib.orc_lit_create.argtypes, lib.orc_lit_create.restype = [u32, u32, i32, u32, u32, u32], vp
+    lib.orc_lit_destroy.argtypes, lib.orc_lit_destroy.restype = [vp], None
+    lib.orc_lit_step.argtypes = [vp, vp, u32, u32, i32, vp, u64, vp, vp, vp, vp, vp]
+    lib.orc_lit_step.restype = ctypes.c_int
+    lib.orc_lit_export.argtypes, lib.orc_lit_export.restype = [vp, vp, vp], None
+    lib.orc_lit_import.argtypes, lib.orc_lit_import.restype = [vp, vp, vp], None
+    lib.orc_lit_rows.argtypes, lib.orc_lit_rows.restype = [vp], vp
+    lib.orc_lit_counters.argtypes, lib.orc_lit_counters.restype = [vp, vp], None
     _lib = lib
     return lib
 
@@ -204,3 +212,67 @@ def workload(M: np.ndarray, X: np.ndarray, begin: int, end: int) -> int:
     M = np.ascontiguousarray(M, dtype=np.uint8).ravel()
     X = np.ascontiguousarray(X, dtype=np.int32).ravel()
     return int(_load().orc_workload(M.ctypes.data, X.ctypes.data, begin, end))
+
+
+LITERAL_A1, LITERAL_A2, LITERAL_R = 1000003, 998244353, 3     # two distinct odd primes; the paper's default retry budget
+
+
+class LiteralOracleTable:
+    """The paper-literal Hash-State table (bounded probing, fingerprints, lossy mappings)."""
+
+    def __init__(self, S: int, row_bytes: int, L: int = 16, R: int = LITERAL_R, a1: int = LITERAL_A1,
+                 a2: int = LITERAL_A2):
+        self._lib = _load()
+        self._h = self._lib.orc_lit_create(S, row_bytes, L, R, a1, a2)
+        if not self._h:
+            raise OracleError(ORC_EINVAL)
+        self.S, self.row_bytes, self.L, self.R, self.a1, self.a2 = S, row_bytes, L, R, a1, a2
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            self._lib.orc_lit_destroy(self._h)
+            self._h = None
+
+    def step(self, X: np.ndarray, N: int, host_kv: Optional[np.ndarray] = None,
+             row_stride: Optional[int] = None) -> StepResult:
+        X = np.ascontiguousarray(X, dtype=np.int32)
+        N_q, K = X.shape
+        O = np.empty((N_q, K), np.int32)
+        M = np.empty((N_q, K), np.uint8)
+        n = np.empty((N_q,), np.int32)
+        xfer = np.empty((N_q * K, 2), np.int32)
+        n_list = ctypes.c_uint32(0)
+        stride = self.row_bytes if row_stride is None else row_stride
+        kv_ptr = host_kv.ctypes.data if host_kv is not None else None
+        rc = self._lib.orc_lit_step(self._h, X.ctypes.data, N_q, K, int(N), kv_ptr, stride, O.ctypes.data,
+                                    M.ctypes.data, n.ctypes.data, xfer.ctypes.data, ctypes.byref(n_list))
+        if rc != ORC_OK:
+            raise OracleError(rc)
+        return StepResult(O, M, n, xfer[: n_list.value].copy())
+
+    def export_state(self) -> Tuple[np.ndarray, np.ndarray]:
+        """(c[S] int32, q[S] uint32 packed words)."""
+        c = np.empty(self.S, np.int32)
+        q = np.empty(self.S, np.uint32)
+        self._lib.orc_lit_export(self._h, c.ctypes.data, q.ctypes.data)
+        return c, q
+
+    def import_state(self, c: np.ndarray, q: np.ndarray) -> None:
+        c = np.ascontiguousarray(c, dtype=np.int32)
+        q = np.ascontiguousarray(q, dtype=np.uint32)
+        assert c.size == self.S and q.size == self.S
+        self._lib.orc_lit_import(self._h, c.ctypes.data, q.ctypes.data)
+
+    def lifetimes(self) -> np.ndarray:
+        return (self.export_state()[1] >> 24).astype(np.uint8).view(np.int8)
+
+    def rows(self) -> np.ndarray:
+        p = self._lib.orc_lit_rows(self._h)
+        buf = (ctypes.c_uint8 * (self.S * self.row_bytes)).from_address(p)
+        return np.frombuffer(buf, dtype=np.uint8).reshape(self.S, self.row_bytes).copy()
+
+    def counters(self) -> dict:
+        out = (ctypes.c_uint64 * 7)()
+        self._lib.orc_lit_counters(self._h, out)
+        keys = ("steps", "tokens", "hits", "misses", "rows_copied", "extra_decays", "lost_mappings")
+        return dict(zip(keys, (int(v) for v in out)))

@@ -286,3 +286,211 @@ void orc_counters(const orc_table *t, uint64_t out[6])
     out[0] = t->steps; out[1] = t->tokens; out[2] = t->hits;
     out[3] = t->misses; out[4] = t->rows_copied; out[5] = t->extra_decays;
 }
+
+/* ==========================================================================
+ * Paper-literal Hash-State mode (Sec. 3.2-3.3, App. B).
+ *
+ * The table is S 64-bit entries E_j = (c_j, q_j); q_j packs, from the most
+ * significant bit: lifetime (8, signed) | invalid (1) | fingerprint (23-m) |
+ * slot (m), S = 2^m (Eq. 2).  The lifetime belongs to SLOT j, the low 24 bits
+ * are BUCKET j's mapping.  Probing is bounded (R + 1 buckets, Eq. 8-11) and a
+ * bucket's mapping can be overwritten by another id (Alg. 2), so a resident id
+ * can be missed and fetched again: this mode is lossy by design and does not
+ * compute Eq. 1 exactly.
+ *
+ * Readings needed to make it deterministic (the paper leaves them open):
+ *   - a1, a2 are parameters (two distinct odd primes);
+ *   - "same-bucket writes retain one nondeterministic writer": here the miss
+ *     with the HIGHEST position wins;
+ *   - Alg. 2 evaluates all probes on the table as it is when UpdateState is
+ *     entered, then writes ids and lifetimes, then writes the bucket words,
+ *     reading the preserved lifetime at that moment (statement order);
+ *   - lifetime saturates at -1; initial word: lifetime -1, invalid 1;
+ *   - phi(c) of an empty slot (c = -1) is taken on the unsigned value.
+ * Beyond its own invariants (tests) this mode is "parity unpinned".
+ * ========================================================================== */
+typedef struct orc_lit_table {
+    uint32_t S, m, row_bytes, R;
+    int32_t  L;
+    uint32_t a1, a2;
+    int32_t  *c;
+    uint32_t *q;
+    uint8_t  *rows;
+    uint64_t steps, tokens, hits, misses, rows_copied, extra_decays, lost_mappings;
+} orc_lit_table;
+
+static int32_t lit_life(uint32_t q) { return (int32_t)(int8_t)(q >> 24); }
+static uint32_t lit_set_life(uint32_t q, int32_t l) { return (q & 0x00FFFFFFu) | ((uint32_t)(uint8_t)(int8_t)l << 24); }
+
+orc_lit_table *orc_lit_create(uint32_t S, uint32_t row_bytes, int32_t L, uint32_t R, uint32_t a1, uint32_t a2)
+{
+    uint32_t m = 0;
+    while ((1u << m) < S) ++m;
+    if (S < 2 || (1u << m) != S || m > 22 || L < 1 || L > 126) return NULL;
+    orc_lit_table *t = (orc_lit_table *)calloc(1, sizeof(*t));
+    if (!t) return NULL;
+    t->S = S; t->m = m; t->row_bytes = row_bytes; t->R = R; t->L = L; t->a1 = a1; t->a2 = a2;
+    t->c = (int32_t *)malloc(sizeof(int32_t) * S);
+    t->q = (uint32_t *)malloc(sizeof(uint32_t) * S);
+    t->rows = (uint8_t *)calloc((size_t)S, row_bytes ? row_bytes : 1);
+    if (!t->c || !t->q || !t->rows) { free(t->c); free(t->q); free(t->rows); free(t); return NULL; }
+    for (uint32_t j = 0; j < S; ++j) { t->c[j] = -1; t->q[j] = 0xFF800000u; }   /* dead, invalid mapping */
+    return t;
+}
+
+void orc_lit_destroy(orc_lit_table *t)
+{
+    if (!t) return;
+    free(t->c); free(t->q); free(t->rows); free(t);
+}
+
+/* Eq. 9-11: bounded double-hashing probe.  Returns 1 on a hit; *h_out is the matching bucket on a hit or
+ * the last examined bucket on a miss. */
+static int lit_probe(const orc_lit_table *t, int32_t x, uint32_t *h_out)
+{
+    const uint32_t S = t->S;
+    uint32_t h = (t->a1 * (uint32_t)x) % S;
+    const uint32_t d = ((t->a2 * (uint32_t)x) % S) | 1u;
+    int m = 0;
+    for (uint32_t r = 0; r <= t->R; ++r) {
+        const uint32_t o = t->q[h] % S;
+        m = (t->c[o] == x);
+        if (m || r == t->R) break;
+        h = (h + d) % S;
+    }
+    *h_out = h;
+    return m;
+}
+
+/* Eq. 4 with the decode chain of App. F. */
+static int lit_reusable(const orc_lit_table *t, uint32_t h)
+{
+    const uint32_t S = t->S, F = 1u << (23 - t->m);
+    const uint32_t u = t->q[h] % (2u * F * S);
+    const uint32_t b = u / (F * S), o = u % S, phi_h = (u % (F * S)) / S;
+    return b == 1 || lit_life(t->q[o]) < 0 || phi_h != ((uint32_t)t->c[o] % F);
+}
+
+static void lit_decay_all(orc_lit_table *t)
+{
+    for (uint32_t j = 0; j < t->S; ++j) {
+        int32_t l = lit_life(t->q[j]);
+        if (l > -1) t->q[j] = lit_set_life(t->q[j], l - 1);
+    }
+}
+
+/* Algorithm 1 with the literal Probe and UpdateState (Algorithm 2). */
+int32_t orc_lit_stage_one_token(orc_lit_table *t, uint32_t g, const int32_t *x, uint32_t K,
+                                int32_t *o, uint8_t *m, orc_xfer *list, uint32_t *n_list)
+{
+    const uint32_t S = t->S, F = 1u << (23 - t->m);
+    int32_t *e = (int32_t *)malloc(sizeof(int32_t) * S);
+    uint32_t *hb = (uint32_t *)malloc(sizeof(uint32_t) * (K ? K : 1));
+    uint8_t *vb = (uint8_t *)malloc(K ? K : 1);
+    if (!e || !hb || !vb) { free(e); free(hb); free(vb); return ORC_ENOMEM; }
+
+    if (g == 0) lit_decay_all(t);
+    for (uint32_t i = 0; i < K; ++i) {                       /* Probe: hit mask m and bucket indices h */
+        m[i] = 0; o[i] = -1;
+        if (x[i] < 0) continue;
+        uint32_t h;
+        if (lit_probe(t, x[i], &h)) { m[i] = 1; o[i] = (int32_t)(t->q[h] % S); }
+    }
+    for (uint32_t i = 0; i < K; ++i)
+        if (m[i]) t->q[o[i]] = lit_set_life(t->q[o[i]], t->L);
+    int32_t n_g = 0;
+    uint32_t valid = 0;
+    for (uint32_t i = 0; i < K; ++i)
+        if (x[i] >= 0) { valid++; n_g += 1 - (int32_t)m[i]; }
+
+    uint32_t n_dead = 0;
+    for (;;) {                                               /* CollectDead / decay loop */
+        n_dead = 0;
+        for (uint32_t j = 0; j < S; ++j) if (lit_life(t->q[j]) < 0) e[n_dead++] = (int32_t)j;
+        if (n_dead >= (uint32_t)n_g) break;
+        int any_alive = 0;
+        for (uint32_t j = 0; j < S; ++j) any_alive |= lit_life(t->q[j]) >= 0;
+        if (!any_alive) { free(e); free(hb); free(vb); return ORC_ECAPACITY; }
+        lit_decay_all(t);
+        t->extra_decays++;
+    }
+
+    /* UpdateState: (1) all probes on the table as it stands */
+    uint32_t k = 0;
+    for (uint32_t i = 0; i < K; ++i) {
+        if (x[i] < 0 || m[i]) continue;
+        uint32_t h = (t->a1 * (uint32_t)x[i]) % S;
+        const uint32_t d = ((t->a2 * (uint32_t)x[i]) % S) | 1u;
+        int v = 0;
+        for (uint32_t r = 0; r <= t->R; ++r) {
+            v = lit_reusable(t, h);
+            if (v || r == t->R) break;
+            h = (h + d) % S;
+        }
+        hb[k] = h; vb[k] = (uint8_t)v; ++k;
+    }
+    /* (2) every miss writes its id and lifetime into its allocated slot */
+    k = 0;
+    for (uint32_t i = 0; i < K; ++i) {
+        if (x[i] < 0 || m[i]) continue;
+        const int32_t j = e[k++];
+        t->c[j] = x[i];
+        t->q[j] = lit_set_life(t->q[j], t->L);
+        o[i] = j;
+        list[*n_list].x = x[i]; list[*n_list].o = j; (*n_list)++;
+    }
+    /* (3) bucket words, in position order: a later miss overwrites an earlier one on the same bucket */
+    k = 0;
+    for (uint32_t i = 0; i < K; ++i) {
+        if (x[i] < 0 || m[i]) continue;
+        if (vb[k]) {
+            const uint32_t h = hb[k];
+            t->q[h] = (t->q[h] & 0xFF000000u) | (((uint32_t)x[i] % F) << t->m) | (uint32_t)o[i];
+        } else {
+            t->lost_mappings++;
+        }
+        ++k;
+    }
+    t->tokens++;
+    t->hits += valid - (uint32_t)n_g;
+    t->misses += (uint32_t)n_g;
+    free(e); free(hb); free(vb);
+    return n_g;
+}
+
+int orc_lit_step(orc_lit_table *t, const int32_t *X, uint32_t N_q, uint32_t K, int32_t N,
+                 const uint8_t *host_kv, uint64_t row_stride,
+                 int32_t *O, uint8_t *M, int32_t *n, orc_xfer *list, uint32_t *n_list)
+{
+    if ((uint64_t)N_q * K > t->S) return ORC_ECAPACITY;
+    *n_list = 0;
+    for (uint32_t g = 0; g < N_q; ++g) {
+        int32_t r = orc_lit_stage_one_token(t, g, X + (size_t)g * K, K, O + (size_t)g * K, M + (size_t)g * K, list, n_list);
+        if (r < 0) return r;
+        n[g] = r;
+    }
+    if (host_kv)
+        for (uint32_t k = 0; k < *n_list; ++k)
+            memcpy(t->rows + (size_t)list[k].o * t->row_bytes, host_kv + (uint64_t)list[k].x * row_stride, t->row_bytes);
+    t->rows_copied += *n_list;
+    for (uint32_t j = 0; j < t->S; ++j) if (t->c[j] >= N) t->c[j] = -1;
+    t->steps++;
+    return ORC_OK;
+}
+
+void orc_lit_export(const orc_lit_table *t, int32_t *c, uint32_t *q)
+{
+    memcpy(c, t->c, sizeof(int32_t) * t->S);
+    memcpy(q, t->q, sizeof(uint32_t) * t->S);
+}
+void orc_lit_import(orc_lit_table *t, const int32_t *c, const uint32_t *q)
+{
+    memcpy(t->c, c, sizeof(int32_t) * t->S);
+    memcpy(t->q, q, sizeof(uint32_t) * t->S);
+}
+const uint8_t *orc_lit_rows(const orc_lit_table *t) { return t->rows; }
+void orc_lit_counters(const orc_lit_table *t, uint64_t out[7])
+{
+    out[0] = t->steps; out[1] = t->tokens; out[2] = t->hits; out[3] = t->misses;
+    out[4] = t->rows_copied; out[5] = t->extra_decays; out[6] = t->lost_mappings;
+}

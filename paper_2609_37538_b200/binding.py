@@ -17,13 +17,13 @@ from . import build as _build
 
 OK, EINVAL, ENOMEM, ECUDA, ECAPACITY, EDEVICE_STATUS, EUNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
 XFER_SM_BALANCED, XFER_COPY_ENGINE, XFER_REQUEST_LEVEL, XFER_ALL_K, XFER_POSITION_LEVEL = 0, 1, 2, 3, 4
-INDEX_HASH, INDEX_DIRECT = 0, 1
+INDEX_HASH, INDEX_DIRECT, INDEX_PAPER = 0, 1, 2
 
 EXPORTS = (
     "avsg_create", "avsg_destroy", "avsg_reset", "avsg_step", "avsg_step_host", "avsg_buffer", "avsg_stats",
     "avsg_sync_status", "avsg_export_state", "avsg_import_state", "avsg_save_state", "avsg_restore_state",
     "avsg_set_transfer_mode", "avsg_set_timing", "avsg_set_transfer_geometry", "avsg_strerror",
-    "avsg_step_noalloc",
+    "avsg_step_noalloc", "avsg_export_hash_state", "avsg_import_hash_state",
 )
 
 
@@ -31,7 +31,8 @@ class AvsgConfig(ctypes.Structure):
     _fields_ = [("num_tables", ctypes.c_uint32), ("buffer_slots", ctypes.c_uint32), ("row_bytes", ctypes.c_uint32),
                 ("max_topk", ctypes.c_uint32), ("max_tokens", ctypes.c_uint32), ("max_lifetime", ctypes.c_int32),
                 ("transfer_mode", ctypes.c_uint32), ("device", ctypes.c_int32), ("index_mode", ctypes.c_uint32),
-                ("max_context", ctypes.c_uint32)]
+                ("max_context", ctypes.c_uint32), ("probe_retries", ctypes.c_uint32), ("hash_a1", ctypes.c_uint32),
+                ("hash_a2", ctypes.c_uint32)]
 
 
 class AvsgStepArgs(ctypes.Structure):
@@ -96,6 +97,8 @@ def load_library():
     lib.avsg_set_transfer_geometry.argtypes, lib.avsg_set_transfer_geometry.restype = [vp, u32, u32], i32
     lib.avsg_strerror.argtypes, lib.avsg_strerror.restype = [i32], ctypes.c_char_p
     lib.avsg_step_noalloc.argtypes, lib.avsg_step_noalloc.restype = [ctypes.POINTER(AvsgNoAllocArgs), vp], i32
+    lib.avsg_export_hash_state.argtypes, lib.avsg_export_hash_state.restype = [vp, u32, vp, vp], i32
+    lib.avsg_import_hash_state.argtypes, lib.avsg_import_hash_state.restype = [vp, u32, vp, vp], i32
     _lib = lib
     return lib
 
@@ -186,11 +189,12 @@ class Context:
 
     def __init__(self, num_tables: int, buffer_slots: int, row_bytes: int, max_topk: int, max_tokens: int = 1,
                  max_lifetime: int = 16, transfer_mode: int = XFER_SM_BALANCED, device: int = 0,
-                 index_mode: int = INDEX_HASH, max_context: int = 0):
+                 index_mode: int = INDEX_HASH, max_context: int = 0, probe_retries: int = 0, hash_a1: int = 0,
+                 hash_a2: int = 0):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         cfg = AvsgConfig(num_tables, buffer_slots, row_bytes, max_topk, max_tokens, max_lifetime, transfer_mode,
-                         device, index_mode, max_context)
+                         device, index_mode, max_context, probe_retries, hash_a1, hash_a2)
         _check(self._lib.avsg_create(ctypes.byref(cfg), ctypes.byref(self._h)), "avsg_create")
         self.num_tables, self.S, self.row_bytes = num_tables, buffer_slots, row_bytes
         self.max_topk, self.max_tokens, self.L, self.device = max_topk, max_tokens, max_lifetime, device
@@ -260,6 +264,21 @@ class Context:
         life = np.ascontiguousarray(life, dtype=np.int8)
         assert tok.size == self.S and life.size == self.S
         _check(self._lib.avsg_import_state(self._h, table_id, tok.ctypes.data, life.ctypes.data), "avsg_import_state")
+
+    def export_hash_state(self, table_id: int):
+        """Paper-literal mode: (c[S] int32, q[S] uint32 packed words)."""
+        c = np.empty(self.S, np.int32)
+        q = np.empty(self.S, np.uint32)
+        _check(self._lib.avsg_export_hash_state(self._h, table_id, c.ctypes.data, q.ctypes.data),
+               "avsg_export_hash_state")
+        return c, q
+
+    def import_hash_state(self, table_id: int, c, q) -> None:
+        c = np.ascontiguousarray(c, dtype=np.int32)
+        q = np.ascontiguousarray(q, dtype=np.uint32)
+        assert c.size == self.S and q.size == self.S
+        _check(self._lib.avsg_import_hash_state(self._h, table_id, c.ctypes.data, q.ctypes.data),
+               "avsg_import_hash_state")
 
     def save_state(self, stream=None) -> None:
         _check(self._lib.avsg_save_state(self._h, _stream_handle(stream)), "avsg_save_state")

@@ -26,6 +26,8 @@ struct avsg_ctx {
     SegDesc* d_seg = nullptr;
     uint32_t* d_status = nullptr;
     uint16_t* d_where = nullptr;       // direct index, or null
+    uint32_t* d_q = nullptr;           // paper-literal mode: packed words, or null
+    uint32_t* d_q_snap = nullptr;
     int32_t* d_tok_snap = nullptr;
     int8_t* d_life_snap = nullptr;
     // staging of avsg_step_host
@@ -69,7 +71,7 @@ uint32_t ilog2(uint32_t v) { uint32_t l = 0; while ((1u << l) < v) ++l; return l
 void free_all(avsg_ctx* c)
 {
     cudaFree(c->d_tok); cudaFree(c->d_life); cudaFree(c->d_buffer); cudaFree(c->d_stats);
-    cudaFree(c->d_list); cudaFree(c->d_seg); cudaFree(c->d_status); cudaFree(c->d_where);
+    cudaFree(c->d_list); cudaFree(c->d_seg); cudaFree(c->d_status); cudaFree(c->d_where); cudaFree(c->d_q); cudaFree(c->d_q_snap);
     cudaFree(c->d_tok_snap); cudaFree(c->d_life_snap);
     cudaFree(c->d_idx_stage); cudaFree(c->d_slots_stage); cudaFree(c->d_hit_stage); cudaFree(c->d_mc_stage);
     if (c->h_seg) cudaFreeHost(c->h_seg);
@@ -87,6 +89,10 @@ int init_tables(avsg_ctx* c, uint32_t first, uint32_t n)
     CU(cudaMemset(c->d_life + first * S, 0xFF, n * S));                         // lifetime -1: dead
     CU(cudaMemset(c->d_buffer + first * S * c->cfg.row_bytes, 0, n * S * c->cfg.row_bytes));
     CU(cudaMemset(c->d_stats + first, 0, n * sizeof(TableStats)));
+    if (c->d_q) {                                           // lifetime -1, mapping invalid: 0xFF800000
+        std::vector<uint32_t> init(n * S, 0xFF800000u);
+        CU(cudaMemcpy(c->d_q + first * S, init.data(), init.size() * sizeof(uint32_t), cudaMemcpyHostToDevice));
+    }
     return AVSG_OK;
 }
 
@@ -206,6 +212,7 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
             p.K = K; p.n_q = n_q; p.L = (uint32_t)c->cfg.max_lifetime;
             p.first = first; p.list_stride = c->list_stride;
             p.where = c->d_where; p.max_context = c->cfg.max_context;
+            p.qword = c->d_q; p.probe_retries = c->cfg.probe_retries; p.hash_a1 = c->cfg.hash_a1; p.hash_a2 = c->cfg.hash_a2;
             for (uint32_t i = 0; i < cnt; ++i) {
                 p.table_id[i] = a->table_ids[first + i];
                 p.verified_len[i] = a->verified_len[first + i];
@@ -270,7 +277,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     if (cfg->row_bytes == 0 || cfg->row_bytes % 16) return AVSG_EINVAL;
     if (cfg->max_topk == 0 || cfg->max_tokens == 0) return AVSG_EINVAL;
     if (cfg->max_lifetime < 1 || cfg->max_lifetime > 126) return AVSG_EINVAL;
-    if (cfg->transfer_mode > AVSG_XFER_POSITION_LEVEL || cfg->index_mode > AVSG_INDEX_DIRECT) return AVSG_EINVAL;
+    if (cfg->transfer_mode > AVSG_XFER_POSITION_LEVEL || cfg->index_mode > AVSG_INDEX_PAPER) return AVSG_EINVAL;
     if (cfg->index_mode == AVSG_INDEX_DIRECT && cfg->max_context == 0) return AVSG_EINVAL;
     if ((uint64_t)cfg->max_topk * cfg->max_tokens > cfg->buffer_slots) return AVSG_ECAPACITY;   // Eq. 7
     int ndev = 0;
@@ -281,6 +288,9 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     avsg_ctx* c = new (std::nothrow) avsg_ctx();
     if (!c) return AVSG_ENOMEM;
     c->cfg = *cfg;
+    if (c->cfg.probe_retries == 0) c->cfg.probe_retries = 3;
+    if (c->cfg.hash_a1 == 0) c->cfg.hash_a1 = 1000003u;
+    if (c->cfg.hash_a2 == 0) c->cfg.hash_a2 = 998244353u;
     c->logS = ilog2(cfg->buffer_slots);
     c->logH = c->logS + 1;
     c->list_stride = cfg->max_topk * cfg->max_tokens;
@@ -290,8 +300,10 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     int max_smem = 0;
     cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, cfg->device);
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device);
-    const size_t need = stage_one_smem_bytes(cfg->buffer_slots, cfg->max_topk, (uint32_t)cfg->max_lifetime,
-                                             cfg->index_mode == AVSG_INDEX_DIRECT);
+    const size_t need = cfg->index_mode == AVSG_INDEX_PAPER
+        ? stage_one_paper_smem_bytes(cfg->buffer_slots, cfg->max_topk, (uint32_t)cfg->max_lifetime)
+        : stage_one_smem_bytes(cfg->buffer_slots, cfg->max_topk, (uint32_t)cfg->max_lifetime,
+                               cfg->index_mode == AVSG_INDEX_DIRECT);
     if (need > (size_t)max_smem) { delete c; return AVSG_EUNSUPPORTED; }
     // always raise the kernel's dynamic shared-memory limit to the device maximum: the attribute is
     // per function, so a context with a small table must not lower it under a context with a large one
@@ -306,6 +318,10 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaMalloc(&c->d_list, n_ids * sizeof(int2)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_seg, T * sizeof(SegDesc)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_status, 256) == cudaSuccess;
+    if (cfg->index_mode == AVSG_INDEX_PAPER) {
+        ok = ok && cudaMalloc(&c->d_q, T * S * sizeof(uint32_t)) == cudaSuccess;
+        ok = ok && cudaMalloc(&c->d_q_snap, T * S * sizeof(uint32_t)) == cudaSuccess;
+    }
     if (cfg->index_mode == AVSG_INDEX_DIRECT)
         ok = ok && cudaMalloc(&c->d_where, T * (size_t)cfg->max_context * sizeof(uint16_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_tok_snap, T * S * sizeof(int32_t)) == cudaSuccess;
@@ -434,6 +450,41 @@ int avsg_import_state(avsg_ctx* c, uint32_t table_id, const int32_t* tok, const 
         CU(launch_direct_index_from_state(c->d_tok, c->d_where, table_id, 1, c->cfg.buffer_slots, c->cfg.max_context, nullptr));
         CU(cudaDeviceSynchronize());
     }
+    if (c->d_q) {                                           // ids and lifetimes kept, every mapping invalid
+        std::vector<uint32_t> q(S);
+        for (size_t j = 0; j < S; ++j) q[j] = ((uint32_t)(uint8_t)life[j] << 24) | 0x00800000u;
+        CU(cudaMemcpy(c->d_q + table_id * S, q.data(), S * sizeof(uint32_t), cudaMemcpyHostToDevice));
+    }
+    return AVSG_OK;
+}
+
+int avsg_export_hash_state(avsg_ctx* c, uint32_t table_id, int32_t* cc, uint32_t* q)
+{
+    if (!c || !cc || !q || table_id >= c->cfg.num_tables || !c->d_q) return AVSG_EINVAL;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return AVSG_ECUDA;
+    const size_t S = c->cfg.buffer_slots;
+    CU(cudaDeviceSynchronize());
+    CU(cudaMemcpy(cc, c->d_tok + table_id * S, S * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    CU(cudaMemcpy(q, c->d_q + table_id * S, S * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    return read_status(c, nullptr);
+}
+
+int avsg_import_hash_state(avsg_ctx* c, uint32_t table_id, const int32_t* cc, const uint32_t* q)
+{
+    if (!c || !cc || !q || table_id >= c->cfg.num_tables || !c->d_q) return AVSG_EINVAL;
+    const size_t S = c->cfg.buffer_slots;
+    std::vector<int8_t> life(S);
+    for (size_t j = 0; j < S; ++j) {
+        life[j] = (int8_t)(q[j] >> 24);
+        if (life[j] < -1 || life[j] > c->cfg.max_lifetime || cc[j] < -1) return AVSG_EINVAL;
+    }
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return AVSG_ECUDA;
+    CU(cudaDeviceSynchronize());
+    CU(cudaMemcpy(c->d_tok + table_id * S, cc, S * sizeof(int32_t), cudaMemcpyHostToDevice));
+    CU(cudaMemcpy(c->d_q + table_id * S, q, S * sizeof(uint32_t), cudaMemcpyHostToDevice));
+    CU(cudaMemcpy(c->d_life + table_id * S, life.data(), S, cudaMemcpyHostToDevice));
     return AVSG_OK;
 }
 
@@ -446,6 +497,7 @@ int avsg_save_state(avsg_ctx* c, void* stream)
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     CU(cudaMemcpyAsync(c->d_tok_snap, c->d_tok, n * sizeof(int32_t), cudaMemcpyDeviceToDevice, s));
     CU(cudaMemcpyAsync(c->d_life_snap, c->d_life, n, cudaMemcpyDeviceToDevice, s));
+    if (c->d_q) CU(cudaMemcpyAsync(c->d_q_snap, c->d_q, n * sizeof(uint32_t), cudaMemcpyDeviceToDevice, s));
     return AVSG_OK;
 }
 
@@ -458,6 +510,7 @@ int avsg_restore_state(avsg_ctx* c, void* stream)
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     CU(cudaMemcpyAsync(c->d_tok, c->d_tok_snap, n * sizeof(int32_t), cudaMemcpyDeviceToDevice, s));
     CU(cudaMemcpyAsync(c->d_life, c->d_life_snap, n, cudaMemcpyDeviceToDevice, s));
+    if (c->d_q) CU(cudaMemcpyAsync(c->d_q, c->d_q_snap, n * sizeof(uint32_t), cudaMemcpyDeviceToDevice, s));
     if (c->d_where)
         CU(launch_direct_index_from_state(c->d_tok, c->d_where, 0, c->cfg.num_tables, c->cfg.buffer_slots,
                                           c->cfg.max_context, s));

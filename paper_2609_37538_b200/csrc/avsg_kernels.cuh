@@ -51,6 +51,8 @@ struct S1Params {
     uint32_t list_stride;        // entries per segment of miss_list
     uint32_t max_context;        // direct index: entries per table
     uint16_t* where;             // direct index [num_tables][max_context], or null for the hash index
+    uint32_t* qword;             // paper-literal mode: packed metadata words [num_tables][S], else null
+    uint32_t probe_retries, hash_a1, hash_a2;   // paper-literal mode: R, a1, a2
     uint32_t table_id[S1_MAX_TABLES];
     int32_t  verified_len[S1_MAX_TABLES];
     uint64_t kv_base[S1_MAX_TABLES];
@@ -89,6 +91,7 @@ struct AllKParams {
 };
 
 size_t stage_one_smem_bytes(uint32_t S, uint32_t K, uint32_t L, bool direct = false);
+size_t stage_one_paper_smem_bytes(uint32_t S, uint32_t K, uint32_t L);
 uint32_t stage_one_threads(uint32_t S, uint32_t K);
 cudaError_t stage_one_prepare(size_t max_smem);
 cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream);

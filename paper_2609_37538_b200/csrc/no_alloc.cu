@@ -94,6 +94,7 @@ extern "C" int avsg_step_noalloc(const avsg_noalloc_args* a, void* cuda_stream)
     p.S = a->buffer_slots; p.row_bytes = a->row_bytes; p.K = a->topk; p.n_q = a->n_tokens;
     p.L = (uint32_t)a->max_lifetime; p.first = 0; p.list_stride = list_stride;
     p.where = nullptr; p.max_context = 0;
+    p.qword = nullptr; p.probe_retries = 0; p.hash_a1 = 0; p.hash_a2 = 0;
     p.logH = 1;
     while ((1u << p.logH) < 2u * a->buffer_slots) ++p.logH;
     for (uint32_t i = 0; i < a->n; ++i) {

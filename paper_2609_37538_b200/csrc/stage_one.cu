@@ -518,6 +518,258 @@ __global__ void avsg_direct_index_from_state_kernel(const int32_t* __restrict__ 
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------------------------
+// Paper-literal Hash-State mode (Sec. 3.2-3.3, Eq. 2-4, Eq. 8-11, Algorithm 2): 64-bit entries (c_j, q_j) with
+// q_j = [lifetime 8 | invalid 1 | fingerprint 23-m | slot m], double hashing with retry budget R, fingerprint
+// check and lazy reclamation of stale bucket words.  Lossy by design: a resident id whose bucket word was
+// overwritten is missed and fetched again.  Where Algorithm 2 leaves "one nondeterministic writer" per bucket,
+// the miss with the highest position wins (an atomicMax on a per-bucket tag), so results are reproducible.
+// ---------------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pack_life_bytes(const uint32_t* q, uint32_t j0, uint32_t spt, bool own,
+                                                uint32_t& w0, uint32_t& w1)
+{
+    w0 = w1 = 0x7F7F7F7Fu;
+    if (!own) return;
+#pragma unroll
+    for (uint32_t k = 0; k < (uint32_t)MAX_SPT; ++k) {
+        if (k < spt) {
+            const uint32_t b = q[j0 + k] >> 24;
+            if (k < 4) w0 = (w0 & ~(0xFFu << (8 * k))) | (b << (8 * k));
+            else w1 = (w1 & ~(0xFFu << (8 * (k - 4)))) | (b << (8 * (k - 4)));
+        }
+    }
+}
+
+__device__ __forceinline__ void unpack_life_bytes(uint32_t* q, uint32_t j0, uint32_t spt, bool own, uint32_t w0, uint32_t w1)
+{
+    if (!own) return;
+#pragma unroll
+    for (uint32_t k = 0; k < (uint32_t)MAX_SPT; ++k) {
+        if (k < spt) {
+            const uint32_t b = k < 4 ? (w0 >> (8 * k)) & 0xFFu : (w1 >> (8 * (k - 4))) & 0xFFu;
+            q[j0 + k] = (q[j0 + k] & 0x00FFFFFFu) | (b << 24);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(1024, 1) avsg_stage_one_paper_kernel(const __grid_constant__ S1Params p)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    const uint32_t S = p.S, K = p.K, Kp = (K + 7u) & ~7u, m = p.logH - 1u, Fm = (1u << (23u - m)) - 1u;
+    const uint32_t tid = threadIdx.x, nt = blockDim.x, R = p.probe_retries, a1 = p.hash_a1, a2 = p.hash_a2;
+    const int32_t L = (int32_t)p.L;
+
+    int32_t*  s_c        = reinterpret_cast<int32_t*>(smem);
+    uint32_t* s_q        = reinterpret_cast<uint32_t*>(s_c + S);
+    uint32_t* s_win      = s_q + S;                                   // per-bucket winner tag of UpdateState
+    int32_t*  s_miss_x   = reinterpret_cast<int32_t*>(s_win + S);
+    uint16_t* s_miss_pos = reinterpret_cast<uint16_t*>(s_miss_x + Kp);
+    uint16_t* s_dead     = s_miss_pos + Kp;
+    uint16_t* s_bucket   = s_dead + Kp;                               // bit 15: a reusable bucket was found
+    uint32_t* s_hist     = reinterpret_cast<uint32_t*>(s_bucket + Kp);
+    uint32_t* s_scan_a   = s_hist + 128;
+    uint32_t* s_scan_b   = s_scan_a + 40;
+    const uint32_t priv_stride = nt + 4u;
+    uint8_t*  s_priv     = L <= PRIV_HIST_MAX_L ? reinterpret_cast<uint8_t*>(s_scan_b + 40) : nullptr;
+
+    const uint32_t ti = p.first + blockIdx.x, table = p.table_id[blockIdx.x];
+    int32_t*  g_c = p.tok + (size_t)table * S;
+    uint32_t* g_q = p.qword + (size_t)table * S;
+    int8_t*   g_life = p.life + (size_t)table * S;
+    const uint32_t spt = S >= nt ? S / nt : 1u, j0 = tid * spt;
+    const bool own = j0 < S;
+    const uint32_t ipt = (K + nt - 1) / nt, i0 = tid * ipt;
+
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    // ---- load the table; global pre-decay ----
+    if (own)
+        for (uint32_t k = 0; k < spt; ++k) {
+            s_c[j0 + k] = __ldg(g_c + j0 + k);
+            s_q[j0 + k] = __ldg(g_q + j0 + k);
+            s_win[j0 + k] = 0;
+        }
+    if (s_priv)
+        for (uint32_t i = tid; i < ((uint32_t)(L + 2) * priv_stride + 15u) / 16u; i += nt)
+            reinterpret_cast<int4*>(s_priv)[i] = make_int4(0, 0, 0, 0);
+    int32_t xs[MAX_IPT];
+    load_ids(p.indices + (size_t)ti * p.n_q * K, i0, ipt, K, xs);
+    __syncthreads();
+    {
+        uint32_t w0, w1;
+        pack_life_bytes(s_q, j0, spt, own, w0, w1);
+        unpack_life_bytes(s_q, j0, spt, own, decay4(w0, 1), decay4(w1, 1));
+    }
+    __syncthreads();
+
+    uint32_t list_off = 0, sum_valid = 0, sum_miss = 0, sum_decay = 0;
+    int2* list = p.miss_list + (size_t)ti * p.list_stride;
+
+    for (uint32_t g = 0; g < p.n_q; ++g) {
+        const size_t row = ((size_t)ti * p.n_q + g) * K;
+        int32_t* O = p.slots + row;
+        uint8_t* Hm = p.hit ? p.hit + row : nullptr;
+        if (tid < 128) s_hist[tid] = 0;
+
+        // ---- Probe (Eq. 8-11): at most R + 1 buckets; the full id is compared ----
+        uint32_t missmask = 0, nmiss = 0, nvalid = 0;
+#pragma unroll
+        for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {
+            const uint32_t i = i0 + k;
+            if (k < ipt && i < K) {
+                const int32_t x = xs[k];
+                if (x >= 0) {
+                    ++nvalid;
+                    uint32_t h = (a1 * (uint32_t)x) & (S - 1u);
+                    const uint32_t d = ((a2 * (uint32_t)x) & (S - 1u)) | 1u;
+                    int32_t j = -1;
+                    for (uint32_t r = 0; r <= R; ++r) {
+                        const uint32_t o = s_q[h] & (S - 1u);
+                        if (s_c[o] == x) { j = (int32_t)o; break; }
+                        if (r < R) h = (h + d) & (S - 1u);
+                    }
+                    if (j >= 0) {
+                        reinterpret_cast<uint8_t*>(s_q)[4u * (uint32_t)j + 3u] = (uint8_t)L;    // lifetime <- L
+                        O[i] = j;
+                        if (Hm) Hm[i] = 1;
+                    } else {
+                        missmask |= 1u << k;
+                        ++nmiss;
+                    }
+                } else {
+                    O[i] = -1;
+                    if (Hm) Hm[i] = 0;
+                }
+            }
+        }
+        uint32_t total;
+        uint32_t off = block_excl_scan(nmiss | (nvalid << 16), s_scan_a, total) & 0xFFFFu;
+        const uint32_t n_g = total & 0xFFFFu;
+        sum_valid += total >> 16;
+        sum_miss += n_g;
+#pragma unroll
+        for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {
+            if (missmask & (1u << k)) {
+                s_miss_x[off] = xs[k];
+                s_miss_pos[off] = (uint16_t)(i0 + k);
+                ++off;
+            }
+        }
+        if (g + 1 < p.n_q) load_ids(p.indices + row + K, i0, ipt, K, xs);
+        if (tid == 0 && p.miss_count) p.miss_count[(size_t)ti * p.n_q + g] = (int32_t)n_g;
+        if (n_g == 0) { __syncthreads(); continue; }
+        __syncthreads();
+
+        // ---- CollectDead / decay until n_g slots are dead ----
+        uint32_t w0, w1;
+        pack_life_bytes(s_q, j0, spt, own, w0, w1);
+        uint32_t sg0 = w0 & 0x80808080u, sg1 = w1 & 0x80808080u;
+        uint32_t dtotal, d = 0;
+        uint32_t doff = block_excl_scan(__popc(sg0) + __popc(sg1), s_scan_b, dtotal);
+        if (dtotal < n_g) {
+            count_lifetimes(w0, w1, spt, own, L, s_priv, priv_stride, s_hist);
+            __syncthreads();
+            uint32_t cum = 0;
+            bool found = false;
+            d = (uint32_t)L + 1u;
+            for (uint32_t b = 0; b <= (uint32_t)L + 1u; ++b) {
+                cum += s_hist[b];
+                if (cum >= n_g) { d = b; found = true; break; }
+            }
+            if (!found && tid == 0) atomicOr(p.status, ST_NO_DEAD_SLOTS);
+            w0 = decay4(w0, d);
+            w1 = decay4(w1, d);
+            unpack_life_bytes(s_q, j0, spt, own, w0, w1);
+            sg0 = w0 & 0x80808080u; sg1 = w1 & 0x80808080u;
+            doff = block_excl_scan(__popc(sg0) + __popc(sg1), s_scan_b, dtotal);
+        }
+#pragma unroll
+        for (uint32_t k = 0; k < (uint32_t)MAX_SPT; ++k) {
+            const uint32_t bit = k < 4 ? (sg0 >> (8 * k + 7)) & 1u : (sg1 >> (8 * (k - 4) + 7)) & 1u;
+            if (bit) {
+                if (doff < n_g) s_dead[doff] = (uint16_t)(j0 + k);
+                ++doff;
+            }
+        }
+        __syncthreads();
+        const uint32_t n_take = n_g < dtotal ? n_g : dtotal;
+
+        // ---- UpdateState (1): every miss looks for a reusable bucket on the table as it stands (Eq. 4) ----
+        for (uint32_t k = tid; k < n_take; k += nt) {
+            const int32_t x = s_miss_x[k];
+            uint32_t h = (a1 * (uint32_t)x) & (S - 1u);
+            const uint32_t dd = ((a2 * (uint32_t)x) & (S - 1u)) | 1u;
+            uint32_t v = 0;
+            for (uint32_t r = 0; r <= R; ++r) {
+                const uint32_t qh = s_q[h], o = qh & (S - 1u);
+                const uint32_t invalid = (qh >> 23) & 1u, fp = (qh >> m) & Fm;
+                const int32_t life_o = (int32_t)(int8_t)(s_q[o] >> 24);
+                v = invalid | (uint32_t)(life_o < 0) | (uint32_t)(fp != ((uint32_t)s_c[o] & Fm));
+                if (v || r == R) break;
+                h = (h + dd) & (S - 1u);
+            }
+            s_bucket[k] = (uint16_t)(h | (v ? 0x8000u : 0u));
+        }
+        __syncthreads();
+        // ---- (2): ids and lifetimes go into the allocated slots ----
+        for (uint32_t k = tid; k < n_take; k += nt) {
+            const uint32_t j = s_dead[k], i = s_miss_pos[k];
+            const int32_t x = s_miss_x[k];
+            if (j < S && i < K) {
+                s_c[j] = x;
+                reinterpret_cast<uint8_t*>(s_q)[4u * j + 3u] = (uint8_t)L;
+                O[i] = (int32_t)j;
+                if (Hm) Hm[i] = 0;
+                list[list_off + k] = make_int2(x, (int32_t)j);
+                if (s_bucket[k] & 0x8000u) atomicMax(&s_win[s_bucket[k] & 0x7FFFu], ((g + 1u) << 16) | k);
+            } else {
+                list[list_off + k] = make_int2(-1, -1);
+                atomicOr(p.status, ST_BAD_SLOT);
+            }
+        }
+        __syncthreads();
+        // ---- (3): the bucket word keeps its slot's lifetime, takes fingerprint and slot, becomes valid ----
+        for (uint32_t k = tid; k < n_take; k += nt) {
+            const uint32_t hb = s_bucket[k];
+            if ((hb & 0x8000u) && s_win[hb & 0x7FFFu] == (((g + 1u) << 16) | k)) {
+                const uint32_t h = hb & 0x7FFFu;
+                s_q[h] = (s_q[h] & 0xFF000000u) | (((uint32_t)s_miss_x[k] & Fm) << m) | (uint32_t)s_dead[k];
+            }
+        }
+        list_off += n_take;
+        sum_decay += d;
+        __syncthreads();
+    }
+
+    // ---- write back; speculative entries (id >= N) become empty ----
+    const int32_t N = p.verified_len[blockIdx.x];
+    if (own)
+        for (uint32_t k = 0; k < spt; ++k) {
+            const int32_t v = s_c[j0 + k];
+            g_c[j0 + k] = v >= N ? -1 : v;
+            g_q[j0 + k] = s_q[j0 + k];
+            g_life[j0 + k] = (int8_t)(s_q[j0 + k] >> 24);
+        }
+    if (tid == 0) {
+        SegDesc sd;
+        sd.src_base = p.kv_base[blockIdx.x];
+        sd.src_stride = p.kv_stride[blockIdx.x];
+        sd.dst_base = reinterpret_cast<uint64_t>(p.buffer + (size_t)table * S * p.row_bytes);
+        sd.count = list_off;
+        sd.pad = 0;
+        p.seg[ti] = sd;
+        TableStats* st = p.stats + table;
+        st->steps += 1;
+        st->tokens += p.n_q;
+        st->hits += sum_valid - sum_miss;
+        st->misses += sum_miss;
+        st->rows += list_off;
+        st->extra_decays += sum_decay;
+    }
+}
+
 // "KV offload" comparator: every selected row moves, position (g, i) -> slot g*K + i.
 __global__ void __launch_bounds__(256) avsg_all_k_prepare_kernel(const __grid_constant__ AllKParams p)
 {
@@ -570,6 +822,14 @@ size_t stage_one_smem_bytes(uint32_t S, uint32_t K, uint32_t L, bool direct)
     return n;
 }
 
+size_t stage_one_paper_smem_bytes(uint32_t S, uint32_t K, uint32_t L)
+{
+    const size_t Kp = (K + 7u) & ~7u;
+    size_t n = S * 12 + Kp * 4 + Kp * 2 * 3 + (128 + 40 + 40) * 4;
+    if ((int32_t)L <= PRIV_HIST_MAX_L) n += ((size_t)(L + 2) * (stage_one_threads(S, K) + 4) + 15) / 16 * 16;
+    return n;
+}
+
 uint32_t stage_one_threads(uint32_t S, uint32_t K)
 {
     (void)K;
@@ -583,7 +843,9 @@ cudaError_t stage_one_prepare(size_t max_smem)
 {
     cudaError_t e = cudaFuncSetAttribute(avsg_stage_one_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(avsg_stage_one_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    e = cudaFuncSetAttribute(avsg_stage_one_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(avsg_stage_one_paper_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
 }
 
 cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream)
@@ -591,14 +853,15 @@ cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_tables);
     cfg.blockDim = dim3(stage_one_threads(p.S, p.K));
-    const bool direct = p.where != nullptr;
-    cfg.dynamicSmemBytes = stage_one_smem_bytes(p.S, p.K, p.L, direct);
+    const bool direct = p.where != nullptr, paper = p.qword != nullptr;
+    cfg.dynamicSmemBytes = paper ? stage_one_paper_smem_bytes(p.S, p.K, p.L) : stage_one_smem_bytes(p.S, p.K, p.L, direct);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (paper) return cudaLaunchKernelEx(&cfg, avsg_stage_one_paper_kernel, p);
     return direct ? cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel<true>, p)
                   : cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel<false>, p);
 }
