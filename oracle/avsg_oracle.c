@@ -15,6 +15,7 @@
  *   - balanced miss partition .......... Eq. 6, Sec. 3.4
  *   - request-level assignment ......... Eq. 13 (comparator S1)
  *   - equal top-K position partition ... Eq. 14 (comparator S2)
+ *   - paper-literal Hash-State mode .... Eq. 2-4, Eq. 8-11, Algorithm 2 (second half of this file)
  *
  * Readings taken where the paper is silent or ambiguous (all listed in the
  * design notes of the repository):
