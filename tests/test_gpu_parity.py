@@ -379,3 +379,36 @@ def test_paper_literal_mode_full_c2_and_small_c3(avsg):
 ])
 def test_paper_literal_mode_shapes(avsg, kw, R):
     _literal_parity(avsg, tr.workload("C2", **kw), R=R)
+
+
+# ---- randomly drawn shapes: tables, S, K, tokens, L, row size, index and transfer mode -------------------------------
+@pytest.mark.parametrize("seed", range(12))
+def test_random_shapes(avsg, seed):
+    rng = np.random.default_rng(1000 + seed)
+    S = int(2 ** rng.integers(5, 14))                                  # 32 .. 8192
+    n_q = int(rng.choice([1, 1, 2, 2, 3, 4]))
+    k_max = S // n_q
+    K = int(rng.integers(1, k_max + 1)) if rng.random() < 0.3 else int(min(k_max, 2 ** rng.integers(0, 12)))
+    L = int(rng.choice([1, 2, 8, 16, 30, 31, 64]))
+    rb = int(rng.choice([16, 48, 656, 1152]))
+    requests = int(rng.choice([1, 2, 5, 9]))
+    ctxlen = int(max(2 * K * n_q, rng.integers(K * n_q + 8, 40 * K * n_q + 64)))
+    base = rng.choice(["C2", "C4", "C5"])
+    kw = dict(topk=K, buffer_slots=S, n_iters=int(rng.integers(3, 14)), max_lifetime=L, row_bytes=rb)
+    if base == "C2":
+        w = tr.workload("C2", context=ctxlen, recent_window=max(1, ctxlen // 8), **kw)
+        if n_q != 2:
+            base = "C5"
+    if base == "C4":
+        w = tr.workload("C4", context=ctxlen, requests=requests, hot_size=min(64, ctxlen // 4),
+                        hot_range=max(64, ctxlen // 2), **kw)
+        if n_q != 2:
+            base = "C5"
+    if base == "C5":
+        w = tr.workload("C5", requests=requests, ctx_lo=max(4, K // 2), ctx_hi=ctxlen, **kw)
+    if w.n_q * w.topk > w.buffer_slots:                                  # the MTP recipes have two tokens
+        w = tr.workload("C5", requests=requests, ctx_lo=max(4, K // 2), ctx_hi=ctxlen, **kw)
+    mode = getattr(avsg, str(rng.choice(["XFER_SM_BALANCED", "XFER_REQUEST_LEVEL", "XFER_POSITION_LEVEL"])))
+    index_mode = int(rng.choice([avsg.INDEX_HASH, avsg.INDEX_DIRECT]))
+    _parity(w, mode=mode, index_mode=index_mode, host_io=bool(rng.random() < 0.3),
+            xfer_geometry=(int(rng.choice([1, 37, 148, 300])), int(rng.choice([32, 128, 256, 1024]))))
