@@ -46,7 +46,7 @@ struct avsg_ctx {
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
     // avsg_step_host: the outputs go back on a side stream while Stage Two runs
     cudaStream_t side = nullptr;
-    cudaEvent_t ev_outputs_ready = nullptr, ev_outputs_copied = nullptr;
+    cudaEvent_t ev_outputs_ready = nullptr, ev_outputs_copied = nullptr, ev_ids_ready = nullptr;
     uint64_t last_rows = 0;
 };
 
@@ -79,6 +79,7 @@ void free_all(avsg_ctx* c)
     for (auto& e : c->ev) if (e) cudaEventDestroy(e);
     if (c->ev_outputs_ready) cudaEventDestroy(c->ev_outputs_ready);
     if (c->ev_outputs_copied) cudaEventDestroy(c->ev_outputs_copied);
+    if (c->ev_ids_ready) cudaEventDestroy(c->ev_ids_ready);
     if (c->side) cudaStreamDestroy(c->side);
 }
 
@@ -177,7 +178,12 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
     uint8_t* hit = a->hit;
     int32_t* miss_count = a->miss_count;
     if (host_io) {
-        CU(cudaMemcpyAsync(c->d_idx_stage, a->indices, n_ids * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+        // The ids go up on the side stream, where they queue behind the previous call's output download (and
+        // therefore behind its Stage One, the last reader of the staging buffer) but not behind its Stage Two:
+        // when calls are issued back to back the upload hides under the previous call's gather.
+        CU(cudaMemcpyAsync(c->d_idx_stage, a->indices, n_ids * sizeof(int32_t), cudaMemcpyHostToDevice, c->side));
+        CU(cudaEventRecord(c->ev_ids_ready, c->side));
+        CU(cudaStreamWaitEvent(stream, c->ev_ids_ready, 0));
         indices = c->d_idx_stage;
         slots = c->d_slots_stage;
         hit = a->hit ? c->d_hit_stage : nullptr;
@@ -336,6 +342,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_ready, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_copied, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_ids_ready, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { cudaGetLastError(); free_all(c); delete c; return AVSG_ENOMEM; }
     if ((c->d_where && cudaMemset(c->d_where, 0xFF, T * (size_t)cfg->max_context * sizeof(uint16_t)) != cudaSuccess) ||
         cudaMemset(c->d_status, 0, 256) != cudaSuccess || cudaMemset(c->d_seg, 0, T * sizeof(SegDesc)) != cudaSuccess ||
