@@ -421,7 +421,8 @@ def _suite_one(avsg, torch, tr, name, mode, mode_name, link_peak, needed_rows=No
         tr.fill_kv(buf.data_ptr(), w.seed, ti, cfg.context, w.row_bytes)
         kv.append(buf)
     ctx = avsg.Context(num_tables=w.num_tables, buffer_slots=w.buffer_slots, row_bytes=w.row_bytes,
-                       max_topk=w.topk, max_tokens=w.n_q, max_lifetime=w.max_lifetime, transfer_mode=mode)
+                       max_topk=w.topk, max_tokens=w.n_q, max_lifetime=w.max_lifetime, transfer_mode=mode,
+                       index_mode=avsg.INDEX_DIRECT, max_context=max(c.context for c in w.tables) + w.n_q)
     ctx.set_timing(True)
     calls = [ctx.prepare(grp, [kv[t] for t in grp], w.n_q, w.topk) for grp in w.calls]
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
