@@ -266,6 +266,7 @@ def run_cuda(args):
         device_step(t)
     torch.cuda.synchronize()
     st0 = ctx.stats()
+    ts0 = [ctx.table_stats(ti) for ti in range(w.num_tables)]
     ctx.save_state()
     torch.cuda.synchronize()
     if world > 1:
@@ -287,6 +288,14 @@ def run_cuda(args):
     st1 = ctx.stats()
     rows_timed = st1["rows_copied"] - st0["rows_copied"]
     hits_timed, miss_timed = st1["hits"] - st0["hits"], st1["misses"] - st0["misses"]
+    # request-level (macro) hit rate: one rate per request over its layers' tables, then the mean over requests
+    ts1 = [ctx.table_stats(ti) for ti in range(w.num_tables)]
+    req_rates = []
+    for r in range(len(w.calls[0])):
+        tabs = [grp[r] for grp in w.calls]
+        h = sum(ts1[ti]["hits"] - ts0[ti]["hits"] for ti in tabs)
+        m = sum(ts1[ti]["misses"] - ts0[ti]["misses"] for ti in tabs)
+        req_rates.append(h / max(1, h + m))
     total_ms = sum(step_ms)
 
     # ---- end to end: ids from pinned host memory, slot table back to pinned host memory ----
@@ -332,7 +341,8 @@ def run_cuda(args):
     # ---- aggregate over ranks: device time = max over ranks, work = sum over ranks ----
     from paper_2609_37538_b200.sharding import aggregate
     tmax, tsum = aggregate({"total_ms": total_ms, "e2e_ms": e2e_ms, "xus": sum(x_us)},
-                           {"rows": rows_timed, "xrows": sum(x_rows), "hits": hits_timed, "misses": miss_timed})
+                           {"rows": rows_timed, "xrows": sum(x_rows), "hits": hits_timed, "misses": miss_timed,
+                            "req_rate_sum": sum(req_rates), "req_n": len(req_rates)})
     total_ms_j, e2e_ms_j, xus_j = tmax["total_ms"], tmax["e2e_ms"], tmax["xus"]
     rows_j, xrows_j, hits_j, miss_j = tsum["rows"], tsum["xrows"], tsum["hits"], tsum["misses"]
 
@@ -369,6 +379,7 @@ def run_cuda(args):
                         "downloaded; h2d bytes = ids + missed KV rows"},
         "gpu_launches": 2 * ncalls * K,
         "hit_rate": hits_j / max(1.0, hits_j + miss_j),
+        "hit_rate_request_macro": tsum["req_rate_sum"] / max(1.0, tsum["req_n"]),
         "miss_rows_per_step": rows_j / K / world,
         "link_peak_gbs": link_peak, "link": "PCIe Gen5 x16 (nominal 63 GB/s per direction); peak = best 1 GiB pinned cudaMemcpyAsync H2D in this run",
         "pct_of_link_peak": 100.0 * x_gbs / link_peak,
@@ -396,11 +407,16 @@ def run_cuda(args):
         cb_steps = min(16, K)
         tables = list(range(w.num_tables))
         secs, rows, _, _ = oracle_run(w, traces, kv_np, tables, W, cb_steps, cores, stride)
+        one_tables = tables[:8]
+        secs1, rows1, _, _ = oracle_run(w, traces, kv_np, one_tables, W, 4, 1, stride)
         line["cpu_baseline"] = {
             "value": sum(rows) * rb / 1e9 / sum(secs), "unit": "GB/s", "cores": cores, "kind": "oracle",
             "ms_per_step": 1e3 * sum(secs) / len(secs),
             "sample": "all %d tables, %d iterations after %d warm-up, one thread per table over %d threads"
-                      % (w.num_tables, cb_steps, W, cores)}
+                      % (w.num_tables, cb_steps, W, cores),
+            "single_thread": {"value": sum(rows1) * rb / 1e9 / sum(secs1), "unit": "GB/s",
+                              "ms_per_table_iteration": 1e3 * sum(secs1) / len(secs1) / len(one_tables),
+                              "sample": "%d tables, 4 iterations after %d warm-up, one thread" % (len(one_tables), W)}}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

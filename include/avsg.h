@@ -148,6 +148,11 @@ int avsg_buffer(avsg_ctx *ctx, uint32_t table_id, void **d_rows);
  * AVSG_EDEVICE_STATUS (and still fills *out) if a kernel flagged a problem. */
 int avsg_stats(avsg_ctx *ctx, avsg_stats_t *out);
 
+/* The same counters for ONE table (the last_* fields stay zero): what the
+ * request-level hit rates of Sec. 4.4 / App. E are averaged from.  Waits for
+ * the device. */
+int avsg_table_stats(avsg_ctx *ctx, uint32_t table_id, avsg_stats_t *out);
+
 /* Waits for the device; returns AVSG_EDEVICE_STATUS if a kernel flagged a
  * problem, and the raw status word in *status_word when not NULL. */
 int avsg_sync_status(avsg_ctx *ctx, uint32_t *status_word);

@@ -20,7 +20,7 @@ XFER_SM_BALANCED, XFER_COPY_ENGINE, XFER_REQUEST_LEVEL, XFER_ALL_K, XFER_POSITIO
 INDEX_HASH, INDEX_DIRECT, INDEX_PAPER = 0, 1, 2
 
 EXPORTS = (
-    "avsg_create", "avsg_destroy", "avsg_reset", "avsg_step", "avsg_step_host", "avsg_buffer", "avsg_stats",
+    "avsg_create", "avsg_destroy", "avsg_reset", "avsg_step", "avsg_step_host", "avsg_buffer", "avsg_stats", "avsg_table_stats",
     "avsg_sync_status", "avsg_export_state", "avsg_import_state", "avsg_save_state", "avsg_restore_state",
     "avsg_set_transfer_mode", "avsg_set_timing", "avsg_set_transfer_geometry", "avsg_strerror",
     "avsg_step_noalloc", "avsg_export_hash_state", "avsg_import_hash_state",
@@ -87,6 +87,7 @@ def load_library():
     lib.avsg_step_host.argtypes, lib.avsg_step_host.restype = [vp, ctypes.POINTER(AvsgStepArgs), vp], i32
     lib.avsg_buffer.argtypes, lib.avsg_buffer.restype = [vp, u32, ctypes.POINTER(vp)], i32
     lib.avsg_stats.argtypes, lib.avsg_stats.restype = [vp, ctypes.POINTER(AvsgStats)], i32
+    lib.avsg_table_stats.argtypes, lib.avsg_table_stats.restype = [vp, u32, ctypes.POINTER(AvsgStats)], i32
     lib.avsg_sync_status.argtypes, lib.avsg_sync_status.restype = [vp, ctypes.POINTER(u32)], i32
     lib.avsg_export_state.argtypes, lib.avsg_export_state.restype = [vp, u32, vp, vp], i32
     lib.avsg_import_state.argtypes, lib.avsg_import_state.restype = [vp, u32, vp, vp], i32
@@ -308,6 +309,12 @@ class Context:
         s = AvsgStats()
         _check(self._lib.avsg_stats(self._h, ctypes.byref(s)), "avsg_stats")
         return {name: getattr(s, name) for name, _ in AvsgStats._fields_}
+
+    def table_stats(self, table_id: int) -> dict:
+        """Counters of one table (request-level hit rates are averaged from these)."""
+        s = AvsgStats()
+        _check(self._lib.avsg_table_stats(self._h, table_id, ctypes.byref(s)), "avsg_table_stats")
+        return {name: getattr(s, name) for name, _ in AvsgStats._fields_ if not name.startswith("last_")}
 
 
 def step_noalloc(tok, life, buffer, indices, kv, verified_len, *, max_lifetime: int = 16, slots, hit=None,

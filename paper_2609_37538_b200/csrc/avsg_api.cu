@@ -421,6 +421,21 @@ int avsg_stats(avsg_ctx* c, avsg_stats_t* out)
     return read_status(c, nullptr);
 }
 
+int avsg_table_stats(avsg_ctx* c, uint32_t table_id, avsg_stats_t* out)
+{
+    if (!c || !out || table_id >= c->cfg.num_tables) return AVSG_EINVAL;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return AVSG_ECUDA;
+    CU(cudaDeviceSynchronize());
+    TableStats t;
+    CU(cudaMemcpy(&t, c->d_stats + table_id, sizeof(t), cudaMemcpyDeviceToHost));
+    memset(out, 0, sizeof(*out));
+    out->steps = t.steps; out->tokens = t.tokens; out->hits = t.hits; out->misses = t.misses;
+    out->rows_copied = t.rows; out->extra_decays = t.extra_decays;
+    out->bytes_copied = out->rows_copied * c->cfg.row_bytes;
+    return read_status(c, nullptr);
+}
+
 int avsg_sync_status(avsg_ctx* c, uint32_t* status_word)
 {
     if (!c) return AVSG_EINVAL;

@@ -299,9 +299,10 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
     int32_t xs[MAX_IPT];
     load_ids(p.indices + (size_t)ti * p.n_q * K, i0, ipt, K, xs);
 
-    if (!DIRECT)
+    if constexpr (!DIRECT) {
         for (uint32_t i = tid; i < H / 4; i += nt)
             reinterpret_cast<int4*>(s_key)[i] = make_int4(EMPTY, EMPTY, EMPTY, EMPTY);
+    }
     if (s_priv)
         for (uint32_t i = tid; i < ((uint32_t)(L + 2) * priv_stride + 15u) / 16u; i += nt)
             reinterpret_cast<int4*>(s_priv)[i] = make_int4(0, 0, 0, 0);
@@ -454,7 +455,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
         if (!rebuild) {
             fill_bound += n_g;
             __syncthreads();
-        } else {
+        } else if constexpr (!DIRECT) {
             __syncthreads();
             for (uint32_t i = tid; i < H / 4; i += nt)
                 reinterpret_cast<int4*>(s_key)[i] = make_int4(EMPTY, EMPTY, EMPTY, EMPTY);

@@ -104,6 +104,11 @@ def run_parity(w: tr.Workload, *, tables: Optional[Sequence[int]] = None, mode: 
         st = ctx.stats()
         oc = {k: sum(o.counters()[k] for o in orc.values()) for k in
               ("steps", "tokens", "hits", "misses", "rows_copied", "extra_decays")}
+        if not all_k:
+            for ti, o in orc.items():                                   # per-table counters (request-level rates)
+                ts, c = ctx.table_stats(local[ti]), o.counters()
+                for k in oc:
+                    assert ts[k] == c[k], ("table counters", w.name, ti, k, ts[k], c[k])
         if check == set(ids):
             if all_k:
                 assert st["rows_copied"] == oc["rows_copied"]
