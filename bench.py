@@ -321,13 +321,14 @@ def run_cuda(args):
     ctx.set_timing(True)
     torch.cuda.synchronize()
     ctx.stats()
-    s1_us, x_us, x_rows = [], [], []
+    s1_us, x_us, x_rows, s1_kus, x_kus = [], [], [], [], []
     for k in range(K):
         for c in range(ncalls):
             flush.fill_(c)
             calls[c].run(Xd[W + k][c], vlen[W + k][c], slots_d[c], None, mc_d[c], stream)
             s = ctx.stats()
             s1_us.append(s["last_stage_one_us"]); x_us.append(s["last_transfer_us"]); x_rows.append(s["last_rows"])
+            s1_kus.append(s["last_stage_one_kernel_us"]); x_kus.append(s["last_transfer_kernel_us"])
     # ---- replay of one recorded steady-state call, 1000 times (L2-warm), the paper's Stage One protocol ----
     rep = []
     ctx.save_state()
@@ -386,10 +387,15 @@ def run_cuda(args):
         "match_reserve_us": {"per_call_mean": s1_avg_us, "per_call_median": statistics.median(s1_us),
                              "per_call_min": min(s1_us), "per_call_max": max(s1_us),
                              "replay_median": statistics.median(rep) if rep else None, "replays": len(rep),
+                             "in_kernel_mean": sum(s1_kus) / len(s1_kus),
                              "tables_per_call": n_tab,
                              "note": "per_call_*: L2 flushed before each call; replay_*: one recorded call re-run from a restored state (L2-warm)"},
         "transfer_us": {"per_call_mean": x_avg_us, "per_call_median": statistics.median(x_us),
-                        "rows_per_call_mean": sum(x_rows) / n_launch},
+                        "in_kernel_mean": sum(x_kus) / len(x_kus),
+                        "in_kernel_gbs": x_bytes_per_launch / 1e3 / (sum(x_kus) / len(x_kus)),
+                        "rows_per_call_mean": sum(x_rows) / n_launch,
+                        "note": "per_call_*: CUDA events around the launch (what the roofline uses); in_kernel_*: first "
+                                "block's start to last block's end on the GPU's clock, without the launch gap"},
         "roofline": {"bound": "host_link", "kernel": "avsg_transfer_kernel", "achieved": x_gbs, "peak": link_peak,
                      "unit": "GB/s", "frac": x_gbs / link_peak,
                      "traffic": NCU_XFER_DRAM_BYTES_PER_ROW * sum(x_rows) / n_launch,

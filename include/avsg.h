@@ -118,6 +118,11 @@ typedef struct {
                                   and of its transfer; 0 unless timing is enabled        */
     float    last_transfer_us;
     uint64_t last_rows;        /* rows the last call moved                               */
+    float    last_stage_one_kernel_us; /* the same two grids timed from inside: first block's
+                                  start to last block's end on the GPU's own clock, i.e.
+                                  without the launch gap an event pair includes; 0 unless
+                                  timing is enabled                                       */
+    float    last_transfer_kernel_us;
 } avsg_stats_t;
 
 /* Allocates all state: tables empty and dead ("each request starts with an

@@ -46,7 +46,8 @@ class AvsgStats(ctypes.Structure):
     _fields_ = [("steps", ctypes.c_uint64), ("tokens", ctypes.c_uint64), ("hits", ctypes.c_uint64),
                 ("misses", ctypes.c_uint64), ("rows_copied", ctypes.c_uint64), ("bytes_copied", ctypes.c_uint64),
                 ("extra_decays", ctypes.c_uint64), ("last_stage_one_us", ctypes.c_float),
-                ("last_transfer_us", ctypes.c_float), ("last_rows", ctypes.c_uint64)]
+                ("last_transfer_us", ctypes.c_float), ("last_rows", ctypes.c_uint64),
+                ("last_stage_one_kernel_us", ctypes.c_float), ("last_transfer_kernel_us", ctypes.c_float)]
 
 
 class AvsgNoAllocArgs(ctypes.Structure):

@@ -22,6 +22,8 @@ struct avsg_ctx {
     int8_t* d_life = nullptr;
     uint8_t* d_buffer = nullptr;
     TableStats* d_stats = nullptr;
+    unsigned long long* d_trange = nullptr;        // [4] grid spans of the last timed call, then [4] their initial values
+    unsigned long long* d_trange_init = nullptr;
     int2* d_list = nullptr;
     SegDesc* d_seg = nullptr;
     uint32_t* d_status = nullptr;
@@ -70,7 +72,7 @@ uint32_t ilog2(uint32_t v) { uint32_t l = 0; while ((1u << l) < v) ++l; return l
 
 void free_all(avsg_ctx* c)
 {
-    cudaFree(c->d_tok); cudaFree(c->d_life); cudaFree(c->d_buffer); cudaFree(c->d_stats);
+    cudaFree(c->d_tok); cudaFree(c->d_life); cudaFree(c->d_buffer); cudaFree(c->d_stats); cudaFree(c->d_trange);
     cudaFree(c->d_list); cudaFree(c->d_seg); cudaFree(c->d_status); cudaFree(c->d_where); cudaFree(c->d_q); cudaFree(c->d_q_snap);
     cudaFree(c->d_tok_snap); cudaFree(c->d_life_snap);
     cudaFree(c->d_idx_stage); cudaFree(c->d_slots_stage); cudaFree(c->d_hit_stage); cudaFree(c->d_mc_stage);
@@ -192,7 +194,11 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
     const uint32_t mode = c->cfg.transfer_mode;
     // the position-level comparator reads the hit mask: use the library's own buffer if the caller wants none
     if (mode == AVSG_XFER_POSITION_LEVEL && !hit) hit = c->d_hit_stage;
-    if (c->timing) CU(cudaEventRecord(c->ev[0], stream));
+    if (c->timing) {
+        // grid spans: [0] Stage One first start, [1] its last end, [2], [3] the same for Stage Two
+        CU(cudaMemcpyAsync(c->d_trange, c->d_trange_init, 4 * sizeof(unsigned long long), cudaMemcpyDeviceToDevice, stream));
+        CU(cudaEventRecord(c->ev[0], stream));
+    }
 
     c->call_kv_host.assign(a->kv_base, a->kv_base + n);
     for (uint32_t first = 0; first < n; first += S1_MAX_TABLES) {
@@ -219,6 +225,7 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
             p.first = first; p.list_stride = c->list_stride;
             p.where = c->d_where; p.max_context = c->cfg.max_context;
             p.qword = c->d_q; p.probe_retries = c->cfg.probe_retries; p.hash_a1 = c->cfg.hash_a1; p.hash_a2 = c->cfg.hash_a2;
+            p.t_range = c->timing ? c->d_trange : nullptr;
             for (uint32_t i = 0; i < cnt; ++i) {
                 p.table_id[i] = a->table_ids[first + i];
                 p.verified_len[i] = a->verified_len[first + i];
@@ -254,6 +261,7 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
         x.n_seg = n; x.list_stride = c->list_stride; x.row_bytes = c->cfg.row_bytes;
         x.request_level = mode == AVSG_XFER_REQUEST_LEVEL; x.S = c->cfg.buffer_slots;
+        x.t_range = c->timing ? c->d_trange + 2 : nullptr;
         const uint32_t blocks = x.request_level ? n : (c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count);
         CU(launch_transfer(x, blocks, c->xfer_threads, stream));
     }
@@ -321,6 +329,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaMalloc(&c->d_life, T * S) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_buffer, T * S * cfg->row_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_stats, T * sizeof(TableStats)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_trange, 8 * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_list, n_ids * sizeof(int2)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_seg, T * sizeof(SegDesc)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_status, 256) == cudaSuccess;
@@ -344,6 +353,13 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_copied, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_ids_ready, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { cudaGetLastError(); free_all(c); delete c; return AVSG_ENOMEM; }
+    {
+        const unsigned long long never = ~0ull, init[8] = {never, 0, never, 0, never, 0, never, 0};
+        c->d_trange_init = c->d_trange + 4;
+        if (cudaMemcpy(c->d_trange, init, sizeof(init), cudaMemcpyHostToDevice) != cudaSuccess) {
+            free_all(c); delete c; return AVSG_ECUDA;
+        }
+    }
     if ((c->d_where && cudaMemset(c->d_where, 0xFF, T * (size_t)cfg->max_context * sizeof(uint16_t)) != cudaSuccess) ||
         cudaMemset(c->d_status, 0, 256) != cudaSuccess || cudaMemset(c->d_seg, 0, T * sizeof(SegDesc)) != cudaSuccess ||
         init_tables(c, 0, (uint32_t)T) != AVSG_OK || cudaDeviceSynchronize() != cudaSuccess) {
@@ -415,6 +431,10 @@ int avsg_stats(avsg_ctx* c, avsg_stats_t* out)
         if (cudaEventElapsedTime(&a, c->ev[0], c->ev[1]) == cudaSuccess) out->last_stage_one_us = a * 1000.f;
         if (cudaEventElapsedTime(&b, c->ev[1], c->ev[2]) == cudaSuccess) out->last_transfer_us = b * 1000.f;
         cudaGetLastError();
+        unsigned long long r[4];
+        CU(cudaMemcpy(r, c->d_trange, sizeof(r), cudaMemcpyDeviceToHost));
+        if (r[1] > r[0]) out->last_stage_one_kernel_us = (float)(r[1] - r[0]) * 1e-3f;
+        if (r[3] > r[2]) out->last_transfer_kernel_us = (float)(r[3] - r[2]) * 1e-3f;
     }
     out->last_rows = out->rows_copied - c->last_rows;
     c->last_rows = out->rows_copied;

@@ -25,6 +25,14 @@ struct SegDesc {
     uint32_t pad;
 };
 
+// Wall-clock span of a grid for avsg_set_timing: every block reports its start and end (globaltimer, ns).
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
 struct TableStats {
     unsigned long long steps, tokens, hits, misses, rows, extra_decays;
 };
@@ -53,6 +61,7 @@ struct S1Params {
     uint16_t* where;             // direct index [num_tables][max_context], or null for the hash index
     uint32_t* qword;             // paper-literal mode: packed metadata words [num_tables][S], else null
     uint32_t probe_retries, hash_a1, hash_a2;   // paper-literal mode: R, a1, a2
+    unsigned long long* t_range = nullptr;      // timing on: [0] earliest block start, [1] latest block end (ns)
     uint32_t table_id[S1_MAX_TABLES];
     int32_t  verified_len[S1_MAX_TABLES];
     uint64_t kv_base[S1_MAX_TABLES];
@@ -64,6 +73,7 @@ struct XferParams {
     const int2*    miss_list;
     uint32_t*      status;
     uint32_t n_seg, list_stride, row_bytes, request_level, S;
+    unsigned long long* t_range = nullptr;      // timing on: [0] earliest block start, [1] latest block end (ns)
 };
 
 struct PosParams {               // comparator S2: equal top-K position partition

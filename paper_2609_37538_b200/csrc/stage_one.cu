@@ -279,6 +279,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
     // allowed to start its own prologue right away - it waits the same way before it reads the miss list.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (p.t_range && threadIdx.x == 0) atomicMin(p.t_range, global_ns());
 
     // ---- issue every global load first: table state and the first token's ids ----
     int4 t4[MAX_SPT / 4];
@@ -503,6 +504,10 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
         st->rows += list_off;
         st->extra_decays += sum_decay;
     }
+    if (p.t_range) {
+        __syncthreads();
+        if (tid == 0) atomicMax(p.t_range + 1, global_ns());
+    }
 }
 
 // Direct index: points every resident id at its slot again, after the table state was replaced from outside
@@ -584,6 +589,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_paper_kernel(const __g
 
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (p.t_range && threadIdx.x == 0) atomicMin(p.t_range, global_ns());
 
     // ---- load the table; global pre-decay ----
     if (own)
@@ -768,6 +774,10 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_paper_kernel(const __g
         st->misses += sum_miss;
         st->rows += list_off;
         st->extra_decays += sum_decay;
+    }
+    if (p.t_range) {
+        __syncthreads();
+        if (tid == 0) atomicMax(p.t_range + 1, global_ns());
     }
 }
 

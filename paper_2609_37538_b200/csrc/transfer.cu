@@ -59,6 +59,7 @@ __global__ void __launch_bounds__(1024) avsg_transfer_kernel(const __grid_consta
     // list is read only after that grid has completed.  The kernel after this one may start its prologue.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (p.t_range && tid == 0) atomicMin(p.t_range, global_ns());
 
     // global miss prefix sum (every block computes the same one)
     uint32_t running = 0;
@@ -117,6 +118,10 @@ __global__ void __launch_bounds__(1024) avsg_transfer_kernel(const __grid_consta
                 if (c < cpr) *reinterpret_cast<int4*>(dst + 16ull * c) = v[k];
             }
         }
+    }
+    if (p.t_range) {
+        __syncthreads();
+        if (tid == 0) atomicMax(p.t_range + 1, global_ns());
     }
 }
 

@@ -204,8 +204,15 @@ def test_timing_and_stats(avsg):
         ctx.step([0], torch.from_numpy(X[t][None]).cuda(), [kv], [int(N[t])])
     st = ctx.stats()
     assert st["last_stage_one_us"] > 0 and st["last_transfer_us"] > 0
+    # the grids timed from inside (first block start to last block end) fit inside the event pairs around them
+    assert 0 < st["last_stage_one_kernel_us"] <= st["last_stage_one_us"] + 1.0
+    assert 0 < st["last_transfer_kernel_us"] <= st["last_transfer_us"] + 1.0
     assert st["steps"] == 4 and st["tokens"] == 8 and st["hits"] + st["misses"] == 8 * 512
     assert st["bytes_copied"] == st["rows_copied"] * w.row_bytes == st["misses"] * w.row_bytes
+    ctx.set_timing(False)
+    ctx.step([0], torch.from_numpy(X[3][None]).cuda(), [kv], [int(N[3])])
+    st = ctx.stats()
+    assert st["last_stage_one_us"] == 0 and st["last_transfer_kernel_us"] == 0 and st["last_stage_one_kernel_us"] == 0
 
 
 def test_argument_errors(avsg):
