@@ -230,7 +230,8 @@ def run_cuda(args):
     ctx = avsg.Context(num_tables=w.num_tables, buffer_slots=w.buffer_slots, row_bytes=w.row_bytes,
                        max_topk=w.topk, max_tokens=w.n_q, max_lifetime=w.max_lifetime, device=local,
                        index_mode=avsg.INDEX_DIRECT if direct else avsg.INDEX_HASH,
-                       max_context=max(c.context for c in w.tables) + w.n_q)
+                       max_context=max(c.context for c in w.tables) + w.n_q,
+                       transfer_mode=avsg.XFER_SM_OVERLAP if args.stage_two == "overlap" else avsg.XFER_SM_BALANCED)
     ncalls = len(w.calls)
     calls = [ctx.prepare(grp, [kv[t] for t in grp], w.n_q, w.topk,
                          [stride] * len(grp) if args.row_stride else None) for grp in w.calls]
@@ -318,6 +319,7 @@ def run_cuda(args):
 
     # ---- per-kernel times (events inside the library around Stage One / Stage Two), L2 flushed per call ----
     ctx.restore_state()
+    ctx.set_transfer_mode(avsg.XFER_SM_BALANCED)      # events between the kernels: one kernel at a time
     ctx.set_timing(True)
     torch.cuda.synchronize()
     ctx.stats()
@@ -371,7 +373,7 @@ def run_cuda(args):
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms_j / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int32/u8", "data": "synthetic", "config": dict(_config(w), host_row_stride=stride, stage_one_index=args.index),
+        "dtype": "int32/u8", "data": "synthetic", "config": dict(_config(w), host_row_stride=stride, stage_one_index=args.index, stage_two=args.stage_two),
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "GB/s",
                 "h2d_bytes_per_step": int(ids_bytes + rows_timed * rb / K), "d2h_bytes_per_step": int(ids_bytes + mc_bytes),
@@ -690,6 +692,9 @@ def main():
     ap.add_argument("--layers", type=int, default=4, help="layers (4 = the full configuration)")
     ap.add_argument("--index", default="direct", choices=["hash", "direct"],
                     help="Stage One index: direct-address table in device memory (default) or shared-memory hash table")
+    ap.add_argument("--stage-two", default="balanced", choices=["balanced", "overlap"],
+                    help="balanced: Stage Two starts when Stage One is complete; overlap: it starts on token g's misses "
+                         "while token g+1 is placed (the per-kernel figures are always taken in balanced mode)")
     ap.add_argument("--row-stride", type=int, default=0,
                     help="bytes between host KV rows (0 = packed, 656); e.g. 768 pads rows to 128-byte lines")
     ap.add_argument("--table3", action="store_true",

@@ -55,6 +55,14 @@ extern "C" {
                                        call are cut into equal ranges, one per thread
                                        block, which walks its range and copies the misses;
                                        hit positions are visited for nothing             */
+#define AVSG_XFER_SM_OVERLAP    5u  /* the operator with Stage Two overlapping Stage One
+                                       (App. G, latency hiding): the transfer kernel is
+                                       resident while Stage One runs and starts on token
+                                       g's misses, cut evenly over all SMs per token,
+                                       while token g+1 is being placed.  Same results.
+                                       Calls with more than 128 tables or more than 8
+                                       tokens, and AVSG_INDEX_PAPER contexts, run as
+                                       AVSG_XFER_SM_BALANCED                             */
 
 /* How Stage One finds the slot that holds an id (same results either way). */
 #define AVSG_INDEX_HASH   0u  /* open-addressing table in shared memory, rebuilt every step     */
@@ -115,7 +123,10 @@ typedef struct {
     uint64_t bytes_copied;     /* rows_copied * row_bytes                                */
     uint64_t extra_decays;     /* unit decays beyond the pre-decay (Alg. 1 while-loop)   */
     float    last_stage_one_us;/* device time of the last call's match+reserve kernels
-                                  and of its transfer; 0 unless timing is enabled        */
+                                  and of its transfer; 0 unless timing is enabled.  With
+                                  AVSG_XFER_SM_OVERLAP no event separates the two grids:
+                                  last_stage_one_us then covers the whole call and
+                                  last_transfer_us is ~0                                 */
     float    last_transfer_us;
     uint64_t last_rows;        /* rows the last call moved                               */
     float    last_stage_one_kernel_us; /* the same two grids timed from inside: first block's
@@ -123,6 +134,10 @@ typedef struct {
                                   without the launch gap an event pair includes; 0 unless
                                   timing is enabled                                       */
     float    last_transfer_kernel_us;
+    float    last_transfer_start_us;   /* first transfer block's start after the first Stage One
+                                  block's start, same clock: below last_stage_one_kernel_us
+                                  when AVSG_XFER_SM_OVERLAP overlaps the two                */
+    float    reserved;
 } avsg_stats_t;
 
 /* Allocates all state: tables empty and dead ("each request starts with an

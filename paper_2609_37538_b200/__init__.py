@@ -1,7 +1,7 @@
 """AVSG per-decode-step operator for B200 (sm_100a): C-ABI library + thin Python binding."""
 from .binding import (  # noqa: F401
     ECAPACITY, ECUDA, EDEVICE_STATUS, EINVAL, ENOMEM, EUNSUPPORTED, EXPORTS, OK, INDEX_DIRECT, INDEX_HASH, INDEX_PAPER,
-    XFER_ALL_K, XFER_COPY_ENGINE, XFER_POSITION_LEVEL, XFER_REQUEST_LEVEL, XFER_SM_BALANCED,
+    XFER_ALL_K, XFER_COPY_ENGINE, XFER_POSITION_LEVEL, XFER_REQUEST_LEVEL, XFER_SM_BALANCED, XFER_SM_OVERLAP,
     AvsgConfig, AvsgError, AvsgStats, AvsgStepArgs, Context, PreparedCall, StepOutput,
     load_library, pinned_empty,
     AvsgNoAllocArgs, NOALLOC_MAX_IDS, NOALLOC_MAX_TABLES, step_noalloc,

@@ -16,7 +16,7 @@ import numpy as np
 from . import build as _build
 
 OK, EINVAL, ENOMEM, ECUDA, ECAPACITY, EDEVICE_STATUS, EUNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
-XFER_SM_BALANCED, XFER_COPY_ENGINE, XFER_REQUEST_LEVEL, XFER_ALL_K, XFER_POSITION_LEVEL = 0, 1, 2, 3, 4
+XFER_SM_BALANCED, XFER_COPY_ENGINE, XFER_REQUEST_LEVEL, XFER_ALL_K, XFER_POSITION_LEVEL, XFER_SM_OVERLAP = 0, 1, 2, 3, 4, 5
 INDEX_HASH, INDEX_DIRECT, INDEX_PAPER = 0, 1, 2
 
 EXPORTS = (
@@ -47,7 +47,8 @@ class AvsgStats(ctypes.Structure):
                 ("misses", ctypes.c_uint64), ("rows_copied", ctypes.c_uint64), ("bytes_copied", ctypes.c_uint64),
                 ("extra_decays", ctypes.c_uint64), ("last_stage_one_us", ctypes.c_float),
                 ("last_transfer_us", ctypes.c_float), ("last_rows", ctypes.c_uint64),
-                ("last_stage_one_kernel_us", ctypes.c_float), ("last_transfer_kernel_us", ctypes.c_float)]
+                ("last_stage_one_kernel_us", ctypes.c_float), ("last_transfer_kernel_us", ctypes.c_float),
+                ("last_transfer_start_us", ctypes.c_float), ("reserved", ctypes.c_float)]
 
 
 class AvsgNoAllocArgs(ctypes.Structure):

@@ -22,6 +22,9 @@ struct avsg_ctx {
     int8_t* d_life = nullptr;
     uint8_t* d_buffer = nullptr;
     TableStats* d_stats = nullptr;
+    unsigned long long* d_ready = nullptr;         // overlapped Stage Two: per-token counters [OVERLAP_MAX_TOKENS]
+    uint32_t* d_tcount = nullptr;                  //   and per-(table of the call, token) miss counts
+    unsigned long long posted[OVERLAP_MAX_TOKENS] = {};   // value each counter has after the calls issued so far
     unsigned long long* d_trange = nullptr;        // [4] grid spans of the last timed call, then [4] their initial values
     unsigned long long* d_trange_init = nullptr;
     int2* d_list = nullptr;
@@ -73,6 +76,7 @@ uint32_t ilog2(uint32_t v) { uint32_t l = 0; while ((1u << l) < v) ++l; return l
 void free_all(avsg_ctx* c)
 {
     cudaFree(c->d_tok); cudaFree(c->d_life); cudaFree(c->d_buffer); cudaFree(c->d_stats); cudaFree(c->d_trange);
+    cudaFree(c->d_ready); cudaFree(c->d_tcount);
     cudaFree(c->d_list); cudaFree(c->d_seg); cudaFree(c->d_status); cudaFree(c->d_where); cudaFree(c->d_q); cudaFree(c->d_q_snap);
     cudaFree(c->d_tok_snap); cudaFree(c->d_life_snap);
     cudaFree(c->d_idx_stage); cudaFree(c->d_slots_stage); cudaFree(c->d_hit_stage); cudaFree(c->d_mc_stage);
@@ -191,7 +195,10 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         hit = a->hit ? c->d_hit_stage : nullptr;
         miss_count = a->miss_count ? c->d_mc_stage : nullptr;
     }
-    const uint32_t mode = c->cfg.transfer_mode;
+    uint32_t mode = c->cfg.transfer_mode;
+    if (mode == AVSG_XFER_SM_OVERLAP &&
+        (n > (uint32_t)S1_MAX_TABLES || n_q > (uint32_t)OVERLAP_MAX_TOKENS || c->cfg.index_mode == AVSG_INDEX_PAPER))
+        mode = AVSG_XFER_SM_BALANCED;
     // the position-level comparator reads the hit mask: use the library's own buffer if the caller wants none
     if (mode == AVSG_XFER_POSITION_LEVEL && !hit) hit = c->d_hit_stage;
     if (c->timing) {
@@ -226,6 +233,7 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
             p.where = c->d_where; p.max_context = c->cfg.max_context;
             p.qword = c->d_q; p.probe_retries = c->cfg.probe_retries; p.hash_a1 = c->cfg.hash_a1; p.hash_a2 = c->cfg.hash_a2;
             p.t_range = c->timing ? c->d_trange : nullptr;
+            if (mode == AVSG_XFER_SM_OVERLAP) { p.ready = c->d_ready; p.tcount = c->d_tcount; }
             for (uint32_t i = 0; i < cnt; ++i) {
                 p.table_id[i] = a->table_ids[first + i];
                 p.verified_len[i] = a->verified_len[first + i];
@@ -235,7 +243,8 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
             CU(launch_stage_one(p, cnt, stream));
         }
     }
-    if (c->timing) CU(cudaEventRecord(c->ev[1], stream));
+    // (no event between the two grids in overlap mode: it would serialise them; ev[1] is recorded with ev[2])
+    if (c->timing && mode != AVSG_XFER_SM_OVERLAP) CU(cudaEventRecord(c->ev[1], stream));
 
     if (host_io) {
         // The slot table, hit mask and miss counts are final once Stage One has run.  They travel device -> host
@@ -256,6 +265,17 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         q.seg = c->d_seg; q.indices = indices; q.slots = slots; q.hit = hit; q.status = c->d_status;
         q.n = n; q.per_table = n_q * K; q.row_bytes = c->cfg.row_bytes; q.S = c->cfg.buffer_slots;
         CU(launch_transfer_positions(q, c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count, c->xfer_threads, stream));
+    } else if (mode == AVSG_XFER_SM_OVERLAP) {
+        XferOverlapParams x;
+        x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
+        x.tcount = c->d_tcount; x.ready = c->d_ready;
+        for (uint32_t g = 0; g < (uint32_t)OVERLAP_MAX_TOKENS; ++g) {
+            if (g < n_q) c->posted[g] += n;            // Stage One of this call (already launched) raises these
+            x.target[g] = c->posted[g];
+        }
+        x.n = n; x.n_q = n_q; x.list_stride = c->list_stride; x.row_bytes = c->cfg.row_bytes; x.S = c->cfg.buffer_slots;
+        x.t_range = c->timing ? c->d_trange + 2 : nullptr;
+        CU(launch_transfer_overlap(x, c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count, c->xfer_threads, stream));
     } else {
         XferParams x;
         x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
@@ -265,7 +285,11 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         const uint32_t blocks = x.request_level ? n : (c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count);
         CU(launch_transfer(x, blocks, c->xfer_threads, stream));
     }
-    if (c->timing) { CU(cudaEventRecord(c->ev[2], stream)); c->events_recorded = true; }
+    if (c->timing) {
+        if (mode == AVSG_XFER_SM_OVERLAP) CU(cudaEventRecord(c->ev[1], stream));
+        CU(cudaEventRecord(c->ev[2], stream));
+        c->events_recorded = true;
+    }
 
     if (host_io) CU(cudaStreamWaitEvent(stream, c->ev_outputs_copied, 0));     // the call ends when the outputs are home
     return AVSG_OK;
@@ -291,7 +315,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     if (cfg->row_bytes == 0 || cfg->row_bytes % 16) return AVSG_EINVAL;
     if (cfg->max_topk == 0 || cfg->max_tokens == 0) return AVSG_EINVAL;
     if (cfg->max_lifetime < 1 || cfg->max_lifetime > 126) return AVSG_EINVAL;
-    if (cfg->transfer_mode > AVSG_XFER_POSITION_LEVEL || cfg->index_mode > AVSG_INDEX_PAPER) return AVSG_EINVAL;
+    if (cfg->transfer_mode > AVSG_XFER_SM_OVERLAP || cfg->index_mode > AVSG_INDEX_PAPER) return AVSG_EINVAL;
     if (cfg->index_mode == AVSG_INDEX_DIRECT && cfg->max_context == 0) return AVSG_EINVAL;
     if ((uint64_t)cfg->max_topk * cfg->max_tokens > cfg->buffer_slots) return AVSG_ECAPACITY;   // Eq. 7
     int ndev = 0;
@@ -330,6 +354,8 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaMalloc(&c->d_buffer, T * S * cfg->row_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_stats, T * sizeof(TableStats)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_trange, 8 * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_ready, OVERLAP_MAX_TOKENS * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_tcount, (size_t)S1_MAX_TABLES * OVERLAP_MAX_TOKENS * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_list, n_ids * sizeof(int2)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_seg, T * sizeof(SegDesc)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_status, 256) == cudaSuccess;
@@ -356,7 +382,8 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     {
         const unsigned long long never = ~0ull, init[8] = {never, 0, never, 0, never, 0, never, 0};
         c->d_trange_init = c->d_trange + 4;
-        if (cudaMemcpy(c->d_trange, init, sizeof(init), cudaMemcpyHostToDevice) != cudaSuccess) {
+        if (cudaMemcpy(c->d_trange, init, sizeof(init), cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemset(c->d_ready, 0, OVERLAP_MAX_TOKENS * sizeof(unsigned long long)) != cudaSuccess) {
             free_all(c); delete c; return AVSG_ECUDA;
         }
     }
@@ -435,6 +462,7 @@ int avsg_stats(avsg_ctx* c, avsg_stats_t* out)
         CU(cudaMemcpy(r, c->d_trange, sizeof(r), cudaMemcpyDeviceToHost));
         if (r[1] > r[0]) out->last_stage_one_kernel_us = (float)(r[1] - r[0]) * 1e-3f;
         if (r[3] > r[2]) out->last_transfer_kernel_us = (float)(r[3] - r[2]) * 1e-3f;
+        if (r[3] > r[2] && r[1] > r[0] && r[2] >= r[0]) out->last_transfer_start_us = (float)(r[2] - r[0]) * 1e-3f;
     }
     out->last_rows = out->rows_copied - c->last_rows;
     c->last_rows = out->rows_copied;
@@ -561,7 +589,7 @@ int avsg_restore_state(avsg_ctx* c, void* stream)
 
 int avsg_set_transfer_mode(avsg_ctx* c, uint32_t mode)
 {
-    if (!c || mode > AVSG_XFER_POSITION_LEVEL) return AVSG_EINVAL;
+    if (!c || mode > AVSG_XFER_SM_OVERLAP) return AVSG_EINVAL;
     c->cfg.transfer_mode = mode;
     return AVSG_OK;
 }

@@ -13,6 +13,7 @@ enum : uint32_t {
     ST_BAD_SLOT        = 1u << 2,   // slot / position index out of range
     ST_BAD_SEGMENT     = 1u << 3,   // transfer kernel could not resolve a miss
     ST_BAD_ID          = 1u << 4,   // direct index: an id beyond max_context (treated as padding)
+    ST_WAIT_TIMEOUT    = 1u << 5,   // overlapped Stage Two: a bounded wait for Stage One ran out
 };
 
 // One segment of the step's miss list = the misses of one table, in token
@@ -62,6 +63,10 @@ struct S1Params {
     uint32_t* qword;             // paper-literal mode: packed metadata words [num_tables][S], else null
     uint32_t probe_retries, hash_a1, hash_a2;   // paper-literal mode: R, a1, a2
     unsigned long long* t_range = nullptr;      // timing on: [0] earliest block start, [1] latest block end (ns)
+    // overlapped Stage Two (null otherwise): ready[g] counts the tables whose token g is placed, over all calls;
+    // tcount[ti * n_q + g] = misses of token g of the ti-th table of the call
+    unsigned long long* ready = nullptr;
+    uint32_t*           tcount = nullptr;
     uint32_t table_id[S1_MAX_TABLES];
     int32_t  verified_len[S1_MAX_TABLES];
     uint64_t kv_base[S1_MAX_TABLES];
@@ -74,6 +79,20 @@ struct XferParams {
     uint32_t*      status;
     uint32_t n_seg, list_stride, row_bytes, request_level, S;
     unsigned long long* t_range = nullptr;      // timing on: [0] earliest block start, [1] latest block end (ns)
+};
+
+constexpr int OVERLAP_MAX_TOKENS = 8;
+constexpr uint32_t OVERLAP_SPIN_LIMIT = 1u << 18;   // polls of >= 64 ns each before the wait gives up (~17 ms)
+
+struct XferOverlapParams {       // Stage Two that starts on token g's misses while Stage One places token g+1
+    const SegDesc* seg;          // bases written by Stage One before it publishes token 0
+    const int2*    miss_list;
+    uint32_t*      status;
+    const uint32_t* tcount;      // [n][n_q]
+    const unsigned long long* ready;             // [OVERLAP_MAX_TOKENS]
+    unsigned long long target[OVERLAP_MAX_TOKENS];   // value of ready[g] once every table of this call has token g placed
+    uint32_t n, n_q, list_stride, row_bytes, S;
+    unsigned long long* t_range = nullptr;
 };
 
 struct PosParams {               // comparator S2: equal top-K position partition
@@ -109,6 +128,7 @@ cudaError_t launch_direct_index_from_state(const int32_t* tok, uint16_t* where, 
                                            uint32_t S, uint32_t max_context, cudaStream_t stream);
 cudaError_t launch_all_k_prepare(const AllKParams& p, uint32_t n_tables, cudaStream_t stream);
 cudaError_t launch_transfer(const XferParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream);
+cudaError_t launch_transfer_overlap(const XferOverlapParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream);
 cudaError_t launch_transfer_positions(const PosParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream);
 
 }  // namespace avsg

@@ -332,6 +332,31 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
     uint32_t list_off = 0, sum_valid = 0, sum_miss = 0, sum_decay = 0;
     int2* list = p.miss_list + (size_t)ti * p.list_stride;
 
+    // Overlapped Stage Two only (p.ready set): tells the transfer kernel, which is already resident, that token
+    // g of this table is placed - `count` more entries of the table's miss list are final.  The block meets
+    // after its list writes; one thread then fences (the barrier makes the fence cover the whole block's
+    // earlier writes, as in a grid-wide barrier) and raises the counter of token g.
+    auto publish = [&](uint32_t g, uint32_t count) {
+        if (!p.ready) return;
+        if (tid == 0) {
+            p.tcount[(size_t)ti * p.n_q + g] = count;
+            if (g == 0) {
+                SegDesc sd;
+                sd.src_base = p.kv_base[blockIdx.x];
+                sd.src_stride = p.kv_stride[blockIdx.x];
+                sd.dst_base = reinterpret_cast<uint64_t>(p.buffer + (size_t)table * S * p.row_bytes);
+                sd.count = 0;
+                sd.pad = 0;
+                p.seg[ti] = sd;
+            }
+        }
+        __syncthreads();
+        if (tid == 0) {
+            __threadfence();
+            atomicAdd(p.ready + g, 1ull);
+        }
+    };
+
     for (uint32_t g = 0; g < p.n_q; ++g) {
         const size_t row = ((size_t)ti * p.n_q + g) * K;
         int32_t* O = p.slots + row;
@@ -392,7 +417,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
         // the next token's ids travel while this token's misses are placed
         if (g + 1 < p.n_q) load_ids(p.indices + row + K, i0, ipt, K, xs);
         if (tid == 0 && p.miss_count) p.miss_count[(size_t)ti * p.n_q + g] = (int32_t)n_g;
-        if (n_g == 0) { __syncthreads(); continue; }
+        if (n_g == 0) { __syncthreads(); publish(g, 0); continue; }
         __syncthreads();
 
         // ---- Pass 3: CollectDead; if fewer than n_g slots are dead, decay until enough are ----
@@ -466,6 +491,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
             __syncthreads();
             fill_bound = *s_fill;
         }
+        publish(g, n_take);
     }
 
     // ---- write the table back; speculative entries (id >= N) become empty (Alg. 4) ----

@@ -47,7 +47,7 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* s_w, u
     return incl - v + s_w[warp];
 }
 
-__global__ void __launch_bounds__(1024) avsg_transfer_kernel(const __grid_constant__ XferParams p)
+__global__ void __launch_bounds__(1024, 1) avsg_transfer_kernel(const __grid_constant__ XferParams p)
 {
     __shared__ uint32_t s_pref[XFER_MAX_SEG + 1];
     __shared__ uint32_t s_w[40];
@@ -125,6 +125,114 @@ __global__ void __launch_bounds__(1024) avsg_transfer_kernel(const __grid_consta
     }
 }
 
+// Stage Two that overlaps Stage One (the latency-hiding direction of App. G).  The grid is launched with
+// programmatic stream serialization and does NOT wait for Stage One to complete: its blocks become resident
+// once every Stage One block has started, then wait - with a bound - until all tables of the call have
+// placed token g (Stage One raises ready[g] per table, after making that token's miss-list entries
+// visible), cut token g's misses evenly over the blocks (Eq. 6 per token) and copy them while Stage One
+// places token g+1.  Every Stage One block is resident before this grid starts, so it always makes progress
+// without this grid's help; if a wait still runs out the block sets ST_WAIT_TIMEOUT and stops copying.
+// Before leaving, every block waits for the completion of the Stage One grid, so that the completion of
+// this grid implies it.  All reads of data written by the running Stage One go to L2 (ld.cg / acquire).
+__global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __grid_constant__ XferOverlapParams p)
+{
+    __shared__ uint32_t s_pref[S1_MAX_TABLES + 1];
+    __shared__ uint32_t s_off[S1_MAX_TABLES];
+    __shared__ uint64_t s_src[S1_MAX_TABLES], s_stride[S1_MAX_TABLES], s_dst[S1_MAX_TABLES];
+    __shared__ uint32_t s_w[40];
+    __shared__ uint32_t s_ok;
+
+    const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31u;
+    const uint32_t n = p.n;
+
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (p.t_range && tid == 0) atomicMin(p.t_range, global_ns());
+    for (uint32_t i = tid; i < n; i += nt) s_off[i] = 0;
+    __syncthreads();
+
+    const uint32_t cpr = p.row_bytes >> 4;
+    for (uint32_t g = 0; g < p.n_q; ++g) {
+        if (tid == 0) {
+            uint32_t ok = 0;
+            for (uint32_t spin = 0; spin < OVERLAP_SPIN_LIMIT; ++spin) {
+                unsigned long long v;
+                asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p.ready + g) : "memory");
+                if (v >= p.target[g]) { ok = 1; break; }
+                __nanosleep(64);
+            }
+            if (!ok) atomicOr(p.status, ST_WAIT_TIMEOUT);
+            s_ok = ok;
+        }
+        __syncthreads();
+        if (!s_ok) break;                                          // same decision in every thread
+        if (g == 0)                                                // the bases are published with token 0
+            for (uint32_t i = tid; i < n; i += nt) {
+                s_src[i] = __ldcg(&p.seg[i].src_base);
+                s_stride[i] = __ldcg(&p.seg[i].src_stride);
+                s_dst[i] = __ldcg(&p.seg[i].dst_base);
+            }
+
+        // prefix sum of token g's miss counts over the tables of the call (n <= S1_MAX_TABLES)
+        uint32_t running = 0;
+        for (uint32_t base = 0; base < n; base += nt) {
+            const uint32_t i = base + tid;
+            const uint32_t c = i < n ? __ldcg(p.tcount + (size_t)i * p.n_q + g) : 0u;
+            uint32_t total;
+            const uint32_t excl = block_excl_scan(c, s_w, total);
+            if (i < n) s_pref[i] = running + excl;
+            running += total;
+            __syncthreads();
+        }
+        if (tid == 0) s_pref[n] = running;
+        __syncthreads();
+
+        const uint32_t C = gridDim.x, cb = blockIdx.x, q = running / C, r = running % C;
+        const uint32_t m0 = cb * q + (cb < r ? cb : r);
+        const uint32_t m1 = m0 + q + (cb < r ? 1u : 0u);
+        for (uint32_t m = m0 + (tid >> 5); m < m1; m += nt >> 5) {
+            uint32_t lo = 0, hi = n;                               // largest lo with s_pref[lo] <= m
+            while (hi - lo > 1) {
+                const uint32_t mid = (lo + hi) >> 1;
+                if (s_pref[mid] <= m) lo = mid; else hi = mid;
+            }
+            const uint32_t local = s_off[lo] + (m - s_pref[lo]);   // entry of the table's miss list
+            if (local >= p.list_stride) {
+                if (lane == 0) atomicOr(p.status, ST_BAD_SEGMENT);
+                continue;
+            }
+            const int2 e = __ldcg(p.miss_list + (size_t)lo * p.list_stride + local);
+            if (e.x < 0) continue;
+            if (e.y < 0 || (uint32_t)e.y >= p.S) {
+                if (lane == 0) atomicOr(p.status, ST_BAD_SLOT);
+                continue;
+            }
+            const uint64_t src = s_src[lo] + (uint64_t)(uint32_t)e.x * s_stride[lo];
+            const uint64_t dst = s_dst[lo] + (uint64_t)(uint32_t)e.y * p.row_bytes;
+            for (uint32_t c0 = lane; c0 < cpr; c0 += 32u * CHUNKS_PER_PASS) {
+                int4 v[CHUNKS_PER_PASS];
+#pragma unroll
+                for (int k = 0; k < CHUNKS_PER_PASS; ++k) {
+                    const uint32_t c = c0 + 32u * k;
+                    if (c < cpr) v[k] = *reinterpret_cast<const int4*>(src + 16ull * c);
+                }
+#pragma unroll
+                for (int k = 0; k < CHUNKS_PER_PASS; ++k) {
+                    const uint32_t c = c0 + 32u * k;
+                    if (c < cpr) *reinterpret_cast<int4*>(dst + 16ull * c) = v[k];
+                }
+            }
+        }
+        __syncthreads();
+        for (uint32_t i = tid; i < n; i += nt) s_off[i] += s_pref[i + 1] - s_pref[i];
+        __syncthreads();
+    }
+    if (p.t_range) {
+        __syncthreads();
+        if (tid == 0) atomicMax(p.t_range + 1, global_ns());
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // Comparator S2 (App. D, Eq. 14): the n * N_q * K selected positions of the call are flattened and cut into
 // gridDim.x near-equal contiguous ranges regardless of hit or miss; a block walks its range, one warp per
 // position, and copies the row of every position that missed.  Work per block = misses in its range (Eq. 15).
@@ -167,6 +275,21 @@ cudaError_t launch_transfer_positions(const PosParams& p, uint32_t blocks, uint3
 {
     avsg_transfer_positions_kernel<<<blocks, threads, 0, stream>>>(p);
     return cudaGetLastError();
+}
+
+cudaError_t launch_transfer_overlap(const XferOverlapParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, avsg_transfer_overlap_kernel, p);
 }
 
 cudaError_t launch_transfer(const XferParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream)

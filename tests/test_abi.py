@@ -27,7 +27,7 @@ def test_library_exports_every_declared_symbol():
 def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(avsg.AvsgConfig) == 52
     assert ctypes.sizeof(avsg.AvsgStepArgs) == 80
-    assert ctypes.sizeof(avsg.AvsgStats) == 80
+    assert ctypes.sizeof(avsg.AvsgStats) == 88
 
 
 def test_error_strings_and_argument_errors_need_no_gpu():

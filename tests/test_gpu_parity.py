@@ -120,6 +120,61 @@ def test_transfer_geometries(avsg):
         _parity(w, xfer_geometry=geo)
 
 
+# ---- Stage Two overlapping Stage One (latency hiding, App. G) ---------------------------------------------------
+@pytest.mark.parametrize("name,kw,index", [
+    ("C1", {}, "INDEX_HASH"), ("C2", {}, "INDEX_HASH"), ("C2", {}, "INDEX_DIRECT"), ("C3", {}, "INDEX_DIRECT"),
+    ("C3", dict(requests=16, layers=2, n_iters=32), "INDEX_HASH"), ("C4", {}, "INDEX_DIRECT"), ("C5", {}, "INDEX_HASH"),
+])
+def test_overlap_mode_full(avsg, name, kw, index):
+    r = _parity(tr.workload(name, **kw), mode=avsg.XFER_SM_OVERLAP, index_mode=getattr(avsg, index), buffer_every=8)
+    assert r["gpu"]["rows_copied"] == r["oracle"]["rows_copied"] > 0
+
+
+@pytest.mark.parametrize("name,kw", SHAPES)
+def test_overlap_mode_shapes(avsg, name, kw):
+    _parity(tr.workload(name, **kw), mode=avsg.XFER_SM_OVERLAP)
+
+
+def test_overlap_mode_host_io_strides_geometries_and_fallbacks(avsg):
+    w = tr.workload("C4", topk=256, buffer_slots=1024, n_iters=12, context=1 << 15, requests=3, hot_size=64,
+                    hot_range=1024)
+    _parity(w, mode=avsg.XFER_SM_OVERLAP, host_io=True)
+    _parity(w, mode=avsg.XFER_SM_OVERLAP, row_stride=1024, index_mode=avsg.INDEX_DIRECT)
+    for geo in [(1, 32), (7, 1024), (600, 256)]:
+        _parity(w, mode=avsg.XFER_SM_OVERLAP, xfer_geometry=geo)
+    # more tables than one Stage One launch takes, and the paper-literal index, run as the balanced mode
+    many = tr.workload("C5", topk=64, buffer_slots=128, n_iters=6, requests=300, ctx_lo=256, ctx_hi=2048)
+    _parity(many, mode=avsg.XFER_SM_OVERLAP, buffer_every=3)
+
+
+def test_overlap_mode_four_tokens_and_mode_switches(avsg):
+    """MTP-3: four tokens per iteration, i.e. four publish / wait rounds per call; the transfer mode is switched
+    between calls, so calls with and without the per-token counters alternate on one context."""
+    import torch
+    S, K, n_q, T, rb, n = 2048, 384, 4, 12, 656, 3
+    w = tr.workload("C5", topk=K, buffer_slots=S, n_iters=n_q * T, requests=n, ctx_lo=20000, ctx_hi=20001, row_bytes=rb)
+    traces = [tr.generate(c) for c in w.tables]
+    kv, kvn = [], []
+    for ti, cfg in enumerate(w.tables):
+        b = avsg.pinned_empty(cfg.context * rb)
+        tr.fill_kv(b.data_ptr(), w.seed, ti, cfg.context, rb)
+        kv.append(b); kvn.append(b.numpy())
+    ctx = avsg.Context(n, S, rb, K, n_q, 16, transfer_mode=avsg.XFER_SM_OVERLAP)
+    orc = [OracleTable(S, rb, 16) for _ in range(n)]
+    for t in range(T):
+        ctx.set_transfer_mode(avsg.XFER_SM_BALANCED if t % 4 == 3 else avsg.XFER_SM_OVERLAP)
+        X = np.stack([traces[ti][0][n_q * t:n_q * (t + 1), 0, :] for ti in range(n)])     # [n, n_q, K]
+        N = [w.tables[ti].context for ti in range(n)]
+        out = ctx.step(list(range(n)), torch.from_numpy(np.ascontiguousarray(X)).cuda(), kv, N)
+        torch.cuda.synchronize()
+        slots, hit, mc = out.slots.cpu().numpy(), out.hit.cpu().numpy(), out.miss_count.cpu().numpy()
+        for ti in range(n):
+            r = orc[ti].step(X[ti], N[ti], kvn[ti], rb)
+            assert (slots[ti] == r.O).all() and (hit[ti] == r.M).all() and (mc[ti] == r.n).all(), (t, ti)
+            assert (ctx.buffer(ti).cpu().numpy() == orc[ti].rows()).all(), (t, ti)
+    assert ctx.sync_status() == 0
+
+
 # ---- behaviours ---------------------------------------------------------------------------------------------
 def test_regenerated_speculative_row_is_fetched_again(avsg):
     import torch
@@ -415,7 +470,8 @@ def test_random_shapes(avsg, seed):
         w = tr.workload("C5", requests=requests, ctx_lo=max(4, K // 2), ctx_hi=ctxlen, **kw)
     if w.n_q * w.topk > w.buffer_slots:                                  # the MTP recipes have two tokens
         w = tr.workload("C5", requests=requests, ctx_lo=max(4, K // 2), ctx_hi=ctxlen, **kw)
-    mode = getattr(avsg, str(rng.choice(["XFER_SM_BALANCED", "XFER_REQUEST_LEVEL", "XFER_POSITION_LEVEL"])))
+    mode = getattr(avsg, str(rng.choice(["XFER_SM_BALANCED", "XFER_REQUEST_LEVEL", "XFER_POSITION_LEVEL",
+                                         "XFER_SM_OVERLAP"])))
     index_mode = int(rng.choice([avsg.INDEX_HASH, avsg.INDEX_DIRECT]))
     _parity(w, mode=mode, index_mode=index_mode, host_io=bool(rng.random() < 0.3),
             xfer_geometry=(int(rng.choice([1, 37, 148, 300])), int(rng.choice([32, 128, 256, 1024]))))
