@@ -47,6 +47,24 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* s_w, u
     return incl - v + s_w[warp];
 }
 
+// One warp moves one row: 16-byte loads from the (host) source, all issued before the 16-byte stores into the slot.
+__device__ __forceinline__ void copy_row(uint64_t src, uint64_t dst, uint32_t cpr, uint32_t lane)
+{
+    for (uint32_t c0 = lane; c0 < cpr; c0 += 32u * CHUNKS_PER_PASS) {
+        int4 v[CHUNKS_PER_PASS];
+#pragma unroll
+        for (int k = 0; k < CHUNKS_PER_PASS; ++k) {
+            const uint32_t c = c0 + 32u * k;
+            if (c < cpr) v[k] = *reinterpret_cast<const int4*>(src + 16ull * c);
+        }
+#pragma unroll
+        for (int k = 0; k < CHUNKS_PER_PASS; ++k) {
+            const uint32_t c = c0 + 32u * k;
+            if (c < cpr) *reinterpret_cast<int4*>(dst + 16ull * c) = v[k];
+        }
+    }
+}
+
 __global__ void __launch_bounds__(1024, 1) avsg_transfer_kernel(const __grid_constant__ XferParams p)
 {
     __shared__ uint32_t s_pref[XFER_MAX_SEG + 1];
@@ -105,19 +123,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_kernel(const __grid_con
         }
         const uint64_t src = __ldg(&p.seg[lo].src_base) + (uint64_t)(uint32_t)e.x * __ldg(&p.seg[lo].src_stride);
         const uint64_t dst = __ldg(&p.seg[lo].dst_base) + (uint64_t)(uint32_t)e.y * p.row_bytes;
-        for (uint32_t c0 = lane; c0 < cpr; c0 += 32u * CHUNKS_PER_PASS) {
-            int4 v[CHUNKS_PER_PASS];
-#pragma unroll
-            for (int k = 0; k < CHUNKS_PER_PASS; ++k) {
-                const uint32_t c = c0 + 32u * k;
-                if (c < cpr) v[k] = *reinterpret_cast<const int4*>(src + 16ull * c);
-            }
-#pragma unroll
-            for (int k = 0; k < CHUNKS_PER_PASS; ++k) {
-                const uint32_t c = c0 + 32u * k;
-                if (c < cpr) *reinterpret_cast<int4*>(dst + 16ull * c) = v[k];
-            }
-        }
+        copy_row(src, dst, cpr, lane);
     }
     if (p.t_range) {
         __syncthreads();
@@ -208,19 +214,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __
             }
             const uint64_t src = s_src[lo] + (uint64_t)(uint32_t)e.x * s_stride[lo];
             const uint64_t dst = s_dst[lo] + (uint64_t)(uint32_t)e.y * p.row_bytes;
-            for (uint32_t c0 = lane; c0 < cpr; c0 += 32u * CHUNKS_PER_PASS) {
-                int4 v[CHUNKS_PER_PASS];
-#pragma unroll
-                for (int k = 0; k < CHUNKS_PER_PASS; ++k) {
-                    const uint32_t c = c0 + 32u * k;
-                    if (c < cpr) v[k] = *reinterpret_cast<const int4*>(src + 16ull * c);
-                }
-#pragma unroll
-                for (int k = 0; k < CHUNKS_PER_PASS; ++k) {
-                    const uint32_t c = c0 + 32u * k;
-                    if (c < cpr) *reinterpret_cast<int4*>(dst + 16ull * c) = v[k];
-                }
-            }
+            copy_row(src, dst, cpr, lane);
         }
         __syncthreads();
         for (uint32_t i = tid; i < n; i += nt) s_off[i] += s_pref[i + 1] - s_pref[i];
@@ -253,19 +247,7 @@ __global__ void __launch_bounds__(1024) avsg_transfer_positions_kernel(const __g
         const uint32_t ti = (uint32_t)(q / p.per_table);
         const uint64_t src = __ldg(&p.seg[ti].src_base) + (uint64_t)(uint32_t)x * __ldg(&p.seg[ti].src_stride);
         const uint64_t dst = __ldg(&p.seg[ti].dst_base) + (uint64_t)(uint32_t)o * p.row_bytes;
-        for (uint32_t c0 = lane; c0 < cpr; c0 += 32u * CHUNKS_PER_PASS) {
-            int4 v[CHUNKS_PER_PASS];
-#pragma unroll
-            for (int k = 0; k < CHUNKS_PER_PASS; ++k) {
-                const uint32_t cc = c0 + 32u * k;
-                if (cc < cpr) v[k] = *reinterpret_cast<const int4*>(src + 16ull * cc);
-            }
-#pragma unroll
-            for (int k = 0; k < CHUNKS_PER_PASS; ++k) {
-                const uint32_t cc = c0 + 32u * k;
-                if (cc < cpr) *reinterpret_cast<int4*>(dst + 16ull * cc) = v[k];
-            }
-        }
+        copy_row(src, dst, cpr, lane);
     }
 }
 
