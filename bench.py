@@ -488,6 +488,46 @@ def _suite_one(avsg, torch, tr, name, mode, mode_name, link_peak, needed_rows=No
     return out
 
 
+def _suite_modes(avsg, torch, tr, name, **kw):
+    """Device time of one iteration (all its calls; CUDA events around it, L2 flushed before it) in the steady state,
+    with Stage Two after Stage One (balanced) and overlapping it, for both Stage One indexes."""
+    w = tr.workload(name, **kw)
+    traces = _gen_traces(w, os.cpu_count() or 1)
+    kv = []
+    for ti, cfg in enumerate(w.tables):
+        buf = avsg.pinned_empty(cfg.context * w.row_bytes)
+        tr.fill_kv(buf.data_ptr(), w.seed, ti, cfg.context, w.row_bytes)
+        kv.append(buf)
+    T = w.n_iters
+    X = [[torch.from_numpy(np.stack([traces[ti][0][t] for ti in grp])).cuda() for grp in w.calls] for t in range(T)]
+    V = [[[int(traces[ti][1][t]) for ti in grp] for grp in w.calls] for t in range(T)]
+    slots = [torch.empty_like(x) for x in X[0]]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    out = {"suite": "stage_two_modes", "config": name, "us_per_iteration": {}}
+    for index, iname in ((avsg.INDEX_DIRECT, "direct"), (avsg.INDEX_HASH, "hash")):
+        for mode, mname in ((avsg.XFER_SM_BALANCED, "balanced"), (avsg.XFER_SM_OVERLAP, "overlap")):
+            ctx = avsg.Context(num_tables=w.num_tables, buffer_slots=w.buffer_slots, row_bytes=w.row_bytes,
+                               max_topk=w.topk, max_tokens=w.n_q, max_lifetime=w.max_lifetime, transfer_mode=mode,
+                               index_mode=index, max_context=max(c.context for c in w.tables) + w.n_q)
+            calls = [ctx.prepare(grp, [kv[t] for t in grp], w.n_q, w.topk, None) for grp in w.calls]
+            us = []
+            for t in range(T):
+                flush.fill_(t & 0xFF)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for c, call in enumerate(calls):
+                    call.run(X[t][c], V[t][c], slots[c], None, None, stream)
+                e1.record()
+                torch.cuda.synchronize()
+                if t >= T // 4:
+                    us.append(e0.elapsed_time(e1) * 1e3)
+            assert ctx.sync_status() == 0
+            out["us_per_iteration"]["%s/%s" % (iname, mname)] = sum(us) / len(us)
+            del ctx, calls
+    return out
+
+
 def run_suite(args):
     import torch
     import __graft_entry__
@@ -521,6 +561,8 @@ def run_suite(args):
                             n_iters=6)
             r2.pop("rows_per_iter_list")
             print(json.dumps(r2), flush=True)
+    for name, kw in (("C1", {}), ("C2", {}), ("C3", {"n_iters": 32}), ("C4", {"n_iters": 32}), ("C5", {})):
+        print(json.dumps(_suite_modes(avsg, torch, tr, name, **kw)), flush=True)
 
 
 # ------------------------------------------------------------------------------------------------------------
