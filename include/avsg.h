@@ -44,6 +44,15 @@ extern "C" {
 #define AVSG_EDEVICE_STATUS -5   /* a kernel reported a problem in the status word      */
 #define AVSG_EUNSUPPORTED   -6   /* shape outside what this build supports              */
 
+/* Bits of the device status word (avsg_sync_status).  The word is sticky until
+ * avsg_clear_status(). */
+#define AVSG_STATUS_PROBE_EXHAUSTED 0x01u /* hash index: a probe visited every bucket          */
+#define AVSG_STATUS_NO_DEAD_SLOTS   0x02u /* fewer reclaimable slots than misses (Eq. 7)        */
+#define AVSG_STATUS_BAD_SLOT        0x04u /* a slot or position index out of range              */
+#define AVSG_STATUS_BAD_SEGMENT     0x08u /* Stage Two could not resolve a miss-list entry      */
+#define AVSG_STATUS_BAD_ID          0x10u /* direct index: id >= max_context (taken as padding) */
+#define AVSG_STATUS_WAIT_TIMEOUT    0x20u /* overlapped Stage Two gave up waiting for Stage One */
+
 /* How Stage Two moves the missed rows (Sec. 3.4; App. D strategies). */
 #define AVSG_XFER_SM_BALANCED   0u  /* miss list cut evenly over all SMs (the operator)  */
 #define AVSG_XFER_COPY_ENGINE   1u  /* comparator: miss list read back, one async copy
@@ -176,6 +185,17 @@ int avsg_table_stats(avsg_ctx *ctx, uint32_t table_id, avsg_stats_t *out);
 /* Waits for the device; returns AVSG_EDEVICE_STATUS if a kernel flagged a
  * problem, and the raw status word in *status_word when not NULL. */
 int avsg_sync_status(avsg_ctx *ctx, uint32_t *status_word);
+
+/* Waits for the device and zeroes the status word. */
+int avsg_clear_status(avsg_ctx *ctx);
+
+/* Diagnostic for AVSG_XFER_SM_OVERLAP: launches the overlapped transfer kernel
+ * alone on cuda_stream, waiting for a Stage One that is never launched.  Its
+ * blocks poll up to their limit (about 0.2 s), raise AVSG_STATUS_WAIT_TIMEOUT,
+ * copy nothing and return: a lost Stage One cannot hang the stream, and the
+ * context stays usable (clear the status word afterwards).  The paper has no
+ * counterpart; its Stage Two starts after Stage One (Alg. 4). */
+int avsg_probe_wait_limit(avsg_ctx *ctx, void *cuda_stream);
 
 /* Table state for checkpoints and parity checks.  HOST tok[S] (cached id per
  * slot, -1 empty) and life[S] (lifetime, -1 dead).  Synchronous. */

@@ -18,12 +18,15 @@ from . import build as _build
 OK, EINVAL, ENOMEM, ECUDA, ECAPACITY, EDEVICE_STATUS, EUNSUPPORTED = 0, -1, -2, -3, -4, -5, -6
 XFER_SM_BALANCED, XFER_COPY_ENGINE, XFER_REQUEST_LEVEL, XFER_ALL_K, XFER_POSITION_LEVEL, XFER_SM_OVERLAP = 0, 1, 2, 3, 4, 5
 INDEX_HASH, INDEX_DIRECT, INDEX_PAPER = 0, 1, 2
+STATUS_PROBE_EXHAUSTED, STATUS_NO_DEAD_SLOTS, STATUS_BAD_SLOT, STATUS_BAD_SEGMENT, STATUS_BAD_ID, STATUS_WAIT_TIMEOUT = (
+    1, 2, 4, 8, 16, 32)
 
 EXPORTS = (
     "avsg_create", "avsg_destroy", "avsg_reset", "avsg_step", "avsg_step_host", "avsg_buffer", "avsg_stats", "avsg_table_stats",
     "avsg_sync_status", "avsg_export_state", "avsg_import_state", "avsg_save_state", "avsg_restore_state",
     "avsg_set_transfer_mode", "avsg_set_timing", "avsg_set_transfer_geometry", "avsg_strerror",
-    "avsg_step_noalloc", "avsg_export_hash_state", "avsg_import_hash_state",
+    "avsg_step_noalloc", "avsg_export_hash_state", "avsg_import_hash_state", "avsg_clear_status",
+    "avsg_probe_wait_limit",
 )
 
 
@@ -91,6 +94,8 @@ def load_library():
     lib.avsg_stats.argtypes, lib.avsg_stats.restype = [vp, ctypes.POINTER(AvsgStats)], i32
     lib.avsg_table_stats.argtypes, lib.avsg_table_stats.restype = [vp, u32, ctypes.POINTER(AvsgStats)], i32
     lib.avsg_sync_status.argtypes, lib.avsg_sync_status.restype = [vp, ctypes.POINTER(u32)], i32
+    lib.avsg_clear_status.argtypes, lib.avsg_clear_status.restype = [vp], i32
+    lib.avsg_probe_wait_limit.argtypes, lib.avsg_probe_wait_limit.restype = [vp, vp], i32
     lib.avsg_export_state.argtypes, lib.avsg_export_state.restype = [vp, u32, vp, vp], i32
     lib.avsg_import_state.argtypes, lib.avsg_import_state.restype = [vp, u32, vp, vp], i32
     lib.avsg_save_state.argtypes, lib.avsg_save_state.restype = [vp, vp], i32
@@ -306,6 +311,13 @@ class Context:
         if rc != EDEVICE_STATUS:
             _check(rc, "avsg_sync_status")
         return w.value
+
+    def clear_status(self) -> None:
+        _check(self._lib.avsg_clear_status(self._h), "avsg_clear_status")
+
+    def probe_wait_limit(self, stream=None) -> None:
+        """Launches the overlapped transfer kernel alone (its Stage One never comes): it must give up by itself."""
+        _check(self._lib.avsg_probe_wait_limit(self._h, _stream_handle(stream)), "avsg_probe_wait_limit")
 
     def stats(self) -> dict:
         s = AvsgStats()

@@ -493,6 +493,32 @@ int avsg_sync_status(avsg_ctx* c, uint32_t* status_word)
     return read_status(c, status_word);
 }
 
+int avsg_clear_status(avsg_ctx* c)
+{
+    if (!c) return AVSG_EINVAL;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return AVSG_ECUDA;
+    CU(cudaDeviceSynchronize());
+    CU(cudaMemset(c->d_status, 0, sizeof(uint32_t)));
+    return AVSG_OK;
+}
+
+int avsg_probe_wait_limit(avsg_ctx* c, void* cuda_stream)
+{
+    if (!c) return AVSG_EINVAL;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return AVSG_ECUDA;
+    XferOverlapParams x;
+    x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
+    x.tcount = c->d_tcount; x.ready = c->d_ready;
+    for (uint32_t g = 0; g < (uint32_t)OVERLAP_MAX_TOKENS; ++g) x.target[g] = c->posted[g];
+    x.target[0] = c->posted[0] + 1;                    // one more table than any Stage One launched so far will post
+    x.n = 1; x.n_q = 1; x.list_stride = c->list_stride; x.row_bytes = c->cfg.row_bytes; x.S = c->cfg.buffer_slots;
+    CU(launch_transfer_overlap(x, c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count, c->xfer_threads,
+                               static_cast<cudaStream_t>(cuda_stream)));
+    return AVSG_OK;
+}
+
 int avsg_export_state(avsg_ctx* c, uint32_t table_id, int32_t* tok, int8_t* life)
 {
     if (!c || !tok || !life || table_id >= c->cfg.num_tables) return AVSG_EINVAL;

@@ -175,6 +175,42 @@ def test_overlap_mode_four_tokens_and_mode_switches(avsg):
     assert ctx.sync_status() == 0
 
 
+def test_overlap_wait_gives_up_and_the_context_stays_usable(avsg):
+    """The overlapped transfer kernel launched without its Stage One: every block polls up to its limit, raises
+    the status bit, copies nothing and returns; after clearing the status word the context works as before."""
+    import time
+    import torch
+    w = tr.workload("C2", topk=256, buffer_slots=1024, n_iters=8, context=16384, recent_window=1024)
+    X, N = tr.generate(w.tables[0])
+    kv = avsg.pinned_empty(w.tables[0].context * w.row_bytes)
+    tr.fill_kv(kv.data_ptr(), w.seed, 0, w.tables[0].context, w.row_bytes)
+    ctx = avsg.Context(1, w.buffer_slots, w.row_bytes, w.topk, w.n_q, 16, transfer_mode=avsg.XFER_SM_OVERLAP)
+    orc = OracleTable(w.buffer_slots, w.row_bytes, 16)
+
+    def step(t):
+        out = ctx.step([0], torch.from_numpy(X[t][None]).cuda(), [kv], [int(N[t])])
+        torch.cuda.synchronize()
+        r = orc.step(X[t], int(N[t]), kv.numpy(), w.row_bytes)
+        assert (out.slots[0].cpu().numpy() == r.O).all() and (out.hit[0].cpu().numpy() == r.M).all(), t
+        assert (ctx.buffer(0).cpu().numpy() == orc.rows()).all(), t
+
+    for t in range(4):
+        step(t)
+    assert ctx.sync_status() == 0
+    before = ctx.buffer(0).cpu().numpy().copy()
+    t0 = time.time()
+    ctx.probe_wait_limit()
+    word = ctx.sync_status()
+    assert time.time() - t0 < 10.0
+    assert word == avsg.STATUS_WAIT_TIMEOUT, word
+    assert (ctx.buffer(0).cpu().numpy() == before).all()
+    ctx.clear_status()
+    assert ctx.sync_status() == 0
+    for t in range(4, 8):
+        step(t)
+    assert ctx.sync_status() == 0
+
+
 # ---- behaviours ---------------------------------------------------------------------------------------------
 def test_regenerated_speculative_row_is_fetched_again(avsg):
     import torch
