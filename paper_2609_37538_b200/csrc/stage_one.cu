@@ -32,6 +32,9 @@
 // the k-th miss in position order takes the k-th of them (ballot-free packed
 // byte arithmetic + warp/block prefix sums, no atomics, so the assignment is
 // deterministic).
+//
+// When Stage Two overlaps Stage One (S1Params::ready set), the block announces
+// every token as soon as its misses are placed: see `publish` in the kernel.
 #include "avsg_kernels.cuh"
 
 namespace avsg {

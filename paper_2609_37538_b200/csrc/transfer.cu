@@ -13,6 +13,10 @@
 //
 // request_level = 1 gives the comparator S1 of App. D: block b serves
 // segment b alone.
+//
+// avsg_transfer_overlap_kernel is the same gather started per token while
+// Stage One still runs (App. G, latency hiding; described at the kernel), and
+// avsg_transfer_positions_kernel is the comparator S2 of App. D.
 #include "avsg_kernels.cuh"
 
 namespace avsg {
