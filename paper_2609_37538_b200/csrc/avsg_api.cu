@@ -5,6 +5,8 @@
 #include <string.h>
 #include <vector>
 
+#include <cuda.h>          // types of the one driver entry point fetched at run time (nothing links libcuda)
+
 #include "avsg.h"
 #include "avsg_kernels.cuh"
 
@@ -51,6 +53,9 @@ struct avsg_ctx {
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
     // avsg_step_host: the outputs go back on a side stream while Stage Two runs
     cudaStream_t side = nullptr;
+    // cuStreamWaitValue64, when the driver offers it: lets the side stream start the output download as soon as
+    // Stage One has published its last token, without an event between Stage One and an overlapped Stage Two
+    CUresult (*wait_value64)(CUstream, CUdeviceptr, cuuint64_t, unsigned int) = nullptr;
     cudaEvent_t ev_outputs_ready = nullptr, ev_outputs_copied = nullptr, ev_ids_ready = nullptr;
     uint64_t last_rows = 0;
 };
@@ -246,16 +251,23 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
     // (no event between the two grids in overlap mode: it would serialise them; ev[1] is recorded with ev[2])
     if (c->timing && mode != AVSG_XFER_SM_OVERLAP) CU(cudaEventRecord(c->ev[1], stream));
 
-    if (host_io) {
-        // The slot table, hit mask and miss counts are final once Stage One has run.  They travel device -> host
-        // on a side stream while Stage Two pulls rows host -> device: the two directions of the link overlap.
-        CU(cudaEventRecord(c->ev_outputs_ready, stream));
-        CU(cudaStreamWaitEvent(c->side, c->ev_outputs_ready, 0));
+    // The slot table, hit mask and miss counts are final once Stage One has run.  They travel device -> host on a
+    // side stream while Stage Two pulls rows host -> device: the two directions of the link overlap.
+    auto download_outputs = [&]() -> int {
         CU(cudaMemcpyAsync(a->slots, c->d_slots_stage, n_ids * sizeof(int32_t), cudaMemcpyDeviceToHost, c->side));
         if (a->hit) CU(cudaMemcpyAsync(a->hit, c->d_hit_stage, n_ids, cudaMemcpyDeviceToHost, c->side));
         if (a->miss_count)
             CU(cudaMemcpyAsync(a->miss_count, c->d_mc_stage, (size_t)n * n_q * sizeof(int32_t), cudaMemcpyDeviceToHost, c->side));
         CU(cudaEventRecord(c->ev_outputs_copied, c->side));
+        return AVSG_OK;
+    };
+    // In overlap mode an event between the two grids would serialise them: the side stream waits for the value
+    // Stage One's last-token counter reaches instead (all outputs are written before that counter is raised).
+    const bool wait_on_counter = host_io && mode == AVSG_XFER_SM_OVERLAP && c->wait_value64 != nullptr;
+    if (host_io && !wait_on_counter) {
+        CU(cudaEventRecord(c->ev_outputs_ready, stream));
+        CU(cudaStreamWaitEvent(c->side, c->ev_outputs_ready, 0));
+        if ((rc = download_outputs()) != AVSG_OK) return rc;
     }
 
     if (mode == AVSG_XFER_COPY_ENGINE) {
@@ -276,6 +288,12 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         x.n = n; x.n_q = n_q; x.list_stride = c->list_stride; x.row_bytes = c->cfg.row_bytes; x.S = c->cfg.buffer_slots;
         x.t_range = c->timing ? c->d_trange + 2 : nullptr;
         CU(launch_transfer_overlap(x, c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count, c->xfer_threads, stream));
+        if (wait_on_counter) {
+            if (c->wait_value64(c->side, reinterpret_cast<CUdeviceptr>(c->d_ready + (n_q - 1)), c->posted[n_q - 1],
+                                CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
+                return AVSG_ECUDA;
+            if ((rc = download_outputs()) != AVSG_OK) return rc;
+        }
     } else {
         XferParams x;
         x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
@@ -375,6 +393,15 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaHostAlloc(&c->h_list, n_ids * sizeof(int2), cudaHostAllocDefault) == cudaSuccess;
     for (auto& e : c->ev) ok = ok && cudaEventCreate(&e) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
+    {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult found = cudaDriverEntryPointSymbolNotFound;
+        if (cudaGetDriverEntryPoint("cuStreamWaitValue64", &fn, cudaEnableDefault, &found) == cudaSuccess &&
+            found == cudaDriverEntryPointSuccess)
+            c->wait_value64 = reinterpret_cast<CUresult (*)(CUstream, CUdeviceptr, cuuint64_t, unsigned int)>(fn);
+        else
+            cudaGetLastError();
+    }
     ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_ready, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_copied, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_ids_ready, cudaEventDisableTiming) == cudaSuccess;
