@@ -739,6 +739,38 @@ def run_sweeps(args):
             h = sum(a for a, _ in per[40:]); m = sum(b for _, b in per[40:])
             print(json.dumps({"sweep": "index_mode", "n_tokens": n_q, "index": label, "hit_rate": h / (h + m),
                               "rows_copied_per_table_iter": m / 16 / 160, "match_reserve_us_median": med}), flush=True)
+    # (f) what the overlapped Stage Two buys as the MTP degree grows: one 32-table call per iteration, K = 2048,
+    #     8K pool, direct index; device time per call (CUDA events, L2 flushed before each), steady iterations
+    kvs = [avsg.pinned_empty(131072 * 656) for _ in range(32)]
+    for i, b in enumerate(kvs):
+        tr.fill_kv(b.data_ptr(), 77, i, 131072, 656)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    for n_q in (1, 2, 3, 4):
+        cfgs = [recipe(i, 2048, n_q, 40) for i in range(32)]
+        traces = [tr.generate(c) for c in cfgs]
+        X = [torch.from_numpy(np.stack([traces[i][0][t] for i in range(32)])).cuda() for t in range(40)]
+        V = [[int(traces[i][1][t]) for i in range(32)] for t in range(40)]
+        slots = torch.empty_like(X[0])
+        row = {"sweep": "overlap_vs_tokens", "n_tokens": n_q}
+        for mode, mname in ((avsg.XFER_SM_BALANCED, "balanced"), (avsg.XFER_SM_OVERLAP, "overlap")):
+            ctx = avsg.Context(num_tables=32, buffer_slots=8192, row_bytes=656, max_topk=2048, max_tokens=n_q,
+                               max_lifetime=16, transfer_mode=mode, index_mode=avsg.INDEX_DIRECT, max_context=131072 + n_q)
+            call = ctx.prepare(list(range(32)), kvs, n_q, 2048)
+            us = []
+            for t in range(40):
+                flush.fill_(t)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); call.run(X[t], V[t], slots, None, None, stream); e1.record()
+                torch.cuda.synchronize()
+                if t >= 10:
+                    us.append(e0.elapsed_time(e1) * 1e3)
+            st = ctx.stats()
+            row[mname + "_us"] = sum(us) / len(us)
+            row["rows_copied_total"] = st["rows_copied"]
+            ctx.close()
+        print(json.dumps(row), flush=True)
+    del kvs
     # (d) MTP cold start: reuse inside the first iteration from an empty buffer, degrees 0..3, 32 tables
     for deg in range(4):
         per, _ = _run_tables(avsg, torch, tr, [recipe(i, 2048, deg + 1, 1) for i in range(32)], 8192, 16)
