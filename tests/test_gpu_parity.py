@@ -175,6 +175,35 @@ def test_overlap_mode_four_tokens_and_mode_switches(avsg):
     assert ctx.sync_status() == 0
 
 
+@pytest.mark.parametrize("n,n_q,K,S", [(128, 2, 64, 256),      # as many tables as one Stage One launch takes
+                                        (5, 8, 96, 1024),       # as many tokens as the overlapped kernel takes
+                                        (3, 9, 100, 1024),      # one more: runs as the balanced mode
+                                        (129, 1, 32, 64)])      # one table more than a launch: balanced mode
+def test_overlap_mode_limits(avsg, n, n_q, K, S):
+    import torch
+    T, rb, ctxlen = 10, 48, 6000
+    cfgs = [tr.TraceConfig(seed=5, table=i, topk=K, n_q=n_q, n_iters=T, context=ctxlen, ctx_growth=n_q > 1,
+                           beta=(9, 1), p_recent=0.5, recent_window=512) for i in range(n)]
+    traces = [tr.generate(c) for c in cfgs]
+    kv = avsg.pinned_empty(ctxlen * rb)                 # every table reads the same host rows
+    tr.fill_kv(kv.data_ptr(), 5, 0, ctxlen, rb)
+    ctx = avsg.Context(n, S, rb, K, n_q, 16, transfer_mode=avsg.XFER_SM_OVERLAP, index_mode=avsg.INDEX_DIRECT,
+                       max_context=ctxlen + n_q)
+    orc = [OracleTable(S, rb, 16) for _ in range(n)]
+    for t in range(T):
+        X = np.stack([traces[i][0][t] for i in range(n)])
+        N = [int(traces[i][1][t]) for i in range(n)]
+        out = ctx.step(list(range(n)), torch.from_numpy(X).cuda(), [kv] * n, N)
+        torch.cuda.synchronize()
+        slots, mc = out.slots.cpu().numpy(), out.miss_count.cpu().numpy()
+        for i in range(n):
+            r = orc[i].step(X[i], N[i], kv.numpy(), rb)
+            assert (slots[i] == r.O).all() and (mc[i] == r.n).all(), (t, i)
+    for i in range(0, n, max(1, n // 7)):
+        assert (ctx.buffer(i).cpu().numpy() == orc[i].rows()).all(), i
+    assert ctx.sync_status() == 0
+
+
 def test_overlap_wait_gives_up_and_the_context_stays_usable(avsg):
     """The overlapped transfer kernel launched without its Stage One: every block polls up to its limit, raises
     the status bit, copies nothing and returns; after clearing the status word the context works as before."""
