@@ -401,6 +401,14 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
             c->wait_value64 = reinterpret_cast<CUresult (*)(CUstream, CUdeviceptr, cuuint64_t, unsigned int)>(fn);
         else
             cudaGetLastError();
+        // 64-bit stream memory operations must be supported by the device (attribute 122 of the driver's numbering,
+        // CU_DEVICE_ATTRIBUTE_CAN_USE_64_BIT_STREAM_MEM_OPS, which the runtime's enum does not name)
+        int can64 = 0;
+        if (cudaDeviceGetAttribute(&can64, static_cast<cudaDeviceAttr>(CU_DEVICE_ATTRIBUTE_CAN_USE_64_BIT_STREAM_MEM_OPS),
+                                   cfg->device) != cudaSuccess || !can64) {
+            c->wait_value64 = nullptr;
+            cudaGetLastError();
+        }
     }
     ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_ready, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_copied, cudaEventDisableTiming) == cudaSuccess;
