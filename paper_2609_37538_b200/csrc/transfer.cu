@@ -51,9 +51,32 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* s_w, u
     return incl - v + s_w[warp];
 }
 
+// 16-byte global load / store in the order written (volatile asm statements keep their relative order).
+__device__ __forceinline__ int4 ld16(uint64_t addr)
+{
+    int4 v;
+    asm volatile("ld.global.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(addr));
+    return v;
+}
+__device__ __forceinline__ void st16(uint64_t addr, const int4& v)
+{
+    asm volatile("st.global.v4.s32 [%0], {%1, %2, %3, %4};" :: "l"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
 // One warp moves one row: 16-byte loads from the (host) source, all issued before the 16-byte stores into the slot.
+// Rows of up to 1 KiB (two loads per lane) take the short path, whose instruction order is fixed by hand: both
+// loads of a lane are in flight together.
 __device__ __forceinline__ void copy_row(uint64_t src, uint64_t dst, uint32_t cpr, uint32_t lane)
 {
+    if (cpr <= 64u) {
+        const bool p0 = lane < cpr, p1 = lane + 32u < cpr;
+        int4 a = make_int4(0, 0, 0, 0), b = make_int4(0, 0, 0, 0);
+        if (p0) a = ld16(src + 16ull * lane);
+        if (p1) b = ld16(src + 16ull * (lane + 32u));
+        if (p0) st16(dst + 16ull * lane, a);
+        if (p1) st16(dst + 16ull * (lane + 32u), b);
+        return;
+    }
     for (uint32_t c0 = lane; c0 < cpr; c0 += 32u * CHUNKS_PER_PASS) {
         int4 v[CHUNKS_PER_PASS];
 #pragma unroll
