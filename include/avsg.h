@@ -186,7 +186,9 @@ int avsg_table_stats(avsg_ctx *ctx, uint32_t table_id, avsg_stats_t *out);
  * problem, and the raw status word in *status_word when not NULL. */
 int avsg_sync_status(avsg_ctx *ctx, uint32_t *status_word);
 
-/* Waits for the device and zeroes the status word. */
+/* Waits for the device, zeroes the status word and the counters of the
+ * overlapped mode (which a call that reported AVSG_STATUS_WAIT_TIMEOUT may have
+ * left raised). */
 int avsg_clear_status(avsg_ctx *ctx);
 
 /* Diagnostic for AVSG_XFER_SM_OVERLAP: launches the overlapped transfer kernel

@@ -5,8 +5,6 @@
 #include <string.h>
 #include <vector>
 
-#include <cuda.h>          // types of the one driver entry point fetched at run time (nothing links libcuda)
-
 #include "avsg.h"
 #include "avsg_kernels.cuh"
 
@@ -24,9 +22,9 @@ struct avsg_ctx {
     int8_t* d_life = nullptr;
     uint8_t* d_buffer = nullptr;
     TableStats* d_stats = nullptr;
-    unsigned long long* d_ready = nullptr;         // overlapped Stage Two: per-token counters [OVERLAP_MAX_TOKENS]
+    unsigned long long* d_ready = nullptr;         // overlapped Stage Two: per-token counters [OVERLAP_MAX_TOKENS],
+                                                   //   then one word counting the transfer blocks that are through
     uint32_t* d_tcount = nullptr;                  //   and per-(table of the call, token) miss counts
-    unsigned long long posted[OVERLAP_MAX_TOKENS] = {};   // value each counter has after the calls issued so far
     unsigned long long* d_trange = nullptr;        // [4] grid spans of the last timed call, then [4] their initial values
     unsigned long long* d_trange_init = nullptr;
     int2* d_list = nullptr;
@@ -53,9 +51,6 @@ struct avsg_ctx {
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
     // avsg_step_host: the outputs go back on a side stream while Stage Two runs
     cudaStream_t side = nullptr;
-    // cuStreamWaitValue64, when the driver offers it: lets the side stream start the output download as soon as
-    // Stage One has published its last token, without an event between Stage One and an overlapped Stage Two
-    CUresult (*wait_value64)(CUstream, CUdeviceptr, cuuint64_t, unsigned int) = nullptr;
     cudaEvent_t ev_outputs_ready = nullptr, ev_outputs_copied = nullptr, ev_ids_ready = nullptr;
     uint64_t last_rows = 0;
 };
@@ -261,10 +256,7 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         CU(cudaEventRecord(c->ev_outputs_copied, c->side));
         return AVSG_OK;
     };
-    // In overlap mode an event between the two grids would serialise them: the side stream waits for the value
-    // Stage One's last-token counter reaches instead (all outputs are written before that counter is raised).
-    const bool wait_on_counter = host_io && mode == AVSG_XFER_SM_OVERLAP && c->wait_value64 != nullptr;
-    if (host_io && !wait_on_counter) {
+    if (host_io) {
         CU(cudaEventRecord(c->ev_outputs_ready, stream));
         CU(cudaStreamWaitEvent(c->side, c->ev_outputs_ready, 0));
         if ((rc = download_outputs()) != AVSG_OK) return rc;
@@ -281,19 +273,11 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         XferOverlapParams x;
         x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
         x.tcount = c->d_tcount; x.ready = c->d_ready;
-        for (uint32_t g = 0; g < (uint32_t)OVERLAP_MAX_TOKENS; ++g) {
-            if (g < n_q) c->posted[g] += n;            // Stage One of this call (already launched) raises these
-            x.target[g] = c->posted[g];
-        }
+        x.done = reinterpret_cast<uint32_t*>(c->d_ready + OVERLAP_MAX_TOKENS);
         x.n = n; x.n_q = n_q; x.list_stride = c->list_stride; x.row_bytes = c->cfg.row_bytes; x.S = c->cfg.buffer_slots;
+        x.expect = n;
         x.t_range = c->timing ? c->d_trange + 2 : nullptr;
         CU(launch_transfer_overlap(x, c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count, c->xfer_threads, stream));
-        if (wait_on_counter) {
-            if (c->wait_value64(c->side, reinterpret_cast<CUdeviceptr>(c->d_ready + (n_q - 1)), c->posted[n_q - 1],
-                                CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
-                return AVSG_ECUDA;
-            if ((rc = download_outputs()) != AVSG_OK) return rc;
-        }
     } else {
         XferParams x;
         x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
@@ -372,7 +356,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaMalloc(&c->d_buffer, T * S * cfg->row_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_stats, T * sizeof(TableStats)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_trange, 8 * sizeof(unsigned long long)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->d_ready, OVERLAP_MAX_TOKENS * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_ready, (OVERLAP_MAX_TOKENS + 1) * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_tcount, (size_t)S1_MAX_TABLES * OVERLAP_MAX_TOKENS * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_list, n_ids * sizeof(int2)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_seg, T * sizeof(SegDesc)) == cudaSuccess;
@@ -393,23 +377,6 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaHostAlloc(&c->h_list, n_ids * sizeof(int2), cudaHostAllocDefault) == cudaSuccess;
     for (auto& e : c->ev) ok = ok && cudaEventCreate(&e) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
-    {
-        void* fn = nullptr;
-        cudaDriverEntryPointQueryResult found = cudaDriverEntryPointSymbolNotFound;
-        if (cudaGetDriverEntryPoint("cuStreamWaitValue64", &fn, cudaEnableDefault, &found) == cudaSuccess &&
-            found == cudaDriverEntryPointSuccess)
-            c->wait_value64 = reinterpret_cast<CUresult (*)(CUstream, CUdeviceptr, cuuint64_t, unsigned int)>(fn);
-        else
-            cudaGetLastError();
-        // 64-bit stream memory operations must be supported by the device (attribute 122 of the driver's numbering,
-        // CU_DEVICE_ATTRIBUTE_CAN_USE_64_BIT_STREAM_MEM_OPS, which the runtime's enum does not name)
-        int can64 = 0;
-        if (cudaDeviceGetAttribute(&can64, static_cast<cudaDeviceAttr>(CU_DEVICE_ATTRIBUTE_CAN_USE_64_BIT_STREAM_MEM_OPS),
-                                   cfg->device) != cudaSuccess || !can64) {
-            c->wait_value64 = nullptr;
-            cudaGetLastError();
-        }
-    }
     ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_ready, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_copied, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_ids_ready, cudaEventDisableTiming) == cudaSuccess;
@@ -418,7 +385,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
         const unsigned long long never = ~0ull, init[8] = {never, 0, never, 0, never, 0, never, 0};
         c->d_trange_init = c->d_trange + 4;
         if (cudaMemcpy(c->d_trange, init, sizeof(init), cudaMemcpyHostToDevice) != cudaSuccess ||
-            cudaMemset(c->d_ready, 0, OVERLAP_MAX_TOKENS * sizeof(unsigned long long)) != cudaSuccess) {
+            cudaMemset(c->d_ready, 0, (OVERLAP_MAX_TOKENS + 1) * sizeof(unsigned long long)) != cudaSuccess) {
             free_all(c); delete c; return AVSG_ECUDA;
         }
     }
@@ -535,6 +502,8 @@ int avsg_clear_status(avsg_ctx* c)
     if (!guard.ok) return AVSG_ECUDA;
     CU(cudaDeviceSynchronize());
     CU(cudaMemset(c->d_status, 0, sizeof(uint32_t)));
+    // a transfer kernel that gave up may have left the per-token counters of the overlapped mode raised
+    CU(cudaMemset(c->d_ready, 0, (OVERLAP_MAX_TOKENS + 1) * sizeof(unsigned long long)));
     return AVSG_OK;
 }
 
@@ -546,9 +515,9 @@ int avsg_probe_wait_limit(avsg_ctx* c, void* cuda_stream)
     XferOverlapParams x;
     x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
     x.tcount = c->d_tcount; x.ready = c->d_ready;
-    for (uint32_t g = 0; g < (uint32_t)OVERLAP_MAX_TOKENS; ++g) x.target[g] = c->posted[g];
-    x.target[0] = c->posted[0] + 1;                    // one more table than any Stage One launched so far will post
+    x.done = reinterpret_cast<uint32_t*>(c->d_ready + OVERLAP_MAX_TOKENS);
     x.n = 1; x.n_q = 1; x.list_stride = c->list_stride; x.row_bytes = c->cfg.row_bytes; x.S = c->cfg.buffer_slots;
+    x.expect = 1;                                       // one table's token that no Stage One will place
     CU(launch_transfer_overlap(x, c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count, c->xfer_threads,
                                static_cast<cudaStream_t>(cuda_stream)));
     return AVSG_OK;

@@ -63,8 +63,8 @@ struct S1Params {
     uint32_t* qword;             // paper-literal mode: packed metadata words [num_tables][S], else null
     uint32_t probe_retries, hash_a1, hash_a2;   // paper-literal mode: R, a1, a2
     unsigned long long* t_range = nullptr;      // timing on: [0] earliest block start, [1] latest block end (ns)
-    // overlapped Stage Two (null otherwise): ready[g] counts the tables whose token g is placed, over all calls;
-    // tcount[ti * n_q + g] = misses of token g of the ti-th table of the call
+    // overlapped Stage Two (null otherwise): ready[g] counts the tables of this call whose token g is placed (the
+    // transfer kernel zeroes it again); tcount[ti * n_q + g] = misses of token g of the ti-th table of the call
     unsigned long long* ready = nullptr;
     uint32_t*           tcount = nullptr;
     uint32_t table_id[S1_MAX_TABLES];
@@ -89,9 +89,10 @@ struct XferOverlapParams {       // Stage Two that starts on token g's misses wh
     const int2*    miss_list;
     uint32_t*      status;
     const uint32_t* tcount;      // [n][n_q]
-    const unsigned long long* ready;             // [OVERLAP_MAX_TOKENS]
-    unsigned long long target[OVERLAP_MAX_TOKENS];   // value of ready[g] once every table of this call has token g placed
+    unsigned long long* ready;   // [OVERLAP_MAX_TOKENS] tables that have placed token g; zero between calls
+    uint32_t*      done;         // blocks of this grid that are through; zero between calls
     uint32_t n, n_q, list_stride, row_bytes, S;
+    uint32_t expect;             // value ready[g] reaches: n, or more than that for the wait-limit diagnostic
     unsigned long long* t_range = nullptr;
 };
 

@@ -166,7 +166,9 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_kernel(const __grid_con
 // places token g+1.  Every Stage One block is resident before this grid starts, so it always makes progress
 // without this grid's help; if a wait still runs out the block sets ST_WAIT_TIMEOUT and stops copying.
 // Before leaving, every block waits for the completion of the Stage One grid, so that the completion of
-// this grid implies it.  All reads of data written by the running Stage One go to L2 (ld.cg / acquire).
+// this grid implies it, and the last block through zeroes the counters for the next call: the kernel
+// arguments hold nothing that changes from call to call, so a captured call can be replayed.  All reads of
+// data written by the running Stage One go to L2 (ld.cg / acquire).
 __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __grid_constant__ XferOverlapParams p)
 {
     __shared__ uint32_t s_pref[S1_MAX_TABLES + 1];
@@ -190,7 +192,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __
             for (uint32_t spin = 0; spin < OVERLAP_SPIN_LIMIT; ++spin) {
                 unsigned long long v;
                 asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p.ready + g) : "memory");
-                if (v >= p.target[g]) { ok = 1; break; }
+                if (v >= p.expect) { ok = 1; break; }
                 __nanosleep(64);
             }
             if (!ok) atomicOr(p.status, ST_WAIT_TIMEOUT);
@@ -252,6 +254,17 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __
         if (tid == 0) atomicMax(p.t_range + 1, global_ns());
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    // Every block that arrives here has read the counters for the last time; the last one zeroes them.
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        if (atomicAdd(p.done, 1u) == gridDim.x - 1u) {
+            for (uint32_t g = 0; g < p.n_q; ++g) p.ready[g] = 0ull;
+            *p.done = 0u;
+            __threadfence();
+        }
+    }
 }
 
 // Comparator S2 (App. D, Eq. 14): the n * N_q * K selected positions of the call are flattened and cut into
