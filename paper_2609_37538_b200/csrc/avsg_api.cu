@@ -5,6 +5,8 @@
 #include <string.h>
 #include <vector>
 
+#include <cuda.h>          // types of the one driver entry point fetched at run time (nothing links libcuda)
+
 #include "avsg.h"
 #include "avsg_kernels.cuh"
 
@@ -23,7 +25,8 @@ struct avsg_ctx {
     uint8_t* d_buffer = nullptr;
     TableStats* d_stats = nullptr;
     unsigned long long* d_ready = nullptr;         // overlapped Stage Two: per-token counters [OVERLAP_MAX_TOKENS],
-                                                   //   then one word counting the transfer blocks that are through
+                                                   //   one word counting the transfer blocks that are through,
+                                                   //   one word with the sequence number of the last host-buffer call
     uint32_t* d_tcount = nullptr;                  //   and per-(table of the call, token) miss counts
     unsigned long long* d_trange = nullptr;        // [4] grid spans of the last timed call, then [4] their initial values
     unsigned long long* d_trange_init = nullptr;
@@ -51,6 +54,11 @@ struct avsg_ctx {
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
     // avsg_step_host: the outputs go back on a side stream while Stage Two runs
     cudaStream_t side = nullptr;
+    // cuStreamWaitValue64, when driver and device offer it: in the overlapped mode the output download of a call
+    // with host buffers waits for the sequence number Stage One writes once all its outputs exist, instead of for
+    // an event between the two grids (which would run them one after the other)
+    CUresult (*wait_value64)(CUstream, CUdeviceptr, cuuint64_t, unsigned int) = nullptr;
+    unsigned long long host_seq = 0;               // calls with host buffers issued in that mode so far
     cudaEvent_t ev_outputs_ready = nullptr, ev_outputs_copied = nullptr, ev_ids_ready = nullptr;
     uint64_t last_rows = 0;
 };
@@ -199,6 +207,8 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
     if (mode == AVSG_XFER_SM_OVERLAP &&
         (n > (uint32_t)S1_MAX_TABLES || n_q > (uint32_t)OVERLAP_MAX_TOKENS || c->cfg.index_mode == AVSG_INDEX_PAPER))
         mode = AVSG_XFER_SM_BALANCED;
+    // host buffers in the overlapped mode: no event between the two grids, the download waits for a sequence number
+    const bool wait_on_sequence = host_io && mode == AVSG_XFER_SM_OVERLAP && c->wait_value64 != nullptr;
     // the position-level comparator reads the hit mask: use the library's own buffer if the caller wants none
     if (mode == AVSG_XFER_POSITION_LEVEL && !hit) hit = c->d_hit_stage;
     if (c->timing) {
@@ -234,6 +244,9 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
             p.qword = c->d_q; p.probe_retries = c->cfg.probe_retries; p.hash_a1 = c->cfg.hash_a1; p.hash_a2 = c->cfg.hash_a2;
             p.t_range = c->timing ? c->d_trange : nullptr;
             if (mode == AVSG_XFER_SM_OVERLAP) { p.ready = c->d_ready; p.tcount = c->d_tcount; }
+            if (wait_on_sequence) {
+                p.done_seq = c->d_ready + OVERLAP_MAX_TOKENS + 1; p.host_seq = c->host_seq + 1; p.expect = n;
+            }
             for (uint32_t i = 0; i < cnt; ++i) {
                 p.table_id[i] = a->table_ids[first + i];
                 p.verified_len[i] = a->verified_len[first + i];
@@ -256,7 +269,7 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         CU(cudaEventRecord(c->ev_outputs_copied, c->side));
         return AVSG_OK;
     };
-    if (host_io) {
+    if (host_io && !wait_on_sequence) {
         CU(cudaEventRecord(c->ev_outputs_ready, stream));
         CU(cudaStreamWaitEvent(c->side, c->ev_outputs_ready, 0));
         if ((rc = download_outputs()) != AVSG_OK) return rc;
@@ -278,6 +291,13 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         x.expect = n;
         x.t_range = c->timing ? c->d_trange + 2 : nullptr;
         CU(launch_transfer_overlap(x, c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count, c->xfer_threads, stream));
+        if (wait_on_sequence) {
+            c->host_seq += 1;
+            if (c->wait_value64(c->side, reinterpret_cast<CUdeviceptr>(c->d_ready + OVERLAP_MAX_TOKENS + 1), c->host_seq,
+                                CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
+                return AVSG_ECUDA;
+            if ((rc = download_outputs()) != AVSG_OK) return rc;
+        }
     } else {
         XferParams x;
         x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
@@ -356,7 +376,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaMalloc(&c->d_buffer, T * S * cfg->row_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_stats, T * sizeof(TableStats)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_trange, 8 * sizeof(unsigned long long)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->d_ready, (OVERLAP_MAX_TOKENS + 1) * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_ready, (OVERLAP_MAX_TOKENS + 2) * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_tcount, (size_t)S1_MAX_TABLES * OVERLAP_MAX_TOKENS * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_list, n_ids * sizeof(int2)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_seg, T * sizeof(SegDesc)) == cudaSuccess;
@@ -377,6 +397,19 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaHostAlloc(&c->h_list, n_ids * sizeof(int2), cudaHostAllocDefault) == cudaSuccess;
     for (auto& e : c->ev) ok = ok && cudaEventCreate(&e) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
+    {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult found = cudaDriverEntryPointSymbolNotFound;
+        int can64 = 0;
+        // attribute 122 of the driver's numbering (the runtime's enum does not name it): 64-bit stream memory operations
+        if (cudaGetDriverEntryPoint("cuStreamWaitValue64", &fn, cudaEnableDefault, &found) == cudaSuccess &&
+            found == cudaDriverEntryPointSuccess &&
+            cudaDeviceGetAttribute(&can64, static_cast<cudaDeviceAttr>(CU_DEVICE_ATTRIBUTE_CAN_USE_64_BIT_STREAM_MEM_OPS),
+                                   cfg->device) == cudaSuccess && can64)
+            c->wait_value64 = reinterpret_cast<CUresult (*)(CUstream, CUdeviceptr, cuuint64_t, unsigned int)>(fn);
+        else
+            cudaGetLastError();
+    }
     ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_ready, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_outputs_copied, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_ids_ready, cudaEventDisableTiming) == cudaSuccess;
@@ -385,7 +418,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
         const unsigned long long never = ~0ull, init[8] = {never, 0, never, 0, never, 0, never, 0};
         c->d_trange_init = c->d_trange + 4;
         if (cudaMemcpy(c->d_trange, init, sizeof(init), cudaMemcpyHostToDevice) != cudaSuccess ||
-            cudaMemset(c->d_ready, 0, (OVERLAP_MAX_TOKENS + 1) * sizeof(unsigned long long)) != cudaSuccess) {
+            cudaMemset(c->d_ready, 0, (OVERLAP_MAX_TOKENS + 2) * sizeof(unsigned long long)) != cudaSuccess) {
             free_all(c); delete c; return AVSG_ECUDA;
         }
     }
@@ -503,7 +536,7 @@ int avsg_clear_status(avsg_ctx* c)
     CU(cudaDeviceSynchronize());
     CU(cudaMemset(c->d_status, 0, sizeof(uint32_t)));
     // a transfer kernel that gave up may have left the per-token counters of the overlapped mode raised
-    CU(cudaMemset(c->d_ready, 0, (OVERLAP_MAX_TOKENS + 1) * sizeof(unsigned long long)));
+    CU(cudaMemset(c->d_ready, 0, (OVERLAP_MAX_TOKENS + 1) * sizeof(unsigned long long)));    // not the sequence word
     return AVSG_OK;
 }
 

@@ -67,6 +67,11 @@ struct S1Params {
     // transfer kernel zeroes it again); tcount[ti * n_q + g] = misses of token g of the ti-th table of the call
     unsigned long long* ready = nullptr;
     uint32_t*           tcount = nullptr;
+    // calls with host buffers in that mode (null otherwise): the table that places the call's last token last
+    // writes the call's sequence number to *done_seq, which the output download waits for
+    unsigned long long* done_seq = nullptr;
+    unsigned long long  host_seq = 0;
+    uint32_t            expect = 0;             // tables of the call
     uint32_t table_id[S1_MAX_TABLES];
     int32_t  verified_len[S1_MAX_TABLES];
     uint64_t kv_base[S1_MAX_TABLES];

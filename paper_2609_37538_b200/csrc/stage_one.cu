@@ -356,7 +356,12 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
         __syncthreads();
         if (tid == 0) {
             __threadfence();
-            atomicAdd(p.ready + g, 1ull);
+            const unsigned long long before = atomicAdd(p.ready + g, 1ull);
+            if (p.done_seq && g + 1 == p.n_q && before + 1ull == p.expect) {
+                // every table of the call has written its slot table, hit mask and miss counts
+                __threadfence();
+                *reinterpret_cast<volatile unsigned long long*>(p.done_seq) = p.host_seq;
+            }
         }
     };
 
