@@ -158,6 +158,19 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_kernel(const __grid_con
     }
 }
 
+// Called once per block after its last look at the per-token counters (or when it gave up).  The last block to
+// call it zeroes the counters for the next call - Stage One raised them for the last time before the last token's
+// wait could end - early and off the critical path.  The kernel arguments hold nothing that changes from call to
+// call, so a captured call can be replayed.
+__device__ __forceinline__ void retire_block(const XferOverlapParams& p)
+{
+    if (atomicAdd(p.done, 1u) == gridDim.x - 1u) {
+        for (uint32_t k = 0; k < p.n_q; ++k) p.ready[k] = 0ull;
+        *p.done = 0u;
+        __threadfence();
+    }
+}
+
 // Stage Two that overlaps Stage One (the latency-hiding direction of App. G).  The grid is launched with
 // programmatic stream serialization and does NOT wait for Stage One to complete: its blocks become resident
 // once every Stage One block has started, then wait - with a bound - until all tables of the call have
@@ -166,9 +179,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_kernel(const __grid_con
 // places token g+1.  Every Stage One block is resident before this grid starts, so it always makes progress
 // without this grid's help; if a wait still runs out the block sets ST_WAIT_TIMEOUT and stops copying.
 // Before leaving, every block waits for the completion of the Stage One grid, so that the completion of
-// this grid implies it, and the last block through zeroes the counters for the next call: the kernel
-// arguments hold nothing that changes from call to call, so a captured call can be replayed.  All reads of
-// data written by the running Stage One go to L2 (ld.cg / acquire).
+// this grid implies it.  All reads of data written by the running Stage One go to L2 (ld.cg / acquire).
 __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __grid_constant__ XferOverlapParams p)
 {
     __shared__ uint32_t s_pref[S1_MAX_TABLES + 1];
@@ -197,9 +208,11 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __
             }
             if (!ok) atomicOr(p.status, ST_WAIT_TIMEOUT);
             s_ok = ok;
+            if (!ok) retire_block(p);
         }
         __syncthreads();
         if (!s_ok) break;                                          // same decision in every thread
+        if (g + 1 == p.n_q && tid == nt - 1) retire_block(p);      // beside the copy, not in front of it
         if (g == 0)                                                // the bases are published with token 0
             for (uint32_t i = tid; i < n; i += nt) {
                 s_src[i] = __ldcg(&p.seg[i].src_base);
@@ -254,17 +267,6 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __
         if (tid == 0) atomicMax(p.t_range + 1, global_ns());
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
-
-    // Every block that arrives here has read the counters for the last time; the last one zeroes them.
-    __syncthreads();
-    if (tid == 0) {
-        __threadfence();
-        if (atomicAdd(p.done, 1u) == gridDim.x - 1u) {
-            for (uint32_t g = 0; g < p.n_q; ++g) p.ready[g] = 0ull;
-            *p.done = 0u;
-            __threadfence();
-        }
-    }
 }
 
 // Comparator S2 (App. D, Eq. 14): the n * N_q * K selected positions of the call are flattened and cut into
