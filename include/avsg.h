@@ -122,6 +122,11 @@ typedef struct {
                                       -1 for padding                                     */
     uint8_t        *hit;           /* DEVICE out [n][n_tokens][topk] 1 = hit, or NULL    */
     int32_t        *miss_count;    /* DEVICE out [n][n_tokens] n_g per token, or NULL    */
+    const int32_t  *verified_len_dev; /* DEVICE [n] or NULL.  When set it replaces
+                                      verified_len (which may then be NULL): the kernel
+                                      reads N when it runs, so that a call captured in a
+                                      CUDA graph follows a sequence that grows between
+                                      replays                                            */
 } avsg_step_args;
 
 typedef struct {

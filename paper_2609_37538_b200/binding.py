@@ -42,7 +42,7 @@ class AvsgStepArgs(ctypes.Structure):
     _fields_ = [("n", ctypes.c_uint32), ("table_ids", ctypes.c_void_p), ("n_tokens", ctypes.c_uint32),
                 ("topk", ctypes.c_uint32), ("indices", ctypes.c_void_p), ("kv_base", ctypes.c_void_p),
                 ("row_stride", ctypes.c_void_p), ("verified_len", ctypes.c_void_p), ("slots", ctypes.c_void_p),
-                ("hit", ctypes.c_void_p), ("miss_count", ctypes.c_void_p)]
+                ("hit", ctypes.c_void_p), ("miss_count", ctypes.c_void_p), ("verified_len_dev", ctypes.c_void_p)]
 
 
 class AvsgStats(ctypes.Structure):
@@ -181,9 +181,15 @@ class PreparedCall:
 
     def run(self, indices, verified_len: Sequence[int], slots, hit=None, miss_count=None, stream=None,
             host: bool = False) -> None:
-        """indices / slots / hit / miss_count: tensors (device, or pinned host when host=True) or addresses."""
-        self._vlen[:] = [int(v) for v in verified_len]
+        """indices / slots / hit / miss_count: tensors (device, or pinned host when host=True) or addresses.
+        verified_len: a sequence of n ints, or an int32 CUDA tensor [n] that the kernel reads when it runs
+        (what a call captured in a CUDA graph needs when the sequences grow between replays)."""
         a = self.args
+        if hasattr(verified_len, "data_ptr"):
+            a.verified_len_dev = verified_len.data_ptr()
+        else:
+            a.verified_len_dev = None
+            self._vlen[:] = [int(v) for v in verified_len]
         a.indices, a.slots = _addr(indices), _addr(slots)
         a.hit = _addr(hit) if hit is not None else None
         a.miss_count = _addr(miss_count) if miss_count is not None else None

@@ -129,7 +129,8 @@ int check_args(avsg_ctx* c, const avsg_step_args* a)
 {
     if (!c || !a) return AVSG_EINVAL;
     if (a->n == 0 || a->n > c->cfg.num_tables || a->n > (uint32_t)XFER_MAX_SEG) return AVSG_EINVAL;
-    if (!a->table_ids || !a->indices || !a->kv_base || !a->verified_len || !a->slots) return AVSG_EINVAL;
+    if (!a->table_ids || !a->indices || !a->kv_base || !(a->verified_len || a->verified_len_dev) || !a->slots)
+        return AVSG_EINVAL;
     if (a->n_tokens == 0 || a->n_tokens > c->cfg.max_tokens || a->topk == 0 || a->topk > c->cfg.max_topk)
         return AVSG_EINVAL;
     if ((uint64_t)a->n_tokens * a->topk > c->cfg.buffer_slots) return AVSG_ECAPACITY;      // Eq. 7
@@ -243,13 +244,14 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
             p.where = c->d_where; p.max_context = c->cfg.max_context;
             p.qword = c->d_q; p.probe_retries = c->cfg.probe_retries; p.hash_a1 = c->cfg.hash_a1; p.hash_a2 = c->cfg.hash_a2;
             p.t_range = c->timing ? c->d_trange : nullptr;
+            p.verified_len_dev = a->verified_len_dev;
             if (mode == AVSG_XFER_SM_OVERLAP) { p.ready = c->d_ready; p.tcount = c->d_tcount; }
             if (wait_on_sequence) {
                 p.done_seq = c->d_ready + OVERLAP_MAX_TOKENS + 1; p.host_seq = c->host_seq + 1; p.expect = n;
             }
             for (uint32_t i = 0; i < cnt; ++i) {
                 p.table_id[i] = a->table_ids[first + i];
-                p.verified_len[i] = a->verified_len[first + i];
+                p.verified_len[i] = a->verified_len ? a->verified_len[first + i] : 0;
                 if ((rc = resolve_kv(c, p.table_id[i], a->kv_base[first + i], &p.kv_base[i])) != AVSG_OK) return rc;
                 p.kv_stride[i] = a->row_stride ? a->row_stride[first + i] : c->cfg.row_bytes;
             }

@@ -72,6 +72,7 @@ struct S1Params {
     unsigned long long* done_seq = nullptr;
     unsigned long long  host_seq = 0;
     uint32_t            expect = 0;             // tables of the call
+    const int32_t* verified_len_dev = nullptr;  // [n] of the call: read instead of verified_len[] when set
     uint32_t table_id[S1_MAX_TABLES];
     int32_t  verified_len[S1_MAX_TABLES];
     uint64_t kv_base[S1_MAX_TABLES];

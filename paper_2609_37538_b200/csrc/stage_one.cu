@@ -503,7 +503,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
     }
 
     // ---- write the table back; speculative entries (id >= N) become empty (Alg. 4) ----
-    const int32_t N = p.verified_len[blockIdx.x];
+    const int32_t N = p.verified_len_dev ? __ldg(p.verified_len_dev + ti) : p.verified_len[blockIdx.x];
     if (own) {
         if ((spt & 3u) == 0) {
             for (uint32_t q = 0; q < spt / 4; ++q) {
@@ -785,7 +785,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_paper_kernel(const __g
     }
 
     // ---- write back; speculative entries (id >= N) become empty ----
-    const int32_t N = p.verified_len[blockIdx.x];
+    const int32_t N = p.verified_len_dev ? __ldg(p.verified_len_dev + ti) : p.verified_len[blockIdx.x];
     if (own)
         for (uint32_t k = 0; k < spt; ++k) {
             const int32_t v = s_c[j0 + k];

@@ -26,7 +26,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(avsg.AvsgConfig) == 52
-    assert ctypes.sizeof(avsg.AvsgStepArgs) == 80
+    assert ctypes.sizeof(avsg.AvsgStepArgs) == 88
     assert ctypes.sizeof(avsg.AvsgStats) == 88
 
 

@@ -206,13 +206,15 @@ def test_overlap_mode_limits(avsg, n, n_q, K, S):
 
 @pytest.mark.parametrize("mode_name", ["XFER_SM_BALANCED", "XFER_SM_OVERLAP"])
 def test_a_captured_call_can_be_replayed(avsg, mode_name):
-    """One avsg_step call captured in a CUDA graph and replayed with new ids in the same input tensor: the kernel
-    arguments hold nothing that changes from call to call (the verified length is constant in this trace)."""
+    """One avsg_step call captured in a CUDA graph and replayed for the following iterations: the ids and the
+    verified lengths (which grow every iteration here) sit in device tensors that are refreshed in place, and the
+    kernel arguments hold nothing else that changes from call to call."""
     import torch
     n, n_q, K, S, T, rb, ctxlen = 4, 2, 256, 1024, 12, 656, 20000
-    cfgs = [tr.TraceConfig(seed=11, table=i, topk=K, n_q=n_q, n_iters=T, context=ctxlen, beta=(18, 2), p_recent=0.5,
-                           recent_window=2048) for i in range(n)]
+    cfgs = [tr.TraceConfig(seed=11, table=i, topk=K, n_q=n_q, n_iters=T, context=ctxlen, ctx_growth=True,
+                           beta=(18, 2), p_recent=0.5, recent_window=2048) for i in range(n)]
     traces = [tr.generate(c) for c in cfgs]
+    assert traces[0][1][0] != traces[0][1][1]                 # the verified length does change
     kv = []
     for i in range(n):
         b = avsg.pinned_empty(ctxlen * rb)
@@ -223,29 +225,33 @@ def test_a_captured_call_can_be_replayed(avsg, mode_name):
     orc = [OracleTable(S, rb, 16) for _ in range(n)]
     call = ctx.prepare(list(range(n)), kv, n_q, K, None)
     X = torch.empty((n, n_q, K), dtype=torch.int32, device="cuda")
+    Nd = torch.empty(n, dtype=torch.int32, device="cuda")
     slots = torch.empty_like(X)
     mc = torch.empty((n, n_q), dtype=torch.int32, device="cuda")
-    N = [ctxlen] * n
 
     def load(t):
         X.copy_(torch.from_numpy(np.stack([traces[i][0][t] for i in range(n)])))
+        Nd.copy_(torch.tensor([int(traces[i][1][t]) for i in range(n)], dtype=torch.int32))
         torch.cuda.synchronize()
 
     def check(t):
         torch.cuda.synchronize()
         for i in range(n):
-            r = orc[i].step(traces[i][0][t], N[i], kv[i].numpy(), rb)
+            r = orc[i].step(traces[i][0][t], int(traces[i][1][t]), kv[i].numpy(), rb)
             assert (slots[i].cpu().numpy() == r.O).all() and (mc[i].cpu().numpy() == r.n).all(), (t, i)
             assert (ctx.buffer(i).cpu().numpy() == orc[i].rows()).all(), (t, i)
+            tok, life = ctx.export_state(i)
+            c, l = orc[i].export_state()
+            assert (tok == c).all() and (life == l).all(), (t, i)
 
     side = torch.cuda.Stream()
     load(0)
     with torch.cuda.stream(side):
-        call.run(X, N, slots, None, mc, side)              # eager first call: resolves and caches the host pointers
+        call.run(X, Nd, slots, None, mc, side)             # eager first call: resolves and caches the host pointers
     check(0)
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph, stream=side):
-        call.run(X, N, slots, None, mc, torch.cuda.current_stream())
+        call.run(X, Nd, slots, None, mc, torch.cuda.current_stream())
     for t in range(1, T):
         load(t)
         graph.replay()
