@@ -205,8 +205,7 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         miss_count = a->miss_count ? c->d_mc_stage : nullptr;
     }
     uint32_t mode = c->cfg.transfer_mode;
-    if (mode == AVSG_XFER_SM_OVERLAP &&
-        (n > (uint32_t)S1_MAX_TABLES || n_q > (uint32_t)OVERLAP_MAX_TOKENS || c->cfg.index_mode == AVSG_INDEX_PAPER))
+    if (mode == AVSG_XFER_SM_OVERLAP && (n > (uint32_t)S1_MAX_TABLES || n_q > (uint32_t)OVERLAP_MAX_TOKENS))
         mode = AVSG_XFER_SM_BALANCED;
     // host buffers in the overlapped mode: no event between the two grids, the download waits for a sequence number
     const bool wait_on_sequence = host_io && mode == AVSG_XFER_SM_OVERLAP && c->wait_value64 != nullptr;

@@ -34,7 +34,7 @@
 // deterministic).
 //
 // When Stage Two overlaps Stage One (S1Params::ready set), the block announces
-// every token as soon as its misses are placed: see `publish` in the kernel.
+// every token as soon as its misses are placed: see publish_token().
 #include "avsg_kernels.cuh"
 
 namespace avsg {
@@ -241,6 +241,38 @@ __device__ __forceinline__ void count_lifetimes(uint32_t w0, uint32_t w1, uint32
     }
 }
 
+// Overlapped Stage Two only (p.ready set): tells the transfer kernel, which is already resident, that token g of
+// this table is placed - `count` more entries of the table's miss list are final.  Called by every thread of the
+// block: the block meets after its list writes; one thread then fences (the barrier makes the fence cover the whole
+// block's earlier writes, as in a grid-wide barrier) and raises the counter of token g.
+__device__ __forceinline__ void publish_token(const S1Params& p, uint32_t ti, uint32_t table, uint32_t g, uint32_t count)
+{
+    if (!p.ready) return;
+    const uint32_t tid = threadIdx.x;
+    if (tid == 0) {
+        p.tcount[(size_t)ti * p.n_q + g] = count;
+        if (g == 0) {
+            SegDesc sd;
+            sd.src_base = p.kv_base[blockIdx.x];
+            sd.src_stride = p.kv_stride[blockIdx.x];
+            sd.dst_base = reinterpret_cast<uint64_t>(p.buffer + (size_t)table * p.S * p.row_bytes);
+            sd.count = 0;
+            sd.pad = 0;
+            p.seg[ti] = sd;
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        const unsigned long long before = atomicAdd(p.ready + g, 1ull);
+        if (p.done_seq && g + 1 == p.n_q && before + 1ull == p.expect) {
+            // every table of the call has written its slot table, hit mask and miss counts
+            __threadfence();
+            *reinterpret_cast<volatile unsigned long long*>(p.done_seq) = p.host_seq;
+        }
+    }
+}
+
 template <bool DIRECT>
 __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_constant__ S1Params p)
 {
@@ -335,35 +367,6 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
     uint32_t list_off = 0, sum_valid = 0, sum_miss = 0, sum_decay = 0;
     int2* list = p.miss_list + (size_t)ti * p.list_stride;
 
-    // Overlapped Stage Two only (p.ready set): tells the transfer kernel, which is already resident, that token
-    // g of this table is placed - `count` more entries of the table's miss list are final.  The block meets
-    // after its list writes; one thread then fences (the barrier makes the fence cover the whole block's
-    // earlier writes, as in a grid-wide barrier) and raises the counter of token g.
-    auto publish = [&](uint32_t g, uint32_t count) {
-        if (!p.ready) return;
-        if (tid == 0) {
-            p.tcount[(size_t)ti * p.n_q + g] = count;
-            if (g == 0) {
-                SegDesc sd;
-                sd.src_base = p.kv_base[blockIdx.x];
-                sd.src_stride = p.kv_stride[blockIdx.x];
-                sd.dst_base = reinterpret_cast<uint64_t>(p.buffer + (size_t)table * S * p.row_bytes);
-                sd.count = 0;
-                sd.pad = 0;
-                p.seg[ti] = sd;
-            }
-        }
-        __syncthreads();
-        if (tid == 0) {
-            __threadfence();
-            const unsigned long long before = atomicAdd(p.ready + g, 1ull);
-            if (p.done_seq && g + 1 == p.n_q && before + 1ull == p.expect) {
-                // every table of the call has written its slot table, hit mask and miss counts
-                __threadfence();
-                *reinterpret_cast<volatile unsigned long long*>(p.done_seq) = p.host_seq;
-            }
-        }
-    };
 
     for (uint32_t g = 0; g < p.n_q; ++g) {
         const size_t row = ((size_t)ti * p.n_q + g) * K;
@@ -425,7 +428,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
         // the next token's ids travel while this token's misses are placed
         if (g + 1 < p.n_q) load_ids(p.indices + row + K, i0, ipt, K, xs);
         if (tid == 0 && p.miss_count) p.miss_count[(size_t)ti * p.n_q + g] = (int32_t)n_g;
-        if (n_g == 0) { __syncthreads(); publish(g, 0); continue; }
+        if (n_g == 0) { __syncthreads(); publish_token(p, ti, table, g, 0); continue; }
         __syncthreads();
 
         // ---- Pass 3: CollectDead; if fewer than n_g slots are dead, decay until enough are ----
@@ -499,7 +502,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
             __syncthreads();
             fill_bound = *s_fill;
         }
-        publish(g, n_take);
+        publish_token(p, ti, table, g, n_take);
     }
 
     // ---- write the table back; speculative entries (id >= N) become empty (Alg. 4) ----
@@ -700,7 +703,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_paper_kernel(const __g
         }
         if (g + 1 < p.n_q) load_ids(p.indices + row + K, i0, ipt, K, xs);
         if (tid == 0 && p.miss_count) p.miss_count[(size_t)ti * p.n_q + g] = (int32_t)n_g;
-        if (n_g == 0) { __syncthreads(); continue; }
+        if (n_g == 0) { __syncthreads(); publish_token(p, ti, table, g, 0); continue; }
         __syncthreads();
 
         // ---- CollectDead / decay until n_g slots are dead ----
@@ -782,6 +785,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_paper_kernel(const __g
         list_off += n_take;
         sum_decay += d;
         __syncthreads();
+        publish_token(p, ti, table, g, n_take);
     }
 
     // ---- write back; speculative entries (id >= N) become empty ----

@@ -142,7 +142,7 @@ def test_overlap_mode_host_io_strides_geometries_and_fallbacks(avsg):
     _parity(w, mode=avsg.XFER_SM_OVERLAP, row_stride=1024, index_mode=avsg.INDEX_DIRECT)
     for geo in [(1, 32), (7, 1024), (600, 256)]:
         _parity(w, mode=avsg.XFER_SM_OVERLAP, xfer_geometry=geo)
-    # more tables than one Stage One launch takes, and the paper-literal index, run as the balanced mode
+    # more tables than one Stage One launch takes run as the balanced mode
     many = tr.workload("C5", topk=64, buffer_slots=128, n_iters=6, requests=300, ctx_lo=256, ctx_hi=2048)
     _parity(many, mode=avsg.XFER_SM_OVERLAP, buffer_every=3)
 
@@ -512,7 +512,7 @@ def test_degenerate_selections(avsg, index_mode):
 
 
 # ---- the paper-literal (lossy) Hash-State mode against its own oracle ---------------------------------------------
-def _literal_parity(avsg, w, n_iters=None, R=3):
+def _literal_parity(avsg, w, n_iters=None, R=3, mode=0):
     import torch
     from oracle import LiteralOracleTable
     from harness import HostKV
@@ -520,7 +520,8 @@ def _literal_parity(avsg, w, n_iters=None, R=3):
     traces = {ti: tr.generate(w.tables[ti]) for ti in ids}
     kv = HostKV(w, ids)
     ctx = avsg.Context(num_tables=len(ids), buffer_slots=w.buffer_slots, row_bytes=w.row_bytes, max_topk=w.topk,
-                       max_tokens=w.n_q, max_lifetime=w.max_lifetime, index_mode=avsg.INDEX_PAPER, probe_retries=R)
+                       max_tokens=w.n_q, max_lifetime=w.max_lifetime, index_mode=avsg.INDEX_PAPER, probe_retries=R,
+                       transfer_mode=mode)
     orc = {ti: LiteralOracleTable(w.buffer_slots, w.row_bytes, w.max_lifetime, R=R) for ti in ids}
     T = w.n_iters if n_iters is None else n_iters
     for t in range(T):
@@ -551,6 +552,11 @@ def test_paper_literal_mode_full_c2_and_small_c3(avsg):
     st = _literal_parity(avsg, tr.workload("C2"), n_iters=64)
     assert st["hits"] / (st["hits"] + st["misses"]) < 0.91          # lossy: below the exact index's 92.4 %
     _literal_parity(avsg, tr.workload("C3", requests=6, layers=2, n_iters=10))
+
+
+def test_paper_literal_mode_with_overlapped_stage_two(avsg):
+    _literal_parity(avsg, tr.workload("C2"), n_iters=32, mode=avsg.XFER_SM_OVERLAP)
+    _literal_parity(avsg, tr.workload("C3", requests=6, layers=2, n_iters=10), mode=avsg.XFER_SM_OVERLAP)
 
 
 @pytest.mark.parametrize("kw,R", [
