@@ -49,6 +49,18 @@ def test_error_strings_and_argument_errors_need_no_gpu():
     assert lib.avsg_create(ctypes.byref(bad), ctypes.byref(h)) == avsg.EINVAL
     assert lib.avsg_step(None, None, None) == avsg.EINVAL
     assert lib.avsg_destroy(None) == avsg.EINVAL
+    bad = avsg.AvsgConfig(1, 1024, 656, 16, 1, 16, 6, 0)            # transfer mode beyond the last one
+    assert lib.avsg_create(ctypes.byref(bad), ctypes.byref(h)) == avsg.EINVAL
+    bad = avsg.AvsgConfig(1, 1024, 656, 16, 1, 16, 0, 0, avsg.INDEX_DIRECT, 0)   # direct index without max_context
+    assert lib.avsg_create(ctypes.byref(bad), ctypes.byref(h)) == avsg.EINVAL
+    st = avsg.AvsgStats()
+    for call in (lambda: lib.avsg_stats(None, ctypes.byref(st)), lambda: lib.avsg_table_stats(None, 0, ctypes.byref(st)),
+                 lambda: lib.avsg_sync_status(None, None), lambda: lib.avsg_clear_status(None),
+                 lambda: lib.avsg_probe_wait_limit(None, None), lambda: lib.avsg_set_transfer_mode(None, 0),
+                 lambda: lib.avsg_set_timing(None, 1), lambda: lib.avsg_set_transfer_geometry(None, 148, 256),
+                 lambda: lib.avsg_save_state(None, None), lambda: lib.avsg_restore_state(None, None),
+                 lambda: lib.avsg_reset(None, None, 0), lambda: lib.avsg_step_host(None, None, None)):
+        assert call() == avsg.EINVAL
 
 
 def test_product_sources_do_not_touch_the_oracle():
