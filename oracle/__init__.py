@@ -35,7 +35,9 @@ def _load():
     global _lib
     if _lib is not None:
         return _lib
-    lib = ctypes.CDLL(build_library())
+    # AVSG_ORACLE_LIB: another build of avsg_oracle.c to load instead (the test that checks that the pins catch
+    # deliberately broken copies of the oracle uses it)
+    lib = ctypes.CDLL(os.environ.get("AVSG_ORACLE_LIB") or build_library())
     vp, u32, i32, u64 = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_int32, ctypes.c_uint64
     lib.orc_create.argtypes, lib.orc_create.restype = [u32, u32, i32], vp
     lib.orc_destroy.argtypes, lib.orc_destroy.restype = [vp], None

@@ -40,6 +40,39 @@ def test_hand_worked_literal_example():
     assert r.xfer.tolist() == [[9, 3]]                                          # the resident id is fetched again
 
 
+def _reclaim_cases():
+    cases, cur = [], None
+    for line in open(os.path.join(GOLDEN, "literal_reclaim_examples.txt")):
+        line = line.split("#")[0].strip()
+        if not line:
+            continue
+        key, *vals = line.split()
+        if key == "case":
+            cur = {"name": vals[0], "steps": [], "buckets": []}
+            cases.append(cur)
+        elif key == "step":
+            cur["steps"].append([int(v) for v in vals])
+        elif key == "bucket":
+            cur["buckets"].append([int(v) for v in vals])
+        else:
+            cur[key] = [int(v) for v in vals]
+    return cases
+
+
+@pytest.mark.parametrize("case", _reclaim_cases(), ids=lambda c: c["name"])
+def test_hand_worked_reclamation_conditions(case):
+    S, m = 8, 3
+    t = LiteralOracleTable(S, 8, case["L"][0], R=1, a1=3, a2=5)
+    for ids in case["steps"]:
+        r = t.step(np.array(ids, dtype=np.int32)[None, :], 1000)
+    assert r.M[0].tolist() == case["expect_M"] and r.O[0].tolist() == case["expect_O"]
+    assert t.counters()["lost_mappings"] == case["expect_lost"][0]
+    _, q = t.export_state()
+    for h, slot, fp, invalid in case["buckets"]:
+        word = int(q[h])
+        assert (word & (S - 1), (word >> m) & ((1 << 20) - 1), (word >> 23) & 1) == (slot, fp, invalid), (h, hex(word))
+
+
 @pytest.mark.parametrize("seed", range(4))
 def test_literal_equals_exact_when_no_mapping_is_lost(seed):
     # few ids in a large table, no expiry within the trace: every id keeps its own bucket, so the bounded probe
