@@ -22,6 +22,17 @@ MUTATIONS = [
     ("misses are placed in reverse order", "for (uint32_t i = 0; i < K; ++i) {\n        if (x[i] < 0 || m[i]) continue;",
      "for (uint32_t i = K; i-- > 0;) {\n        if (x[i] < 0 || m[i]) continue;"),
     ("later tokens are pre-decayed too", "if (g == 0) decay_all(t);", "decay_all(t);"),
+    ("hits are refreshed after the allocation instead of before",
+     ["if (m[i]) t->life[o[i]] = t->L;", "    t->tokens++;\n    t->hits += valid"],
+     ["if (0) t->life[o[i]] = t->L;",
+      "    for (uint32_t i = 0; i < K; ++i) if (m[i]) t->life[o[i]] = t->L;\n    t->tokens++;\n    t->hits += valid"]),
+    ("padding counts as a miss", "if (x[i] >= 0) { valid++; n_g += 1 - (int32_t)m[i]; }",
+     "{ valid += x[i] >= 0; n_g += 1 - (int32_t)m[i]; }"),
+    ("Eq. 6 drops the remainder", "*end = *begin + q + (c < r ? 1 : 0);", "*end = *begin + q;"),
+    ("Eq. 13 ignores the remainder", "return B / C + (c < B % C ? 1u : 0u);", "return B / C;"),
+    ("Eq. 14 rounds the upper end up", "*end = (uint64_t)(c + 1) * n_positions / C;",
+     "*end = ((uint64_t)(c + 1) * n_positions + C - 1) / C;"),
+    ("transfer-all-K keeps a padding row", "if (X[p] < 0) { O[p] = -1; continue; }", "if (X[p] < 0) { O[p] = (int32_t)p; continue; }"),
 ]
 
 # the paper-literal Hash-State mode (Eq. 2-4, 8-11, Alg. 2), against its own pins
@@ -44,8 +55,10 @@ LITERAL_MUTATIONS = [
 def _run_pins(tmp_path, pins, label, old, new):
     text = open(SRC).read()
     if old is not None:
-        assert text.count(old) >= 1, "the line to change was not found"
-        text = text.replace(old, new, 1)          # the first occurrence is the exact oracle's (the literal mode follows it)
+        olds, news = (old, new) if isinstance(old, list) else ([old], [new])
+        for o, n in zip(olds, news):
+            assert text.count(o) >= 1, "the line to change was not found"
+            text = text.replace(o, n, 1)          # the first occurrence is the exact oracle's (the literal mode follows it)
     src, lib = tmp_path / "avsg_oracle.c", tmp_path / "libavsg_oracle_variant.so"
     src.write_text(text)
     subprocess.check_call(["gcc", "-O2", "-std=c99", "-fPIC", "-shared", "-o", str(lib), str(src)])

@@ -398,6 +398,18 @@ def test_all_k_comparator():
     assert O.ravel().tolist() == list(range(64))
     assert (t.rows() == kv.reshape(500, rb)[X.ravel()]).all()
     assert t.counters()["rows_copied"] == 64
+    # padding (negative ids) moves nothing and gets no slot; the other positions keep their slots g*K + i
+    t2 = OracleTable(64, rb, 16)
+    Xp = X.copy()
+    Xp[0, 5] = Xp[1, 31] = -1
+    O2 = t2.step_all_k(Xp, kv)
+    want = np.arange(64)
+    want[[5, 63]] = -1
+    assert O2.ravel().tolist() == want.tolist()
+    assert t2.counters()["rows_copied"] == 62
+    keep = want >= 0
+    assert (t2.rows()[keep] == kv.reshape(500, rb)[Xp.ravel()[keep]]).all()
+    assert not t2.rows()[~keep].any()                      # the two padded slots were never written
 
 
 # ----------------------------------------------------------------------------
