@@ -100,6 +100,8 @@ def test_padding_when_context_is_shorter_than_k(avsg):
     w = tr.workload("C5", topk=128, buffer_slots=256, n_iters=6, requests=4, ctx_lo=40, ctx_hi=100)
     r = _parity(w)
     assert r["gpu"]["hits"] + r["gpu"]["misses"] < 4 * 6 * 128
+    for mode in (avsg.XFER_ALL_K, avsg.XFER_POSITION_LEVEL, avsg.XFER_REQUEST_LEVEL, avsg.XFER_SM_OVERLAP):
+        _parity(w, mode=mode)                                # padded positions: slot -1, nothing moved, in every mode
 
 
 def test_strided_host_rows_and_host_io(avsg):
