@@ -69,8 +69,9 @@ extern "C" {
                                        resident while Stage One runs and starts on token
                                        g's misses, cut evenly over all SMs per token,
                                        while token g+1 is being placed.  Same results.
-                                       Calls with more than 128 tables or more than 8
-                                       tokens run as AVSG_XFER_SM_BALANCED               */
+                                       Calls with more than 1024 tables (128 with
+                                       AVSG_INDEX_PAPER) or more than 8 tokens run as
+                                       AVSG_XFER_SM_BALANCED                             */
 
 /* How Stage One finds the slot that holds an id (same results either way). */
 #define AVSG_INDEX_HASH   0u  /* open-addressing table in shared memory, rebuilt every step     */

@@ -28,6 +28,7 @@ struct avsg_ctx {
                                                    //   one word counting the transfer blocks that are through,
                                                    //   one word with the sequence number of the last host-buffer call
     uint32_t* d_tcount = nullptr;                  //   and per-(table of the call, token) miss counts
+    S1ParamsBig* big_args = nullptr;               // host: the large Stage One argument block, built in place per call
     unsigned long long* d_trange = nullptr;        // [4] grid spans of the last timed call, then [4] their initial values
     unsigned long long* d_trange_init = nullptr;
     int2* d_list = nullptr;
@@ -85,6 +86,7 @@ void free_all(avsg_ctx* c)
 {
     cudaFree(c->d_tok); cudaFree(c->d_life); cudaFree(c->d_buffer); cudaFree(c->d_stats); cudaFree(c->d_trange);
     cudaFree(c->d_ready); cudaFree(c->d_tcount);
+    delete c->big_args;
     cudaFree(c->d_list); cudaFree(c->d_seg); cudaFree(c->d_status); cudaFree(c->d_where); cudaFree(c->d_q); cudaFree(c->d_q_snap);
     cudaFree(c->d_tok_snap); cudaFree(c->d_life_snap);
     cudaFree(c->d_idx_stage); cudaFree(c->d_slots_stage); cudaFree(c->d_hit_stage); cudaFree(c->d_mc_stage);
@@ -205,8 +207,12 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         miss_count = a->miss_count ? c->d_mc_stage : nullptr;
     }
     uint32_t mode = c->cfg.transfer_mode;
-    if (mode == AVSG_XFER_SM_OVERLAP && (n > (uint32_t)S1_MAX_TABLES || n_q > (uint32_t)OVERLAP_MAX_TOKENS))
-        mode = AVSG_XFER_SM_BALANCED;
+    // tables per Stage One launch: the small argument block when it is enough (and for the kernels that only have
+    // that one), else the large one
+    const uint32_t chunk = (n <= (uint32_t)S1_MAX_TABLES || mode == AVSG_XFER_ALL_K || c->cfg.index_mode == AVSG_INDEX_PAPER)
+                               ? (uint32_t)S1_MAX_TABLES : (uint32_t)S1_BIG_TABLES;
+    if (mode == AVSG_XFER_SM_OVERLAP && (n > chunk || n_q > (uint32_t)OVERLAP_MAX_TOKENS))
+        mode = AVSG_XFER_SM_BALANCED;                  // the overlapped kernel pairs with ONE Stage One launch
     // host buffers in the overlapped mode: no event between the two grids, the download waits for a sequence number
     const bool wait_on_sequence = host_io && mode == AVSG_XFER_SM_OVERLAP && c->wait_value64 != nullptr;
     // the position-level comparator reads the hit mask: use the library's own buffer if the caller wants none
@@ -218,8 +224,37 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
     }
 
     c->call_kv_host.assign(a->kv_base, a->kv_base + n);
-    for (uint32_t first = 0; first < n; first += S1_MAX_TABLES) {
-        const uint32_t cnt = n - first < (uint32_t)S1_MAX_TABLES ? n - first : (uint32_t)S1_MAX_TABLES;
+    // Stage One for tables [first, first + cnt) of the call, with the small or the large argument block
+    auto stage_one = [&](auto& p, uint32_t first, uint32_t cnt) -> int {
+        p.tok = c->d_tok; p.life = c->d_life; p.buffer = c->d_buffer; p.stats = c->d_stats;
+        p.miss_list = c->d_list; p.seg = c->d_seg; p.status = c->d_status;
+        p.indices = indices; p.slots = slots; p.hit = hit; p.miss_count = miss_count;
+        p.S = c->cfg.buffer_slots; p.logH = c->logH; p.row_bytes = c->cfg.row_bytes;
+        p.K = K; p.n_q = n_q; p.L = (uint32_t)c->cfg.max_lifetime;
+        p.first = first; p.list_stride = c->list_stride;
+        p.where = c->d_where; p.max_context = c->cfg.max_context;
+        p.qword = c->d_q; p.probe_retries = c->cfg.probe_retries; p.hash_a1 = c->cfg.hash_a1; p.hash_a2 = c->cfg.hash_a2;
+        p.t_range = c->timing ? c->d_trange : nullptr;
+        p.verified_len_dev = a->verified_len_dev;
+        // (every field is assigned: the large block is re-used from call to call)
+        const bool overlap = mode == AVSG_XFER_SM_OVERLAP;
+        p.ready = overlap ? c->d_ready : nullptr;
+        p.tcount = overlap ? c->d_tcount : nullptr;
+        p.done_seq = wait_on_sequence ? c->d_ready + OVERLAP_MAX_TOKENS + 1 : nullptr;
+        p.host_seq = wait_on_sequence ? c->host_seq + 1 : 0;
+        p.expect = n;
+        for (uint32_t i = 0; i < cnt; ++i) {
+            p.table_id[i] = a->table_ids[first + i];
+            p.verified_len[i] = a->verified_len ? a->verified_len[first + i] : 0;
+            const int r = resolve_kv(c, p.table_id[i], a->kv_base[first + i], &p.kv_base[i]);
+            if (r != AVSG_OK) return r;
+            p.kv_stride[i] = a->row_stride ? a->row_stride[first + i] : c->cfg.row_bytes;
+        }
+        CU(launch_stage_one(p, cnt, stream));
+        return AVSG_OK;
+    };
+    for (uint32_t first = 0; first < n; first += chunk) {
+        const uint32_t cnt = n - first < chunk ? n - first : chunk;
         if (mode == AVSG_XFER_ALL_K) {
             AllKParams p;
             p.indices = indices; p.slots = slots; p.hit = hit; p.miss_count = miss_count;
@@ -232,29 +267,11 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
                 p.kv_stride[i] = a->row_stride ? a->row_stride[first + i] : c->cfg.row_bytes;
             }
             CU(launch_all_k_prepare(p, cnt, stream));
-        } else {
+        } else if (chunk == (uint32_t)S1_MAX_TABLES) {
             S1Params p;
-            p.tok = c->d_tok; p.life = c->d_life; p.buffer = c->d_buffer; p.stats = c->d_stats;
-            p.miss_list = c->d_list; p.seg = c->d_seg; p.status = c->d_status;
-            p.indices = indices; p.slots = slots; p.hit = hit; p.miss_count = miss_count;
-            p.S = c->cfg.buffer_slots; p.logH = c->logH; p.row_bytes = c->cfg.row_bytes;
-            p.K = K; p.n_q = n_q; p.L = (uint32_t)c->cfg.max_lifetime;
-            p.first = first; p.list_stride = c->list_stride;
-            p.where = c->d_where; p.max_context = c->cfg.max_context;
-            p.qword = c->d_q; p.probe_retries = c->cfg.probe_retries; p.hash_a1 = c->cfg.hash_a1; p.hash_a2 = c->cfg.hash_a2;
-            p.t_range = c->timing ? c->d_trange : nullptr;
-            p.verified_len_dev = a->verified_len_dev;
-            if (mode == AVSG_XFER_SM_OVERLAP) { p.ready = c->d_ready; p.tcount = c->d_tcount; }
-            if (wait_on_sequence) {
-                p.done_seq = c->d_ready + OVERLAP_MAX_TOKENS + 1; p.host_seq = c->host_seq + 1; p.expect = n;
-            }
-            for (uint32_t i = 0; i < cnt; ++i) {
-                p.table_id[i] = a->table_ids[first + i];
-                p.verified_len[i] = a->verified_len ? a->verified_len[first + i] : 0;
-                if ((rc = resolve_kv(c, p.table_id[i], a->kv_base[first + i], &p.kv_base[i])) != AVSG_OK) return rc;
-                p.kv_stride[i] = a->row_stride ? a->row_stride[first + i] : c->cfg.row_bytes;
-            }
-            CU(launch_stage_one(p, cnt, stream));
+            if ((rc = stage_one(p, first, cnt)) != AVSG_OK) return rc;
+        } else {
+            if ((rc = stage_one(*c->big_args, first, cnt)) != AVSG_OK) return rc;
         }
     }
     // (no event between the two grids in overlap mode: it would serialise them; ev[1] is recorded with ev[2])
@@ -378,7 +395,9 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaMalloc(&c->d_stats, T * sizeof(TableStats)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_trange, 8 * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_ready, (OVERLAP_MAX_TOKENS + 2) * sizeof(unsigned long long)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->d_tcount, (size_t)S1_MAX_TABLES * OVERLAP_MAX_TOKENS * sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_tcount, (size_t)OVERLAP_MAX_TABLES * OVERLAP_MAX_TOKENS * sizeof(uint32_t)) == cudaSuccess;
+    c->big_args = new (std::nothrow) S1ParamsBig();
+    ok = ok && c->big_args != nullptr;
     ok = ok && cudaMalloc(&c->d_list, n_ids * sizeof(int2)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_seg, T * sizeof(SegDesc)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_status, 256) == cudaSuccess;

@@ -38,12 +38,15 @@ struct TableStats {
     unsigned long long steps, tokens, hits, misses, rows, extra_decays;
 };
 
-constexpr int S1_MAX_TABLES = 128;   // tables per Stage One launch (kernel parameter space)
+constexpr int S1_MAX_TABLES = 128;   // tables per Stage One launch with the small argument block (3.3 KB)
+constexpr int S1_BIG_TABLES = 1024;  // ... with the large one (25 KB; kernel arguments may take up to 32 764 bytes)
 constexpr int MAX_IPT = 8;           // ids per thread
 constexpr int MAX_SPT = 8;           // slots per thread
 constexpr int XFER_MAX_SEG = 2048;   // segments per Stage Two launch (prefix sums live in shared memory)
 
-struct S1Params {
+// The per-call host arrays travel as kernel arguments, CAP tables' worth of them: a call needs no staging copy.
+template <int CAP>
+struct S1ParamsT {
     int32_t*       tok;          // [num_tables][S]
     int8_t*        life;         // [num_tables][S]
     uint8_t*       buffer;       // [num_tables][S * row_bytes]
@@ -73,11 +76,14 @@ struct S1Params {
     unsigned long long  host_seq = 0;
     uint32_t            expect = 0;             // tables of the call
     const int32_t* verified_len_dev = nullptr;  // [n] of the call: read instead of verified_len[] when set
-    uint32_t table_id[S1_MAX_TABLES];
-    int32_t  verified_len[S1_MAX_TABLES];
-    uint64_t kv_base[S1_MAX_TABLES];
-    uint64_t kv_stride[S1_MAX_TABLES];
+    uint32_t table_id[CAP];
+    int32_t  verified_len[CAP];
+    uint64_t kv_base[CAP];
+    uint64_t kv_stride[CAP];
 };
+using S1Params = S1ParamsT<S1_MAX_TABLES>;
+using S1ParamsBig = S1ParamsT<S1_BIG_TABLES>;
+static_assert(sizeof(S1ParamsBig) <= 32764, "kernel argument block too large");
 
 struct XferParams {
     const SegDesc* seg;
@@ -88,6 +94,7 @@ struct XferParams {
 };
 
 constexpr int OVERLAP_MAX_TOKENS = 8;
+constexpr int OVERLAP_MAX_TABLES = S1_BIG_TABLES;   // one Stage One launch
 constexpr uint32_t OVERLAP_SPIN_LIMIT = 1u << 18;   // polls of >= 64 ns each before the wait gives up (~17 ms)
 
 struct XferOverlapParams {       // Stage Two that starts on token g's misses while Stage One places token g+1
@@ -131,6 +138,7 @@ size_t stage_one_paper_smem_bytes(uint32_t S, uint32_t K, uint32_t L);
 uint32_t stage_one_threads(uint32_t S, uint32_t K);
 cudaError_t stage_one_prepare(size_t max_smem);
 cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream);
+cudaError_t launch_stage_one(const S1ParamsBig& p, uint32_t n_tables, cudaStream_t stream);   // hash / direct index only
 cudaError_t launch_direct_index_from_state(const int32_t* tok, uint16_t* where, uint32_t first_table, uint32_t n_tables,
                                            uint32_t S, uint32_t max_context, cudaStream_t stream);
 cudaError_t launch_all_k_prepare(const AllKParams& p, uint32_t n_tables, cudaStream_t stream);

@@ -245,7 +245,8 @@ __device__ __forceinline__ void count_lifetimes(uint32_t w0, uint32_t w1, uint32
 // this table is placed - `count` more entries of the table's miss list are final.  Called by every thread of the
 // block: the block meets after its list writes; one thread then fences (the barrier makes the fence cover the whole
 // block's earlier writes, as in a grid-wide barrier) and raises the counter of token g.
-__device__ __forceinline__ void publish_token(const S1Params& p, uint32_t ti, uint32_t table, uint32_t g, uint32_t count)
+template <typename P>
+__device__ __forceinline__ void publish_token(const P& p, uint32_t ti, uint32_t table, uint32_t g, uint32_t count)
 {
     if (!p.ready) return;
     const uint32_t tid = threadIdx.x;
@@ -273,8 +274,8 @@ __device__ __forceinline__ void publish_token(const S1Params& p, uint32_t ti, ui
     }
 }
 
-template <bool DIRECT>
-__global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_constant__ S1Params p)
+template <bool DIRECT, int CAP>
+__global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_constant__ S1ParamsT<CAP> p)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     const uint32_t S = p.S, K = p.K, H = DIRECT ? 0u : 1u << p.logH, Kp = (K + 7u) & ~7u;
@@ -890,29 +891,58 @@ uint32_t stage_one_threads(uint32_t S, uint32_t K)
 
 cudaError_t stage_one_prepare(size_t max_smem)
 {
-    cudaError_t e = cudaFuncSetAttribute(avsg_stage_one_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(avsg_stage_one_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(avsg_stage_one_paper_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    const void* kernels[] = {
+        reinterpret_cast<const void*>(avsg_stage_one_kernel<false, S1_MAX_TABLES>),
+        reinterpret_cast<const void*>(avsg_stage_one_kernel<true, S1_MAX_TABLES>),
+        reinterpret_cast<const void*>(avsg_stage_one_kernel<false, S1_BIG_TABLES>),
+        reinterpret_cast<const void*>(avsg_stage_one_kernel<true, S1_BIG_TABLES>),
+        reinterpret_cast<const void*>(avsg_stage_one_paper_kernel)};
+    for (const void* k : kernels) {
+        cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
-cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream)
+namespace {
+template <int CAP>
+cudaError_t launch_stage_one_t(const S1ParamsT<CAP>& p, uint32_t n_tables, cudaStream_t stream)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_tables);
     cfg.blockDim = dim3(stage_one_threads(p.S, p.K));
-    const bool direct = p.where != nullptr, paper = p.qword != nullptr;
-    cfg.dynamicSmemBytes = paper ? stage_one_paper_smem_bytes(p.S, p.K, p.L) : stage_one_smem_bytes(p.S, p.K, p.L, direct);
+    const bool direct = p.where != nullptr;
+    cfg.dynamicSmemBytes = stage_one_smem_bytes(p.S, p.K, p.L, direct);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (paper) return cudaLaunchKernelEx(&cfg, avsg_stage_one_paper_kernel, p);
-    return direct ? cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel<true>, p)
-                  : cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel<false>, p);
+    return direct ? cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel<true, CAP>, p)
+                  : cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel<false, CAP>, p);
+}
+}  // namespace
+
+cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream)
+{
+    if (p.qword == nullptr) return launch_stage_one_t(p, n_tables, stream);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_tables);
+    cfg.blockDim = dim3(stage_one_threads(p.S, p.K));
+    cfg.dynamicSmemBytes = stage_one_paper_smem_bytes(p.S, p.K, p.L);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, avsg_stage_one_paper_kernel, p);
+}
+
+cudaError_t launch_stage_one(const S1ParamsBig& p, uint32_t n_tables, cudaStream_t stream)
+{
+    return launch_stage_one_t(p, n_tables, stream);
 }
 
 cudaError_t launch_direct_index_from_state(const int32_t* tok, uint16_t* where, uint32_t first_table, uint32_t n_tables,

@@ -182,9 +182,9 @@ __device__ __forceinline__ void retire_block(const XferOverlapParams& p)
 // this grid implies it.  All reads of data written by the running Stage One go to L2 (ld.cg / acquire).
 __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __grid_constant__ XferOverlapParams p)
 {
-    __shared__ uint32_t s_pref[S1_MAX_TABLES + 1];
-    __shared__ uint32_t s_off[S1_MAX_TABLES];
-    __shared__ uint64_t s_src[S1_MAX_TABLES], s_stride[S1_MAX_TABLES], s_dst[S1_MAX_TABLES];
+    __shared__ uint32_t s_pref[OVERLAP_MAX_TABLES + 1];
+    __shared__ uint32_t s_off[OVERLAP_MAX_TABLES];
+    __shared__ uint64_t s_src[OVERLAP_MAX_TABLES], s_stride[OVERLAP_MAX_TABLES], s_dst[OVERLAP_MAX_TABLES];
     __shared__ uint32_t s_w[40];
     __shared__ uint32_t s_ok;
 
@@ -220,7 +220,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __
                 s_dst[i] = __ldcg(&p.seg[i].dst_base);
             }
 
-        // prefix sum of token g's miss counts over the tables of the call (n <= S1_MAX_TABLES)
+        // prefix sum of token g's miss counts over the tables of the call (n <= OVERLAP_MAX_TABLES)
         uint32_t running = 0;
         for (uint32_t base = 0; base < n; base += nt) {
             const uint32_t i = base + tid;

@@ -177,10 +177,11 @@ def test_overlap_mode_four_tokens_and_mode_switches(avsg):
     assert ctx.sync_status() == 0
 
 
-@pytest.mark.parametrize("n,n_q,K,S", [(128, 2, 64, 256),      # as many tables as one Stage One launch takes
+@pytest.mark.parametrize("n,n_q,K,S", [(128, 2, 64, 256),      # as many tables as the small argument block takes
                                         (5, 8, 96, 1024),       # as many tokens as the overlapped kernel takes
                                         (3, 9, 100, 1024),      # one more: runs as the balanced mode
-                                        (129, 1, 32, 64)])      # one table more than a launch: balanced mode
+                                        (129, 1, 32, 64),       # more tables than the small argument block takes
+                                        (1030, 1, 16, 32)])     # more than the large one takes: balanced mode, two launches
 def test_overlap_mode_limits(avsg, n, n_q, K, S):
     import torch
     T, rb, ctxlen = 10, 48, 6000
