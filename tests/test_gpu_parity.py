@@ -196,7 +196,10 @@ def test_overlap_mode_limits(avsg, n, n_q, K, S):
     for t in range(T):
         X = np.stack([traces[i][0][t] for i in range(n)])
         N = [int(traces[i][1][t]) for i in range(n)]
-        out = ctx.step(list(range(n)), torch.from_numpy(X).cuda(), [kv] * n, N)
+        if t % 2:                                        # every other iteration through the host-buffer entry point
+            out = ctx.step_host(list(range(n)), torch.from_numpy(X).pin_memory(), [kv] * n, N)
+        else:
+            out = ctx.step(list(range(n)), torch.from_numpy(X).cuda(), [kv] * n, N)
         torch.cuda.synchronize()
         slots, mc = out.slots.cpu().numpy(), out.miss_count.cpu().numpy()
         for i in range(n):
