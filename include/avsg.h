@@ -163,6 +163,11 @@ int avsg_destroy(avsg_ctx *ctx);
  * Synchronous. */
 int avsg_reset(avsg_ctx *ctx, const uint32_t *table_ids, uint32_t n);
 
+/* The same, stream-ordered: one kernel on cuda_stream, after the calls issued
+ * to that stream before it and before those issued after it; nothing waits on
+ * the host.  What a serving loop uses when a request leaves the batch. */
+int avsg_reset_async(avsg_ctx *ctx, const uint32_t *table_ids, uint32_t n, void *cuda_stream);
+
 /* One decode iteration for the listed tables (Algorithm 4), asynchronous on
  * cuda_stream (a cudaStream_t; NULL = default stream).  When the stream has
  * finished this call, buffer[table][slots[...]] holds host row x for every

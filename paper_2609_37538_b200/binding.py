@@ -22,7 +22,7 @@ STATUS_PROBE_EXHAUSTED, STATUS_NO_DEAD_SLOTS, STATUS_BAD_SLOT, STATUS_BAD_SEGMEN
     1, 2, 4, 8, 16, 32)
 
 EXPORTS = (
-    "avsg_create", "avsg_destroy", "avsg_reset", "avsg_step", "avsg_step_host", "avsg_buffer", "avsg_stats", "avsg_table_stats",
+    "avsg_create", "avsg_destroy", "avsg_reset", "avsg_reset_async", "avsg_step", "avsg_step_host", "avsg_buffer", "avsg_stats", "avsg_table_stats",
     "avsg_sync_status", "avsg_export_state", "avsg_import_state", "avsg_save_state", "avsg_restore_state",
     "avsg_set_transfer_mode", "avsg_set_timing", "avsg_set_transfer_geometry", "avsg_strerror",
     "avsg_step_noalloc", "avsg_export_hash_state", "avsg_import_hash_state", "avsg_clear_status",
@@ -94,6 +94,7 @@ def load_library():
     lib.avsg_stats.argtypes, lib.avsg_stats.restype = [vp, ctypes.POINTER(AvsgStats)], i32
     lib.avsg_table_stats.argtypes, lib.avsg_table_stats.restype = [vp, u32, ctypes.POINTER(AvsgStats)], i32
     lib.avsg_sync_status.argtypes, lib.avsg_sync_status.restype = [vp, ctypes.POINTER(u32)], i32
+    lib.avsg_reset_async.argtypes, lib.avsg_reset_async.restype = [vp, vp, u32, vp], i32
     lib.avsg_clear_status.argtypes, lib.avsg_clear_status.restype = [vp], i32
     lib.avsg_probe_wait_limit.argtypes, lib.avsg_probe_wait_limit.restype = [vp, vp], i32
     lib.avsg_export_state.argtypes, lib.avsg_export_state.restype = [vp, u32, vp, vp], i32
@@ -258,6 +259,11 @@ class Context:
     def reset(self, table_ids: Sequence[int]) -> None:
         ids = (ctypes.c_uint32 * len(table_ids))(*[int(t) for t in table_ids])
         _check(self._lib.avsg_reset(self._h, ids, len(table_ids)), "avsg_reset")
+
+    def reset_async(self, table_ids: Sequence[int], stream=None) -> None:
+        """Stream-ordered reset: nothing waits on the host."""
+        ids = (ctypes.c_uint32 * len(table_ids))(*[int(t) for t in table_ids])
+        _check(self._lib.avsg_reset_async(self._h, ids, len(table_ids), _stream_handle(stream)), "avsg_reset_async")
 
     def buffer(self, table_id: int):
         """The table's S rows as a uint8 CUDA tensor [S, row_bytes] (a view, no copy)."""

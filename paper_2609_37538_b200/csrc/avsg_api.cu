@@ -477,6 +477,26 @@ int avsg_reset(avsg_ctx* c, const uint32_t* table_ids, uint32_t n)
     return AVSG_OK;
 }
 
+int avsg_reset_async(avsg_ctx* c, const uint32_t* table_ids, uint32_t n, void* cuda_stream)
+{
+    if (!c || (!table_ids && n)) return AVSG_EINVAL;
+    for (uint32_t i = 0; i < n; ++i) if (table_ids[i] >= c->cfg.num_tables) return AVSG_EINVAL;
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return AVSG_ECUDA;
+    for (uint32_t first = 0; first < n; first += S1_MAX_TABLES) {
+        const uint32_t cnt = n - first < (uint32_t)S1_MAX_TABLES ? n - first : (uint32_t)S1_MAX_TABLES;
+        ResetParams p;
+        p.tok = c->d_tok; p.life = c->d_life; p.buffer = c->d_buffer; p.stats = c->d_stats; p.qword = c->d_q;
+        p.S = c->cfg.buffer_slots; p.row_bytes = c->cfg.row_bytes;
+        for (uint32_t i = 0; i < cnt; ++i) {
+            p.table_id[i] = table_ids[first + i];
+            c->kv_host[p.table_id[i]] = 0; c->kv_dev[p.table_id[i]] = 0;      // the next request brings its own host KV
+        }
+        CU(launch_reset_tables(p, cnt, static_cast<cudaStream_t>(cuda_stream)));
+    }
+    return AVSG_OK;
+}
+
 int avsg_step(avsg_ctx* c, const avsg_step_args* a, void* stream)
 {
     return step_impl(c, a, static_cast<cudaStream_t>(stream), false);

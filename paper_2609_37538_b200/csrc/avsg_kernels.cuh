@@ -133,6 +133,14 @@ struct AllKParams {
     uint64_t kv_stride[S1_MAX_TABLES];
 };
 
+struct ResetParams {             // stream-ordered reset of some tables: empty, dead, counters and rows zeroed
+    int32_t* tok; int8_t* life; uint8_t* buffer; TableStats* stats;
+    uint32_t* qword;             // paper-literal mode, else null
+    uint32_t S, row_bytes;
+    uint32_t table_id[S1_MAX_TABLES];
+};
+cudaError_t launch_reset_tables(const ResetParams& p, uint32_t n_tables, cudaStream_t stream);
+
 size_t stage_one_smem_bytes(uint32_t S, uint32_t K, uint32_t L, bool direct = false);
 size_t stage_one_paper_smem_bytes(uint32_t S, uint32_t K, uint32_t L);
 uint32_t stage_one_threads(uint32_t S, uint32_t K);

@@ -563,6 +563,23 @@ __global__ void avsg_direct_index_from_state_kernel(const int32_t* __restrict__ 
 }
 
 
+// A request ended: its tables become empty (id -1) and dead (lifetime -1) again, their counters and rows zero;
+// in the paper-literal mode every bucket word returns to (lifetime -1, invalid, fingerprint 0, slot 0).  The
+// direct index needs no reset: its entries are verified against the cached ids.  Grid (blocks per table, tables).
+__global__ void avsg_reset_tables_kernel(const __grid_constant__ ResetParams p)
+{
+    const uint32_t table = p.table_id[blockIdx.y];
+    const size_t S = p.S, tid = blockIdx.x * (size_t)blockDim.x + threadIdx.x, nth = (size_t)gridDim.x * blockDim.x;
+    for (size_t j = tid; j < S; j += nth) {
+        p.tok[table * S + j] = -1;
+        p.life[table * S + j] = (int8_t)-1;
+        if (p.qword) p.qword[table * S + j] = 0xFF800000u;
+    }
+    int4* rows = reinterpret_cast<int4*>(p.buffer + table * S * p.row_bytes);
+    for (size_t i = tid; i < S * (p.row_bytes >> 4); i += nth) rows[i] = make_int4(0, 0, 0, 0);
+    if (tid == 0) p.stats[table] = TableStats{0, 0, 0, 0, 0, 0};
+}
+
 // ---------------------------------------------------------------------------------------------------------------
 // Paper-literal Hash-State mode (Sec. 3.2-3.3, Eq. 2-4, Eq. 8-11, Algorithm 2): 64-bit entries (c_j, q_j) with
 // q_j = [lifetime 8 | invalid 1 | fingerprint 23-m | slot m], double hashing with retry budget R, fingerprint
@@ -951,6 +968,12 @@ cudaError_t launch_direct_index_from_state(const int32_t* tok, uint16_t* where, 
     const size_t n = (size_t)n_tables * S;
     const uint32_t blocks = (uint32_t)((n + 255) / 256 < 1184 ? (n + 255) / 256 : 1184);
     avsg_direct_index_from_state_kernel<<<blocks, 256, 0, stream>>>(tok, where, first_table, n_tables, S, max_context);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_reset_tables(const ResetParams& p, uint32_t n_tables, cudaStream_t stream)
+{
+    avsg_reset_tables_kernel<<<dim3(32, n_tables), 256, 0, stream>>>(p);
     return cudaGetLastError();
 }
 

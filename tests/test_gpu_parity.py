@@ -265,6 +265,44 @@ def test_a_captured_call_can_be_replayed(avsg, mode_name):
     assert ctx.sync_status() == 0
 
 
+@pytest.mark.parametrize("mode_name,index_name", [("XFER_SM_BALANCED", "INDEX_HASH"), ("XFER_SM_OVERLAP", "INDEX_DIRECT")])
+def test_stream_ordered_reset(avsg, mode_name, index_name):
+    """A request leaves the batch: its table is reset by a kernel in stream order, between two steps, with no host
+    synchronisation in between; the other tables carry on untouched."""
+    import torch
+    n, n_q, K, S, T, rb, ctxlen = 3, 2, 128, 512, 12, 48, 8000
+    cfgs = [tr.TraceConfig(seed=21, table=i, topk=K, n_q=n_q, n_iters=T, context=ctxlen, beta=(9, 1), p_recent=0.5,
+                           recent_window=1024) for i in range(n)]
+    traces = [tr.generate(c) for c in cfgs]
+    kv = avsg.pinned_empty(ctxlen * rb)
+    tr.fill_kv(kv.data_ptr(), 21, 0, ctxlen, rb)
+    ctx = avsg.Context(n, S, rb, K, n_q, 16, transfer_mode=getattr(avsg, mode_name),
+                       index_mode=getattr(avsg, index_name), max_context=ctxlen + n_q)
+    orc = [OracleTable(S, rb, 16) for _ in range(n)]
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for t in range(T):
+            X = np.stack([traces[i][0][t] for i in range(n)])
+            if t in (4, 9):                                  # table 1 (then tables 0 and 2) start over
+                gone = [1] if t == 4 else [0, 2]
+                ctx.reset_async(gone, stream)
+                for i in gone:
+                    orc[i].reset()
+            out = ctx.step(list(range(n)), torch.from_numpy(X).cuda(), [kv] * n, [ctxlen] * n, stream=stream)
+            stream.synchronize()
+            slots, hit = out.slots.cpu().numpy(), out.hit.cpu().numpy()
+            for i in range(n):
+                r = orc[i].step(X[i], ctxlen, kv.numpy(), rb)
+                assert (slots[i] == r.O).all() and (hit[i] == r.M).all(), (t, i)
+                tok, life = ctx.export_state(i)
+                c, l = orc[i].export_state()
+                assert (tok == c).all() and (life == l).all(), (t, i)
+                assert (ctx.buffer(i).cpu().numpy() == orc[i].rows()).all(), (t, i)
+                ts, oc = ctx.table_stats(i), orc[i].counters()
+                assert ts["hits"] == oc["hits"] and ts["misses"] == oc["misses"] and ts["steps"] == oc["steps"], (t, i)
+    assert ctx.sync_status() == 0
+
+
 def test_overlap_wait_gives_up_and_the_context_stays_usable(avsg):
     """The overlapped transfer kernel launched without its Stage One: every block polls up to its limit, raises
     the status bit, copies nothing and returns; after clearing the status word the context works as before."""
