@@ -106,7 +106,8 @@ typedef struct {
 } avsg_config;
 
 typedef struct {
-    uint32_t        n;             /* tables taking part in this call (1 .. num_tables)  */
+    uint32_t        n;             /* tables taking part in this call (1 .. num_tables,
+                                      at most 2048)                                      */
     const uint32_t *table_ids;     /* HOST [n]   distinct, each < num_tables             */
     uint32_t        n_tokens;      /* N_q of this call (<= max_tokens)                   */
     uint32_t        topk;          /* K of this call (<= max_topk)                       */
