@@ -155,37 +155,48 @@ typedef struct {
     float    reserved;
 } avsg_stats_t;
 
-/* Allocates all state: tables empty and dead ("each request starts with an
- * empty cache", App. E), buffers zeroed.  *out is set only on success. */
+/* App. E (a request starts with nothing cached), Sec. 3.1-3.2 (one S-slot
+ * buffer plus S state entries per request): allocates all state, every table
+ * empty (id -1) and dead (lifetime -1), buffers zeroed.  *out is set only on
+ * success.  buffer_slots above 8192 needs AVSG_INDEX_DIRECT (see the field). */
 int avsg_create(const avsg_config *cfg, avsg_ctx **out);
+
+/* No passage of the paper: releases everything avsg_create allocated, after
+ * waiting for the device.  The pointer is dead afterwards. */
 int avsg_destroy(avsg_ctx *ctx);
 
-/* A request ended: its tables become empty and dead again.  HOST table_ids[n].
- * Synchronous. */
+/* App. E: the next request served by a table starts with an empty cache.  The
+ * listed tables become empty and dead again, their rows and counters zero.
+ * HOST table_ids[n].  Synchronous. */
 int avsg_reset(avsg_ctx *ctx, const uint32_t *table_ids, uint32_t n);
 
-/* The same, stream-ordered: one kernel on cuda_stream, after the calls issued
- * to that stream before it and before those issued after it; nothing waits on
- * the host.  What a serving loop uses when a request leaves the batch. */
+/* The same (App. E), stream-ordered: one kernel on cuda_stream, after the
+ * calls issued to that stream before it and before those issued after it;
+ * nothing waits on the host.  What a serving loop uses when a request leaves
+ * the batch. */
 int avsg_reset_async(avsg_ctx *ctx, const uint32_t *table_ids, uint32_t n, void *cuda_stream);
 
-/* One decode iteration for the listed tables (Algorithm 4), asynchronous on
+/* Algorithm 4 (with Algorithm 1 and 3 per token, Sec. 3.4 for the gather): one
+ * decode iteration for the listed tables, asynchronous on
  * cuda_stream (a cudaStream_t; NULL = default stream).  When the stream has
  * finished this call, buffer[table][slots[...]] holds host row x for every
  * non-padding id x.  Host KV, indices and outputs must stay valid until then.
  * Host arrays of the argument block are consumed before the call returns. */
 int avsg_step(avsg_ctx *ctx, const avsg_step_args *args, void *cuda_stream);
 
-/* Same, but indices / slots / hit / miss_count are HOST pointers (pinned for
+/* Same operation (Algorithm 4), but indices / slots / hit / miss_count are HOST pointers (pinned for
  * asynchrony); the library stages them through its own device buffers on the
  * stream: one upload of the ids, one download per requested output. */
 int avsg_step_host(avsg_ctx *ctx, const avsg_step_args *args, void *cuda_stream);
 
-/* DEVICE base of a table's S rows of row_bytes (what attention gathers from). */
+/* Sec. 3.1: the S-slot device buffer that sparse attention reads through the
+ * slot matrix O.  Returns the DEVICE base of a table's S rows of row_bytes. */
 int avsg_buffer(avsg_ctx *ctx, uint32_t table_id, void **d_rows);
 
-/* Waits for the device, then reports cumulative counters.  Returns
- * AVSG_EDEVICE_STATUS (and still fills *out) if a kernel flagged a problem. */
+/* Sec. 4.4 (hit rate) and App. D (effective bandwidth V / t with V = row_bytes
+ * x missed rows): waits for the device, then reports the cumulative counters
+ * those figures are formed from.  Returns AVSG_EDEVICE_STATUS (and still fills
+ * *out) if a kernel flagged a problem. */
 int avsg_stats(avsg_ctx *ctx, avsg_stats_t *out);
 
 /* The same counters for ONE table (the last_* fields stay zero): what the
@@ -193,12 +204,13 @@ int avsg_stats(avsg_ctx *ctx, avsg_stats_t *out);
  * the device. */
 int avsg_table_stats(avsg_ctx *ctx, uint32_t table_id, avsg_stats_t *out);
 
-/* Waits for the device; returns AVSG_EDEVICE_STATUS if a kernel flagged a
- * problem, and the raw status word in *status_word when not NULL. */
+/* No passage of the paper (error reporting): waits for the device; returns
+ * AVSG_EDEVICE_STATUS if a kernel flagged a problem, and the raw status word
+ * in *status_word when not NULL. */
 int avsg_sync_status(avsg_ctx *ctx, uint32_t *status_word);
 
-/* Waits for the device, zeroes the status word and the counters of the
- * overlapped mode (which a call that reported AVSG_STATUS_WAIT_TIMEOUT may have
+/* No passage of the paper: waits for the device, zeroes the status word and
+ * the counters of the overlapped mode (which a call that reported AVSG_STATUS_WAIT_TIMEOUT may have
  * left raised). */
 int avsg_clear_status(avsg_ctx *ctx);
 
@@ -210,8 +222,10 @@ int avsg_clear_status(avsg_ctx *ctx);
  * counterpart; its Stage Two starts after Stage One (Alg. 4). */
 int avsg_probe_wait_limit(avsg_ctx *ctx, void *cuda_stream);
 
-/* Table state for checkpoints and parity checks.  HOST tok[S] (cached id per
- * slot, -1 empty) and life[S] (lifetime, -1 dead).  Synchronous. */
+/* Sec. 3.2: the state of a table is its S entries (cached id c_j, lifetime);
+ * these two calls read and replace it, for checkpoints and parity checks.
+ * HOST tok[S] (cached id per slot, -1 empty) and life[S] (lifetime, -1 dead).
+ * Synchronous. */
 int avsg_export_state(avsg_ctx *ctx, uint32_t table_id, int32_t *tok, int8_t *life);
 int avsg_import_state(avsg_ctx *ctx, uint32_t table_id, const int32_t *tok, const int8_t *life);
 
@@ -220,19 +234,23 @@ int avsg_import_state(avsg_ctx *ctx, uint32_t table_id, const int32_t *tok, cons
 int avsg_export_hash_state(avsg_ctx *ctx, uint32_t table_id, int32_t *c, uint32_t *q);
 int avsg_import_hash_state(avsg_ctx *ctx, uint32_t table_id, const int32_t *c, const uint32_t *q);
 
-/* Device-side snapshot of every table's (tok, life) and its restore, both
- * asynchronous on the stream: lets a measurement replay one step many times. */
+/* App. C times Stage One as the median over repeated runs of one step: a
+ * device-side snapshot of every table's (tok, life) and its restore, both
+ * asynchronous on the stream, let a measurement replay one step many times. */
 int avsg_save_state(avsg_ctx *ctx, void *cuda_stream);
 int avsg_restore_state(avsg_ctx *ctx, void *cuda_stream);
 
-/* Switches the Stage Two strategy of later calls (AVSG_XFER_*). */
+/* App. D compares transfer strategies on the same misses: switches the Stage
+ * Two strategy of later calls (AVSG_XFER_*). */
 int avsg_set_transfer_mode(avsg_ctx *ctx, uint32_t mode);
 
-/* enable != 0: later calls record CUDA events around Stage One and Stage Two;
+/* App. C / App. D report Stage One and Stage Two times separately.  enable
+ * != 0: later calls record CUDA events around Stage One and Stage Two;
  * avsg_stats() then reports the last call's device times. */
 int avsg_set_timing(avsg_ctx *ctx, int enable);
 
-/* Stage Two geometry: thread blocks (0 = one per SM) and threads per block. */
+/* Eq. 6 cuts the miss list over C cores: C = thread blocks (0 = one per SM);
+ * threads per block is this build's own knob. */
 int avsg_set_transfer_geometry(avsg_ctx *ctx, uint32_t blocks, uint32_t threads);
 
 /*
@@ -293,6 +311,7 @@ typedef struct {
 
 int avsg_step_noalloc(const avsg_noalloc_args *args, void *cuda_stream);
 
+/* No passage of the paper: a static string naming an AVSG_E* code. */
 const char *avsg_strerror(int code);
 
 #ifdef __cplusplus

@@ -82,7 +82,7 @@ void orc_destroy(orc_table *t)
     free(t->c); free(t->life); free(t->rows); free(t);
 }
 
-/* "Each request starts with an empty cache" (App. E): empty and dead. */
+/* A new request finds nothing cached (App. E): every slot empty and dead, rows and counters zero. */
 void orc_reset(orc_table *t)
 {
     for (uint32_t j = 0; j < t->S; ++j) { t->c[j] = -1; t->life[j] = -1; }
@@ -301,8 +301,9 @@ void orc_counters(const orc_table *t, uint64_t out[6])
  *
  * Readings needed to make it deterministic (the paper leaves them open):
  *   - a1, a2 are parameters (two distinct odd primes);
- *   - "same-bucket writes retain one nondeterministic writer": here the miss
- *     with the HIGHEST position wins;
+ *   - when several misses of one token write the same bucket word, the paper
+ *     lets an unspecified one of them win (Alg. 2): here the miss with the
+ *     HIGHEST position wins;
  *   - Alg. 2 evaluates all probes on the table as it is when UpdateState is
  *     entered, then writes ids and lifetimes, then writes the bucket words,
  *     reading the preserved lifetime at that moment (statement order);

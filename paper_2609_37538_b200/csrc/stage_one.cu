@@ -48,34 +48,6 @@ __device__ __forceinline__ uint32_t hash_id(int32_t x, uint32_t logH)
     return ((uint32_t)x * 2654435769u) >> (32u - logH);
 }
 
-__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, uint32_t lane)
-{
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        uint32_t n = __shfl_up_sync(0xffffffffu, v, o);
-        if (lane >= (uint32_t)o) v += n;
-    }
-    return v;
-}
-
-// Exclusive prefix sum over the block in thread order; s_w holds 33 words.
-__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* s_w, uint32_t& total)
-{
-    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    const uint32_t incl = warp_incl_scan(v, lane);
-    if (lane == 31) s_w[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-        uint32_t w = lane < nwarps ? s_w[lane] : 0u;
-        uint32_t wi = warp_incl_scan(w, lane);
-        s_w[lane] = wi - w;
-        if (lane == 31) s_w[32] = wi;
-    }
-    __syncthreads();
-    total = s_w[32];
-    return incl - v + s_w[warp];
-}
-
 struct Index {
     int32_t*  key;
     uint16_t* val;
@@ -584,8 +556,8 @@ __global__ void avsg_reset_tables_kernel(const __grid_constant__ ResetParams p)
 // Paper-literal Hash-State mode (Sec. 3.2-3.3, Eq. 2-4, Eq. 8-11, Algorithm 2): 64-bit entries (c_j, q_j) with
 // q_j = [lifetime 8 | invalid 1 | fingerprint 23-m | slot m], double hashing with retry budget R, fingerprint
 // check and lazy reclamation of stale bucket words.  Lossy by design: a resident id whose bucket word was
-// overwritten is missed and fetched again.  Where Algorithm 2 leaves "one nondeterministic writer" per bucket,
-// the miss with the highest position wins (an atomicMax on a per-bucket tag), so results are reproducible.
+// overwritten is missed and fetched again.  Where Algorithm 2 leaves open which of several writers of one bucket
+// wins, the miss with the highest position wins (an atomicMax on a per-bucket tag), so results are reproducible.
 // ---------------------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void pack_life_bytes(const uint32_t* q, uint32_t j0, uint32_t spt, bool own,
                                                 uint32_t& w0, uint32_t& w1)

@@ -24,33 +24,6 @@ namespace {
 
 constexpr int CHUNKS_PER_PASS = 4;     // 16-byte loads a lane keeps in flight (covers rows up to 2 KiB per pass)
 
-__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, uint32_t lane)
-{
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        uint32_t n = __shfl_up_sync(0xffffffffu, v, o);
-        if (lane >= (uint32_t)o) v += n;
-    }
-    return v;
-}
-
-__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* s_w, uint32_t& total)
-{
-    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    const uint32_t incl = warp_incl_scan(v, lane);
-    if (lane == 31) s_w[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-        uint32_t w = lane < nwarps ? s_w[lane] : 0u;
-        uint32_t wi = warp_incl_scan(w, lane);
-        s_w[lane] = wi - w;
-        if (lane == 31) s_w[32] = wi;
-    }
-    __syncthreads();
-    total = s_w[32];
-    return incl - v + s_w[warp];
-}
-
 // 16-byte global load / store in the order written (volatile asm statements keep their relative order).
 __device__ __forceinline__ int4 ld16(uint64_t addr)
 {

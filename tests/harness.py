@@ -31,10 +31,12 @@ class HostKV:
 def run_parity(w: tr.Workload, *, tables: Optional[Sequence[int]] = None, mode: int = 0, host_io: bool = False,
                row_stride: Optional[int] = None, buffer_every: int = 1, oracle_tables: Optional[Sequence[int]] = None,
                n_iters: Optional[int] = None, threads: Optional[int] = None, xfer_geometry=None,
-               index_mode: int = 0) -> Dict:
+               index_mode: int = 0, permute_seed: Optional[int] = None) -> Dict:
     """Steps every call group of w for every iteration on the GPU; the tables in oracle_tables (default: all)
     are stepped by the oracle too and compared after EVERY step: hit mask, slot table, miss counts, (tok, life);
-    the buffer rows every buffer_every iterations and at the end.  Returns counters of both sides."""
+    the buffer rows every buffer_every iterations and at the end.  With permute_seed the K positions of every token
+    of every table are shuffled (seeded) before either side sees them, so that position order and id order differ
+    (the k-th miss in POSITION order takes the k-th dead slot).  Returns counters of both sides."""
     import torch
     import paper_2609_37538_b200 as avsg
 
@@ -44,6 +46,12 @@ def run_parity(w: tr.Workload, *, tables: Optional[Sequence[int]] = None, mode: 
     with ThreadPoolExecutor(max_workers=threads or os.cpu_count()) as ex:
         for ti, res in zip(ids, ex.map(lambda i: tr.generate(w.tables[i]), ids)):
             traces[ti] = res
+    if permute_seed is not None:
+        for ti in ids:
+            X, N = traces[ti]
+            rng = np.random.default_rng([permute_seed, ti])
+            order = np.argsort(rng.random(X.shape), axis=-1)
+            traces[ti] = (np.ascontiguousarray(np.take_along_axis(X, order, axis=-1)), N)
     kv = HostKV(w, ids, row_stride)
     T = w.n_iters if n_iters is None else min(n_iters, w.n_iters)
     local = {ti: k for k, ti in enumerate(ids)}                  # context table id of a workload table

@@ -122,6 +122,44 @@ def test_transfer_geometries(avsg):
         _parity(w, xfer_geometry=geo)
 
 
+# ---- ids that are not ascending: position order and id order differ (Alg. 1 Pass 3: the k-th miss in POSITION
+# ---- order takes the k-th dead slot; the input need not be sorted) ---------------------------------------------
+UNSORTED_SHAPES = [
+    ("C2", dict(topk=37, buffer_slots=128, n_iters=40, context=4096, recent_window=128)),
+    ("C2", dict(topk=1000, buffer_slots=2048, n_iters=24, context=65536, recent_window=2048)),
+    ("C4", dict(topk=300, buffer_slots=1024, n_iters=30, context=1 << 16, requests=5, hot_size=64, hot_range=1024)),
+    ("C5", dict(topk=128, buffer_slots=256, n_iters=8, requests=4, ctx_lo=40, ctx_hi=100)),     # padding lands anywhere
+]
+
+
+@pytest.mark.parametrize("name,kw", UNSORTED_SHAPES)
+@pytest.mark.parametrize("index", ["INDEX_HASH", "INDEX_DIRECT"])
+@pytest.mark.parametrize("mode", ["XFER_SM_BALANCED", "XFER_SM_OVERLAP", "XFER_REQUEST_LEVEL"])
+def test_unsorted_ids_shapes(avsg, name, kw, index, mode):
+    _parity(tr.workload(name, **kw), mode=getattr(avsg, mode), index_mode=getattr(avsg, index), permute_seed=7)
+
+
+def test_unsorted_ids_c2_full(avsg):
+    r = _parity(tr.workload("C2"), permute_seed=11, buffer_every=8, index_mode=avsg.INDEX_DIRECT,
+                mode=avsg.XFER_SM_OVERLAP)
+    assert r["gpu"]["tokens"] == 256
+    _parity(tr.workload("C2", n_iters=48), permute_seed=12, buffer_every=8)
+
+
+def test_unsorted_ids_differ_from_sorted(avsg):
+    """The permutation matters: the same selections in ascending order give another slot table (so a kernel that
+    ordered the misses by id could not pass the tests above)."""
+    w = tr.workload("C2", topk=64, buffer_slots=256, n_iters=3, context=4096, recent_window=256)
+    X, N = tr.generate(w.tables[0])
+    order = np.argsort(np.random.default_rng([7, 0]).random(X.shape), axis=-1)
+    Xp = np.take_along_axis(X, order, axis=-1)
+    a, b = OracleTable(w.buffer_slots, 16, w.max_lifetime), OracleTable(w.buffer_slots, 16, w.max_lifetime)
+    ra, rb = a.step(X[0], int(N[0])), b.step(Xp[0], int(N[0]))
+    slot_of_a = dict(zip(X[0].ravel().tolist(), ra.O.ravel().tolist()))
+    slot_of_b = dict(zip(Xp[0].ravel().tolist(), rb.O.ravel().tolist()))
+    assert slot_of_a != slot_of_b
+
+
 # ---- Stage Two overlapping Stage One (latency hiding, App. G) ---------------------------------------------------
 @pytest.mark.parametrize("name,kw,index", [
     ("C1", {}, "INDEX_HASH"), ("C2", {}, "INDEX_HASH"), ("C2", {}, "INDEX_DIRECT"), ("C3", {}, "INDEX_DIRECT"),
@@ -556,12 +594,17 @@ def test_degenerate_selections(avsg, index_mode):
 
 
 # ---- the paper-literal (lossy) Hash-State mode against its own oracle ---------------------------------------------
-def _literal_parity(avsg, w, n_iters=None, R=3, mode=0):
+def _literal_parity(avsg, w, n_iters=None, R=3, mode=0, permute_seed=None):
     import torch
     from oracle import LiteralOracleTable
     from harness import HostKV
     ids = list(range(w.num_tables))
     traces = {ti: tr.generate(w.tables[ti]) for ti in ids}
+    if permute_seed is not None:             # ids in a seeded random order: position order differs from id order
+        for ti in ids:
+            X, N = traces[ti]
+            order = np.argsort(np.random.default_rng([permute_seed, ti]).random(X.shape), axis=-1)
+            traces[ti] = (np.ascontiguousarray(np.take_along_axis(X, order, axis=-1)), N)
     kv = HostKV(w, ids)
     ctx = avsg.Context(num_tables=len(ids), buffer_slots=w.buffer_slots, row_bytes=w.row_bytes, max_topk=w.topk,
                        max_tokens=w.n_q, max_lifetime=w.max_lifetime, index_mode=avsg.INDEX_PAPER, probe_retries=R,
@@ -613,6 +656,15 @@ def test_paper_literal_mode_shapes(avsg, kw, R):
     _literal_parity(avsg, tr.workload("C2", **kw), R=R)
 
 
+def test_paper_literal_mode_unsorted_ids(avsg):
+    # position order decides both the slot of a miss and, in this mode, the winner of a shared bucket
+    _literal_parity(avsg, tr.workload("C2", topk=37, buffer_slots=128, n_iters=40, context=4096, recent_window=128),
+                    permute_seed=5)
+    _literal_parity(avsg, tr.workload("C2", topk=1000, buffer_slots=2048, n_iters=16, context=65536,
+                                      recent_window=2048), R=7, permute_seed=6, mode=avsg.XFER_SM_OVERLAP)
+    _literal_parity(avsg, tr.workload("C3", requests=4, layers=1, n_iters=8), permute_seed=8)
+
+
 # ---- randomly drawn shapes: tables, S, K, tokens, L, row size, index and transfer mode -------------------------------
 @pytest.mark.parametrize("seed", range(12))
 def test_random_shapes(avsg, seed):
@@ -644,4 +696,5 @@ def test_random_shapes(avsg, seed):
                                          "XFER_SM_OVERLAP"])))
     index_mode = int(rng.choice([avsg.INDEX_HASH, avsg.INDEX_DIRECT]))
     _parity(w, mode=mode, index_mode=index_mode, host_io=bool(rng.random() < 0.3),
-            xfer_geometry=(int(rng.choice([1, 37, 148, 300])), int(rng.choice([32, 128, 256, 1024]))))
+            xfer_geometry=(int(rng.choice([1, 37, 148, 300])), int(rng.choice([32, 128, 256, 1024]))),
+            permute_seed=seed if seed % 2 else None)

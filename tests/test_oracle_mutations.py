@@ -32,6 +32,16 @@ MUTATIONS = [
     ("Eq. 13 ignores the remainder", "return B / C + (c < B % C ? 1u : 0u);", "return B / C;"),
     ("Eq. 14 rounds the upper end up", "*end = (uint64_t)(c + 1) * n_positions / C;",
      "*end = ((uint64_t)(c + 1) * n_positions + C - 1) / C;"),
+    ("the gather steps through the host rows by row_bytes instead of the stride",
+     "host_kv + (uint64_t)list[k].x * row_stride, t->row_bytes);", "host_kv + (uint64_t)list[k].x * t->row_bytes, t->row_bytes);"),
+    ("transfer-all-K ignores the host row stride",
+     "host_kv + (uint64_t)X[p] * row_stride, t->row_bytes);", "host_kv + (uint64_t)X[p] * t->row_bytes, t->row_bytes);"),
+    ("reset forgets the counters",
+     "    t->steps = t->tokens = t->hits = t->misses = t->rows_copied = t->extra_decays = 0;\n}", "}"),
+    ("reset leaves the rows", "    memset(t->rows, 0, (size_t)t->S * t->row_bytes);\n    t->steps = ", "    t->steps = "),
+    ("reset leaves the lifetimes",
+     "for (uint32_t j = 0; j < t->S; ++j) { t->c[j] = -1; t->life[j] = -1; }\n    memset(",
+     "for (uint32_t j = 0; j < t->S; ++j) { t->c[j] = -1; }\n    memset("),
     ("transfer-all-K keeps a padding row", "if (X[p] < 0) { O[p] = -1; continue; }", "if (X[p] < 0) { O[p] = (int32_t)p; continue; }"),
 ]
 

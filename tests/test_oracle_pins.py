@@ -32,7 +32,8 @@ def _read_example(name):
 # hand-worked examples (Algorithm 1: pre-decay, refresh-before-allocate, decay
 # loop, ordered assignment of dead slots)
 # ----------------------------------------------------------------------------
-@pytest.mark.parametrize("name", ["alloc_example.txt", "refresh_example.txt"])
+@pytest.mark.parametrize("name", ["alloc_example.txt", "refresh_example.txt", "descending_example.txt",
+                                  "descending_decay_example.txt"])
 def test_hand_worked_example(name):
     ex = _read_example(name)
     S, L, g = int(ex["S"][0]), int(ex["L"][0]), int(ex["g"][0])
@@ -65,7 +66,10 @@ def test_membership_bruteforce_tiny(seed):
     t = OracleTable(S, 8, L)
     universe = 3 * S
     for step in range(40):
-        X = np.stack([np.sort(rng.choice(universe, K, replace=False)) for _ in range(n_q)]).astype(np.int32)
+        # ids in ascending order on even seeds, in a random order on odd seeds (the input need not be sorted)
+        X = np.stack([rng.choice(universe, K, replace=False) for _ in range(n_q)]).astype(np.int32)
+        if seed % 2 == 0:
+            X.sort(axis=1)
         # token by token, so that "resident" is the table content at the moment the token is
         # processed: an old id may be reclaimed by an earlier token of the same iteration (App. B)
         O = np.empty((n_q, K), np.int32)
@@ -410,6 +414,63 @@ def test_all_k_comparator():
     keep = want >= 0
     assert (t2.rows()[keep] == kv.reshape(500, rb)[Xp.ravel()[keep]]).all()
     assert not t2.rows()[~keep].any()                      # the two padded slots were never written
+
+
+# ----------------------------------------------------------------------------
+# A request that ends leaves its table as a new request finds it (App. E: every request starts with an empty
+# cache): after a busy trace, reset() must give a table that cannot be told from a fresh one - ids, lifetimes,
+# rows and all six counters - now and on the steps that follow.
+# ----------------------------------------------------------------------------
+def test_reset_equals_fresh_table():
+    w = tr.workload("C2", topk=64, buffer_slots=128, n_iters=30, context=4096, recent_window=256, max_lifetime=16)
+    X, N = tr.generate(w.tables[0])
+    rb = 16
+    kv = np.empty(w.tables[0].context * rb, np.uint8)
+    tr.fill_kv(kv, w.seed, 0, w.tables[0].context, rb)
+    used, fresh = OracleTable(w.buffer_slots, rb, w.max_lifetime), OracleTable(w.buffer_slots, rb, w.max_lifetime)
+    for t in range(20):
+        used.step(X[t], int(N[t]), kv)
+    c = used.counters()
+    assert c["misses"] > 0 and c["extra_decays"] > 0 and used.rows().any()       # the trace was busy
+    used.reset()
+    assert used.counters() == fresh.counters() == dict.fromkeys(c, 0)
+    assert (used.export_state()[0] == -1).all() and (used.export_state()[1] == -1).all()
+    assert not used.rows().any()
+    for t in range(20, 30):                                                      # and behaves like one from here on
+        a, b = used.step(X[t], int(N[t]), kv), fresh.step(X[t], int(N[t]), kv)
+        assert (a.O == b.O).all() and (a.M == b.M).all() and (a.n == b.n).all()
+    assert used.counters() == fresh.counters()
+    assert (used.rows() == fresh.rows()).all()
+
+
+# ----------------------------------------------------------------------------
+# Host rows with a stride: row x starts at x * row_stride and only its first row_bytes bytes are the row.  A
+# padded host array (gaps filled with 0xEE) must give exactly the rows of the packed array, for the operator
+# and for the transfer-all-K comparator.
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("stride", [48, 1024])
+def test_strided_host_rows_equal_packed_rows(stride):
+    rb, ctx_len = 32, 2048
+    w = tr.workload("C2", topk=48, buffer_slots=128, n_iters=12, context=ctx_len, recent_window=256, row_bytes=rb)
+    X, N = tr.generate(w.tables[0])
+    packed = np.empty(ctx_len * rb, np.uint8)
+    tr.fill_kv(packed, w.seed, 0, ctx_len, rb)
+    padded = np.full(ctx_len * stride, 0xEE, np.uint8)
+    padded.reshape(ctx_len, stride)[:, :rb] = packed.reshape(ctx_len, rb)
+    a, b = OracleTable(w.buffer_slots, rb, 4), OracleTable(w.buffer_slots, rb, 4)
+    for t in range(X.shape[0]):
+        ra, rb_ = a.step(X[t], int(N[t]), packed), b.step(X[t], int(N[t]), padded, stride)
+        assert (ra.O == rb_.O).all() and (ra.xfer == rb_.xfer).all()
+        assert (a.rows() == b.rows()).all(), t
+        # and the rows are the right ones: slot O[g, i] holds host row X[g, i]
+        for g in range(X.shape[1]):
+            assert (b.rows()[rb_.O[g]] == packed.reshape(ctx_len, rb)[X[t, g]]).all()
+    assert a.counters() == b.counters()
+    ka, kb = OracleTable(w.buffer_slots, rb, 4), OracleTable(w.buffer_slots, rb, 4)
+    ka.step_all_k(X[3], packed)
+    kb.step_all_k(X[3], padded, stride)
+    assert (ka.rows() == kb.rows()).all() and ka.rows().any()
+    assert (kb.rows()[: X[3].size] == packed.reshape(ctx_len, rb)[X[3].ravel()]).all()
 
 
 # ----------------------------------------------------------------------------
