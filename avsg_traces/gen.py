@@ -190,37 +190,38 @@ def _c1(seed=0, **kw) -> Workload:
                     "1 table, fixed 90% overlap, uniform new ids")
 
 
-def _mtp_tables(seed, n_tables, K, T, ctx, beta, **mix) -> List[TraceConfig]:
-    return [TraceConfig(seed=seed, table=i, topk=K, n_q=2, n_iters=T, context=ctx, ctx_growth=True,
+def _mtp_tables(seed, n_tables, K, T, ctx, beta, n_q=2, **mix) -> List[TraceConfig]:
+    return [TraceConfig(seed=seed, table=i, topk=K, n_q=n_q, n_iters=T, context=ctx, ctx_growth=True,
                         beta=beta, **mix) for i in range(n_tables)]
 
 
 def _c2(seed=2, **kw) -> Workload:
     K, S, T = kw.get("topk", 2048), kw.get("buffer_slots", 8192), kw.get("n_iters", 128)
     ctx = kw.get("context", 131072)
-    tabs = _mtp_tables(seed, 1, K, T, ctx, (18, 2), p_recent=0.5, recent_window=kw.get("recent_window", 4096))
-    return Workload("C2", seed, S, ROW_BYTES, 16, K, 2, T, tabs, [[0]],
-                    "1 table, MTP 2 tokens, Beta(18,2) overlap, half recent / half uniform")
+    n_q = kw.get("n_q", 2)
+    tabs = _mtp_tables(seed, 1, K, T, ctx, (18, 2), n_q=n_q, p_recent=0.5, recent_window=kw.get("recent_window", 4096))
+    return Workload("C2", seed, S, ROW_BYTES, 16, K, n_q, T, tabs, [[0]],
+                    "1 table, MTP %d tokens, Beta(18,2) overlap, half recent / half uniform" % n_q)
 
 
 def _c3(seed=3, **kw) -> Workload:
     K, S, T = kw.get("topk", 2048), kw.get("buffer_slots", 8192), kw.get("n_iters", 64)
     ctx = kw.get("context", 131072)
-    n_req, n_layers = kw.get("requests", 32), kw.get("layers", 4)
-    tabs = _mtp_tables(seed, n_req * n_layers, K, T, ctx, (18, 2), p_recent=0.5,
+    n_req, n_layers, n_q = kw.get("requests", 32), kw.get("layers", 4), kw.get("n_q", 2)
+    tabs = _mtp_tables(seed, n_req * n_layers, K, T, ctx, (18, 2), n_q=n_q, p_recent=0.5,
                        recent_window=kw.get("recent_window", 4096))
     calls = [[layer * n_req + r for r in range(n_req)] for layer in range(n_layers)]
-    return Workload("C3", seed, S, ROW_BYTES, 16, K, 2, T, tabs, calls,
+    return Workload("C3", seed, S, ROW_BYTES, 16, K, n_q, T, tabs, calls,
                     "%d requests x %d layers, one call per layer" % (n_req, n_layers))
 
 
 def _c4(seed=4, **kw) -> Workload:
     K, S, T = kw.get("topk", 2048), kw.get("buffer_slots", 8192), kw.get("n_iters", 64)
     ctx = kw.get("context", 1 << 20)
-    n_req = kw.get("requests", 16)
-    tabs = _mtp_tables(seed, n_req, K, T, ctx, (9, 1), p_hot=0.2, hot_size=kw.get("hot_size", 512),
+    n_req, n_q = kw.get("requests", 16), kw.get("n_q", 2)
+    tabs = _mtp_tables(seed, n_req, K, T, ctx, (9, 1), n_q=n_q, p_hot=0.2, hot_size=kw.get("hot_size", 512),
                        hot_range=kw.get("hot_range", 8192))
-    return Workload("C4", seed, S, ROW_BYTES, 16, K, 2, T, tabs, [list(range(n_req))],
+    return Workload("C4", seed, S, ROW_BYTES, 16, K, n_q, T, tabs, [list(range(n_req))],
                     "%d requests, 1 Mi context, Beta(9,1) overlap, 20%% hot set" % n_req)
 
 

@@ -22,10 +22,13 @@
  *     of caller memory.  The context owns all state, the KV buffers and the
  *     scratch it needs; everything is allocated in avsg_create().
  *   - Calls on one context must not overlap in time (one stream at a time).
- *   - Kernel-side problems (a bounded loop that ran out, an index out of
- *     range) never fault: the kernel records a code in a status word that
- *     avsg_stats(), avsg_export_state() and avsg_sync_status() report as
- *     AVSG_EDEVICE_STATUS.
+ *   - Kernel-side problems (a bounded loop that ran out, a slot or segment
+ *     index out of range, an id beyond kv_rows or the direct index) never
+ *     fault: the kernel records a code in a status word that avsg_stats(),
+ *     avsg_export_state() and avsg_sync_status() report as
+ *     AVSG_EDEVICE_STATUS.  An id beyond a table's host rows is only caught
+ *     when the call states kv_rows: the library cannot know the extent of
+ *     the caller's host allocation otherwise.
  */
 #ifndef AVSG_H
 #define AVSG_H
@@ -50,8 +53,11 @@ extern "C" {
 #define AVSG_STATUS_NO_DEAD_SLOTS   0x02u /* fewer reclaimable slots than misses (Eq. 7)        */
 #define AVSG_STATUS_BAD_SLOT        0x04u /* a slot or position index out of range              */
 #define AVSG_STATUS_BAD_SEGMENT     0x08u /* Stage Two could not resolve a miss-list entry      */
-#define AVSG_STATUS_BAD_ID          0x10u /* direct index: id >= max_context (taken as padding) */
+#define AVSG_STATUS_BAD_ID          0x10u /* an id >= kv_rows of its table, or >= max_context
+                                             with the direct index (taken as padding)          */
 #define AVSG_STATUS_WAIT_TIMEOUT    0x20u /* overlapped Stage Two gave up waiting for Stage One */
+#define AVSG_STATUS_LAUNCH_FAILED   0x40u /* a Stage Two launch failed after Stage One had run:
+                                             slots were reserved whose rows were never copied  */
 
 /* How Stage Two moves the missed rows (Sec. 3.4; App. D strategies). */
 #define AVSG_XFER_SM_BALANCED   0u  /* miss list cut evenly over all SMs (the operator)  */
@@ -89,7 +95,7 @@ typedef struct avsg_ctx avsg_ctx;   /* opaque */
 
 typedef struct {
     uint32_t num_tables;     /* persistent tables, each with its own S-slot buffer      */
-    uint32_t buffer_slots;   /* S: power of two, 32 .. 8192                             */
+    uint32_t buffer_slots;   /* S: power of two, 32 .. 32768 (AVSG_INDEX_PAPER: .. 8192) */
     uint32_t row_bytes;      /* bytes per KV row, multiple of 16                        */
     uint32_t max_topk;       /* largest K of any step                                   */
     uint32_t max_tokens;     /* largest N_q = N_mtp + 1; max_tokens*max_topk <= S (Eq. 7) */
@@ -103,6 +109,11 @@ typedef struct {
                                 paper's default 3)                                       */
     uint32_t hash_a1;        /* AVSG_INDEX_PAPER: the two distinct odd primes of Eq. 9   */
     uint32_t hash_a2;        /*   (0 = 1000003 and 998244353; the paper names none)      */
+    uint32_t stage_one_cluster; /* thread blocks that share one table in Stage One: 0 = chosen by
+                                the library (one block while the table fits one SM's shared
+                                memory, i.e. S <= 8192; above that the smallest thread-block
+                                cluster that holds it), or 1, 2, 4, 8.  Same results.  Not with
+                                AVSG_INDEX_PAPER; needs S / cluster >= 32                */
 } avsg_config;
 
 typedef struct {
@@ -128,6 +139,12 @@ typedef struct {
                                       reads N when it runs, so that a call captured in a
                                       CUDA graph follows a sequence that grows between
                                       replays                                            */
+    const uint32_t *kv_rows;       /* HOST [n] or NULL: rows each table's host KV holds.
+                                      When given, an id >= kv_rows[i] is never fetched:
+                                      it is taken as padding (slot -1) and reported as
+                                      AVSG_STATUS_BAD_ID.  Without it ids are not checked
+                                      against the host allocation (the direct index still
+                                      bounds them by max_context)                        */
 } avsg_step_args;
 
 typedef struct {
@@ -158,7 +175,8 @@ typedef struct {
 /* App. E (a request starts with nothing cached), Sec. 3.1-3.2 (one S-slot
  * buffer plus S state entries per request): allocates all state, every table
  * empty (id -1) and dead (lifetime -1), buffers zeroed.  *out is set only on
- * success.  buffer_slots above 8192 needs AVSG_INDEX_DIRECT (see the field). */
+ * success.  Tables above 8192 slots are handled by a thread-block cluster
+ * per table (stage_one_cluster). */
 int avsg_create(const avsg_config *cfg, avsg_ctx **out);
 
 /* No passage of the paper: releases everything avsg_create allocated, after
@@ -307,6 +325,8 @@ typedef struct {
     uint8_t        *hit;           /* DEVICE out or NULL                                 */
     int32_t        *miss_count;    /* DEVICE out [n][n_tokens] or NULL                   */
     uint32_t       *status;        /* DEVICE out or NULL: 0, or the kernels' status bits */
+    const uint32_t *kv_rows;       /* HOST [n] or NULL: rows of each table's host KV; an
+                                      id at or beyond it is not fetched (see avsg_step_args) */
 } avsg_noalloc_args;
 
 int avsg_step_noalloc(const avsg_noalloc_args *args, void *cuda_stream);

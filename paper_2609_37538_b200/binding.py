@@ -20,6 +20,7 @@ XFER_SM_BALANCED, XFER_COPY_ENGINE, XFER_REQUEST_LEVEL, XFER_ALL_K, XFER_POSITIO
 INDEX_HASH, INDEX_DIRECT, INDEX_PAPER = 0, 1, 2
 STATUS_PROBE_EXHAUSTED, STATUS_NO_DEAD_SLOTS, STATUS_BAD_SLOT, STATUS_BAD_SEGMENT, STATUS_BAD_ID, STATUS_WAIT_TIMEOUT = (
     1, 2, 4, 8, 16, 32)
+STATUS_LAUNCH_FAILED = 64
 
 EXPORTS = (
     "avsg_create", "avsg_destroy", "avsg_reset", "avsg_reset_async", "avsg_step", "avsg_step_host", "avsg_buffer", "avsg_stats", "avsg_table_stats",
@@ -35,14 +36,15 @@ class AvsgConfig(ctypes.Structure):
                 ("max_topk", ctypes.c_uint32), ("max_tokens", ctypes.c_uint32), ("max_lifetime", ctypes.c_int32),
                 ("transfer_mode", ctypes.c_uint32), ("device", ctypes.c_int32), ("index_mode", ctypes.c_uint32),
                 ("max_context", ctypes.c_uint32), ("probe_retries", ctypes.c_uint32), ("hash_a1", ctypes.c_uint32),
-                ("hash_a2", ctypes.c_uint32)]
+                ("hash_a2", ctypes.c_uint32), ("stage_one_cluster", ctypes.c_uint32)]
 
 
 class AvsgStepArgs(ctypes.Structure):
     _fields_ = [("n", ctypes.c_uint32), ("table_ids", ctypes.c_void_p), ("n_tokens", ctypes.c_uint32),
                 ("topk", ctypes.c_uint32), ("indices", ctypes.c_void_p), ("kv_base", ctypes.c_void_p),
                 ("row_stride", ctypes.c_void_p), ("verified_len", ctypes.c_void_p), ("slots", ctypes.c_void_p),
-                ("hit", ctypes.c_void_p), ("miss_count", ctypes.c_void_p), ("verified_len_dev", ctypes.c_void_p)]
+                ("hit", ctypes.c_void_p), ("miss_count", ctypes.c_void_p), ("verified_len_dev", ctypes.c_void_p),
+                ("kv_rows", ctypes.c_void_p)]
 
 
 class AvsgStats(ctypes.Structure):
@@ -60,7 +62,7 @@ class AvsgNoAllocArgs(ctypes.Structure):
                 ("tok", ctypes.c_void_p), ("life", ctypes.c_void_p), ("buffer", ctypes.c_void_p),
                 ("indices", ctypes.c_void_p), ("kv_base", ctypes.c_void_p), ("row_stride", ctypes.c_void_p),
                 ("verified_len", ctypes.c_void_p), ("slots", ctypes.c_void_p), ("hit", ctypes.c_void_p),
-                ("miss_count", ctypes.c_void_p), ("status", ctypes.c_void_p)]
+                ("miss_count", ctypes.c_void_p), ("status", ctypes.c_void_p), ("kv_rows", ctypes.c_void_p)]
 
 
 NOALLOC_MAX_TABLES, NOALLOC_MAX_IDS = 32, 131072
@@ -163,7 +165,7 @@ class PreparedCall:
     """The argument block of one recurring call (same tables, same host KV): built once, re-used per step."""
 
     def __init__(self, ctx: "Context", table_ids: Sequence[int], kv: Sequence, n_tokens: int, topk: int,
-                 row_stride: Optional[Sequence[int]] = None):
+                 row_stride: Optional[Sequence[int]] = None, kv_rows: Optional[Sequence[int]] = None):
         n = len(table_ids)
         assert len(kv) == n
         self.ctx, self.n, self.n_tokens, self.topk = ctx, n, n_tokens, topk
@@ -172,12 +174,14 @@ class PreparedCall:
         self._kv = (ctypes.c_void_p * n)(*[_addr(k) for k in kv])
         self._stride = (ctypes.c_uint64 * n)(*[int(s) for s in row_stride]) if row_stride is not None else None
         self._vlen = (ctypes.c_int32 * n)()
+        self._rows = (ctypes.c_uint32 * n)(*[int(r) for r in kv_rows]) if kv_rows is not None else None
         a = AvsgStepArgs()
         a.n, a.n_tokens, a.topk = n, n_tokens, topk
         a.table_ids = ctypes.addressof(self._tids)
         a.kv_base = ctypes.addressof(self._kv)
         a.row_stride = ctypes.addressof(self._stride) if self._stride is not None else None
         a.verified_len = ctypes.addressof(self._vlen)
+        a.kv_rows = ctypes.addressof(self._rows) if self._rows is not None else None
         self.args = a
 
     def run(self, indices, verified_len: Sequence[int], slots, hit=None, miss_count=None, stream=None,
@@ -205,11 +209,11 @@ class Context:
     def __init__(self, num_tables: int, buffer_slots: int, row_bytes: int, max_topk: int, max_tokens: int = 1,
                  max_lifetime: int = 16, transfer_mode: int = XFER_SM_BALANCED, device: int = 0,
                  index_mode: int = INDEX_HASH, max_context: int = 0, probe_retries: int = 0, hash_a1: int = 0,
-                 hash_a2: int = 0):
+                 hash_a2: int = 0, stage_one_cluster: int = 0):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         cfg = AvsgConfig(num_tables, buffer_slots, row_bytes, max_topk, max_tokens, max_lifetime, transfer_mode,
-                         device, index_mode, max_context, probe_retries, hash_a1, hash_a2)
+                         device, index_mode, max_context, probe_retries, hash_a1, hash_a2, stage_one_cluster)
         _check(self._lib.avsg_create(ctypes.byref(cfg), ctypes.byref(self._h)), "avsg_create")
         self.num_tables, self.S, self.row_bytes = num_tables, buffer_slots, row_bytes
         self.max_topk, self.max_tokens, self.L, self.device = max_topk, max_tokens, max_lifetime, device
@@ -226,16 +230,16 @@ class Context:
             pass
 
     # -- the hot call ---------------------------------------------------------------------------------
-    def prepare(self, table_ids, kv, n_tokens: int, topk: int, row_stride=None) -> PreparedCall:
-        return PreparedCall(self, table_ids, kv, n_tokens, topk, row_stride)
+    def prepare(self, table_ids, kv, n_tokens: int, topk: int, row_stride=None, kv_rows=None) -> PreparedCall:
+        return PreparedCall(self, table_ids, kv, n_tokens, topk, row_stride, kv_rows)
 
     def step(self, table_ids, indices, kv, verified_len, row_stride=None, want_hit: bool = True,
-             want_miss_count: bool = True, stream=None) -> StepOutput:
+             want_miss_count: bool = True, stream=None, kv_rows=None) -> StepOutput:
         """One decode iteration. indices: int32 CUDA tensor [n, n_tokens, topk]. Returns device tensors."""
         import torch
         assert indices.is_cuda and indices.dtype == torch.int32 and indices.is_contiguous() and indices.dim() == 3
         n, n_q, K = indices.shape
-        call = PreparedCall(self, table_ids, kv, n_q, K, row_stride)
+        call = PreparedCall(self, table_ids, kv, n_q, K, row_stride, kv_rows)
         slots = torch.empty_like(indices)
         hit = torch.empty(indices.shape, dtype=torch.uint8, device=indices.device) if want_hit else None
         mc = torch.empty((n, n_q), dtype=torch.int32, device=indices.device) if want_miss_count else None
@@ -344,7 +348,7 @@ class Context:
 
 
 def step_noalloc(tok, life, buffer, indices, kv, verified_len, *, max_lifetime: int = 16, slots, hit=None,
-                 miss_count=None, status=None, row_stride=None, stream=None) -> None:
+                 miss_count=None, status=None, row_stride=None, stream=None, kv_rows=None) -> None:
     """avsg_step_noalloc: one decode iteration on caller-owned state, for callers that cannot allocate
     (an engine whose own pool holds all device memory, or a path where an allocation's device-wide
     synchronisation is not acceptable).  Every tensor is the caller's; the library allocates nothing and
@@ -370,4 +374,6 @@ def step_noalloc(tok, life, buffer, indices, kv, verified_len, *, max_lifetime: 
     a.hit = _addr(hit) if hit is not None else None
     a.miss_count = _addr(miss_count) if miss_count is not None else None
     a.status = _addr(status) if status is not None else None
+    rows = (ctypes.c_uint32 * n)(*[int(r) for r in kv_rows]) if kv_rows is not None else None
+    a.kv_rows = ctypes.addressof(rows) if rows is not None else None
     _check(load_library().avsg_step_noalloc(ctypes.byref(a), _stream_handle(stream)), "avsg_step_noalloc")

@@ -15,6 +15,8 @@ using namespace avsg;
 struct avsg_ctx {
     avsg_config cfg;
     uint32_t logS = 0, logH = 0;
+    uint32_t s1_cluster = 1;           // blocks that share one table in Stage One (1 = the single-block kernel)
+    uint32_t host_status = 0;          // status bits raised on the host side (sticky like the device word)
     uint32_t list_stride = 0;          // entries per miss-list segment
     int sm_count = 0;
     uint32_t xfer_blocks = 0, xfer_threads = 256;
@@ -52,6 +54,7 @@ struct avsg_ctx {
     std::vector<uint32_t> seen;                // distinctness check of table ids
     uint32_t epoch = 0;
     std::vector<const void*> call_kv_host;     // host pointers of the current call (copy-engine mode)
+    std::vector<uint64_t> call_kv_dev;         // their device-visible addresses, resolved before anything is launched
     cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
     // avsg_step_host: the outputs go back on a side stream while Stage Two runs
     cudaStream_t side = nullptr;
@@ -143,6 +146,7 @@ int check_args(avsg_ctx* c, const avsg_step_args* a)
         c->seen[t] = c->epoch;
         if (a->row_stride && (a->row_stride[i] % 16 || a->row_stride[i] < c->cfg.row_bytes)) return AVSG_EINVAL;
         if (!a->kv_base[i] || (reinterpret_cast<uint64_t>(a->kv_base[i]) & 15u)) return AVSG_EINVAL;
+        if (a->kv_rows && a->kv_rows[i] > 0x80000000u) return AVSG_EINVAL;
     }
     return AVSG_OK;
 }
@@ -224,6 +228,18 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
     }
 
     c->call_kv_host.assign(a->kv_base, a->kv_base + n);
+    // every host KV base is resolved (and refused, if the GPU cannot read it) before the first launch of the call:
+    // a call either starts completely or not at all
+    c->call_kv_dev.resize(n);
+    for (uint32_t i = 0; i < n; ++i)
+        if ((rc = resolve_kv(c, a->table_ids[i], a->kv_base[i], &c->call_kv_dev[i])) != AVSG_OK) return rc;
+    // ids at or beyond this are never looked up or fetched: the table's host rows when the caller states them,
+    // and the size of the direct index
+    auto id_limit_of = [&](uint32_t i) -> uint32_t {
+        uint32_t lim = a->kv_rows ? a->kv_rows[i] : 0x80000000u;
+        if (c->d_where && c->cfg.max_context < lim) lim = c->cfg.max_context;
+        return lim;
+    };
     // Stage One for tables [first, first + cnt) of the call, with the small or the large argument block
     auto stage_one = [&](auto& p, uint32_t first, uint32_t cnt) -> int {
         p.tok = c->d_tok; p.life = c->d_life; p.buffer = c->d_buffer; p.stats = c->d_stats;
@@ -241,16 +257,18 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         p.ready = overlap ? c->d_ready : nullptr;
         p.tcount = overlap ? c->d_tcount : nullptr;
         p.done_seq = wait_on_sequence ? c->d_ready + OVERLAP_MAX_TOKENS + 1 : nullptr;
+        p.done_ctr = reinterpret_cast<uint32_t*>(c->d_ready + OVERLAP_MAX_TOKENS + 2);
         p.host_seq = wait_on_sequence ? c->host_seq + 1 : 0;
         p.expect = n;
         for (uint32_t i = 0; i < cnt; ++i) {
             p.table_id[i] = a->table_ids[first + i];
             p.verified_len[i] = a->verified_len ? a->verified_len[first + i] : 0;
-            const int r = resolve_kv(c, p.table_id[i], a->kv_base[first + i], &p.kv_base[i]);
-            if (r != AVSG_OK) return r;
+            p.id_limit[i] = id_limit_of(first + i);
+            p.kv_base[i] = c->call_kv_dev[first + i];
             p.kv_stride[i] = a->row_stride ? a->row_stride[first + i] : c->cfg.row_bytes;
         }
-        CU(launch_stage_one(p, cnt, stream));
+        if (c->s1_cluster > 1) CU(launch_stage_one_cluster(p, cnt, c->s1_cluster, stream));
+        else CU(launch_stage_one(p, cnt, stream));
         return AVSG_OK;
     };
     for (uint32_t first = 0; first < n; first += chunk) {
@@ -259,11 +277,13 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
             AllKParams p;
             p.indices = indices; p.slots = slots; p.hit = hit; p.miss_count = miss_count;
             p.miss_list = c->d_list; p.seg = c->d_seg; p.stats = c->d_stats; p.buffer = c->d_buffer;
+            p.status = c->d_status;
             p.S = c->cfg.buffer_slots; p.row_bytes = c->cfg.row_bytes; p.K = K; p.n_q = n_q;
             p.first = first; p.list_stride = c->list_stride;
             for (uint32_t i = 0; i < cnt; ++i) {
                 p.table_id[i] = a->table_ids[first + i];
-                if ((rc = resolve_kv(c, p.table_id[i], a->kv_base[first + i], &p.kv_base[i])) != AVSG_OK) return rc;
+                p.id_limit[i] = id_limit_of(first + i);
+                p.kv_base[i] = c->call_kv_dev[first + i];
                 p.kv_stride[i] = a->row_stride ? a->row_stride[first + i] : c->cfg.row_bytes;
             }
             CU(launch_all_k_prepare(p, cnt, stream));
@@ -308,7 +328,15 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         x.n = n; x.n_q = n_q; x.list_stride = c->list_stride; x.row_bytes = c->cfg.row_bytes; x.S = c->cfg.buffer_slots;
         x.expect = n;
         x.t_range = c->timing ? c->d_trange + 2 : nullptr;
-        CU(launch_transfer_overlap(x, c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count, c->xfer_threads, stream));
+        if (launch_transfer_overlap(x, c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count, c->xfer_threads, stream)
+            != cudaSuccess) {
+            // Stage One has run and raised the per-token counters, nothing will lower them: do it here, in
+            // stream order, and remember that this call reserved slots whose rows were never copied
+            cudaGetLastError();
+            cudaMemsetAsync(c->d_ready, 0, (OVERLAP_MAX_TOKENS + 1) * sizeof(unsigned long long), stream);
+            c->host_status |= AVSG_STATUS_LAUNCH_FAILED;
+            return AVSG_ECUDA;
+        }
         if (wait_on_sequence) {
             c->host_seq += 1;
             if (c->wait_value64(c->side, reinterpret_cast<CUdeviceptr>(c->d_ready + OVERLAP_MAX_TOKENS + 1), c->host_seq,
@@ -323,7 +351,11 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         x.request_level = mode == AVSG_XFER_REQUEST_LEVEL; x.S = c->cfg.buffer_slots;
         x.t_range = c->timing ? c->d_trange + 2 : nullptr;
         const uint32_t blocks = x.request_level ? n : (c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count);
-        CU(launch_transfer(x, blocks, c->xfer_threads, stream));
+        if (launch_transfer(x, blocks, c->xfer_threads, stream) != cudaSuccess) {
+            cudaGetLastError();
+            c->host_status |= AVSG_STATUS_LAUNCH_FAILED;
+            return AVSG_ECUDA;
+        }
     }
     if (c->timing) {
         if (mode == AVSG_XFER_SM_OVERLAP) CU(cudaEventRecord(c->ev[1], stream));
@@ -339,6 +371,7 @@ int read_status(avsg_ctx* c, uint32_t* word)
 {
     uint32_t st = 0;
     CU(cudaMemcpy(&st, c->d_status, sizeof(st), cudaMemcpyDeviceToHost));
+    st |= c->host_status;
     if (word) *word = st;
     return st ? AVSG_EDEVICE_STATUS : AVSG_OK;
 }
@@ -351,7 +384,9 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
 {
     if (!cfg || !out) return AVSG_EINVAL;
     if (cfg->num_tables == 0 || !is_pow2(cfg->buffer_slots) || cfg->buffer_slots < 32) return AVSG_EINVAL;
-    if (cfg->buffer_slots > 8192) return AVSG_EUNSUPPORTED;
+    if (cfg->buffer_slots > 32768) return AVSG_EUNSUPPORTED;
+    if (cfg->stage_one_cluster > 8 || (cfg->stage_one_cluster & (cfg->stage_one_cluster - 1))) return AVSG_EINVAL;
+    if (cfg->max_topk > 32768) return AVSG_EUNSUPPORTED;
     if (cfg->row_bytes == 0 || cfg->row_bytes % 16) return AVSG_EINVAL;
     if (cfg->max_topk == 0 || cfg->max_tokens == 0) return AVSG_EINVAL;
     if (cfg->max_lifetime < 1 || cfg->max_lifetime > 126) return AVSG_EINVAL;
@@ -378,14 +413,28 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     int max_smem = 0;
     cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, cfg->device);
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, cfg->device);
-    const size_t need = cfg->index_mode == AVSG_INDEX_PAPER
-        ? stage_one_paper_smem_bytes(cfg->buffer_slots, cfg->max_topk, (uint32_t)cfg->max_lifetime)
-        : stage_one_smem_bytes(cfg->buffer_slots, cfg->max_topk, (uint32_t)cfg->max_lifetime,
-                               cfg->index_mode == AVSG_INDEX_DIRECT);
-    if (need > (size_t)max_smem) { delete c; return AVSG_EUNSUPPORTED; }
-    // always raise the kernel's dynamic shared-memory limit to the device maximum: the attribute is
+    // Blocks per table in Stage One: what the configuration asks for, else the single-block kernel while the table
+    // fits one SM's shared memory and the smallest cluster that holds it above that.
+    {
+        const bool direct = cfg->index_mode == AVSG_INDEX_DIRECT;
+        const uint32_t S = cfg->buffer_slots, K = cfg->max_topk, L = (uint32_t)cfg->max_lifetime;
+        auto fits = [&](uint32_t C) -> bool {
+            if (cfg->index_mode == AVSG_INDEX_PAPER)
+                return C == 1 && S <= 8192 && stage_one_paper_smem_bytes(S, K, L) <= (size_t)max_smem;
+            if (C == 1) return S <= 8192 && stage_one_smem_bytes(S, K, L, direct) <= (size_t)max_smem;
+            return S / C >= 32 && S / C <= 8192 && stage_one_cluster_smem_bytes(S, K, L, C, direct) <= (size_t)max_smem;
+        };
+        uint32_t C = cfg->stage_one_cluster;
+        if (C == 0)
+            for (C = 1; C <= 8 && !fits(C); C *= 2) {}
+        if (C > 8 || !fits(C)) { delete c; return AVSG_EUNSUPPORTED; }
+        c->s1_cluster = C;
+    }
+    // always raise the kernels' dynamic shared-memory limit to the device maximum: the attribute is
     // per function, so a context with a small table must not lower it under a context with a large one
-    if (stage_one_prepare((size_t)max_smem) != cudaSuccess) { delete c; return AVSG_ECUDA; }
+    if (stage_one_prepare((size_t)max_smem) != cudaSuccess || stage_one_cluster_prepare((size_t)max_smem) != cudaSuccess) {
+        delete c; return AVSG_ECUDA;
+    }
 
     const size_t n_ids = T * c->list_stride;
     bool ok = true;
@@ -394,7 +443,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaMalloc(&c->d_buffer, T * S * cfg->row_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_stats, T * sizeof(TableStats)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_trange, 8 * sizeof(unsigned long long)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->d_ready, (OVERLAP_MAX_TOKENS + 2) * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_ready, (OVERLAP_MAX_TOKENS + 3) * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_tcount, (size_t)OVERLAP_MAX_TABLES * OVERLAP_MAX_TOKENS * sizeof(uint32_t)) == cudaSuccess;
     c->big_args = new (std::nothrow) S1ParamsBig();
     ok = ok && c->big_args != nullptr;
@@ -438,7 +487,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
         const unsigned long long never = ~0ull, init[8] = {never, 0, never, 0, never, 0, never, 0};
         c->d_trange_init = c->d_trange + 4;
         if (cudaMemcpy(c->d_trange, init, sizeof(init), cudaMemcpyHostToDevice) != cudaSuccess ||
-            cudaMemset(c->d_ready, 0, (OVERLAP_MAX_TOKENS + 2) * sizeof(unsigned long long)) != cudaSuccess) {
+            cudaMemset(c->d_ready, 0, (OVERLAP_MAX_TOKENS + 3) * sizeof(unsigned long long)) != cudaSuccess) {
             free_all(c); delete c; return AVSG_ECUDA;
         }
     }
@@ -577,6 +626,8 @@ int avsg_clear_status(avsg_ctx* c)
     CU(cudaMemset(c->d_status, 0, sizeof(uint32_t)));
     // a transfer kernel that gave up may have left the per-token counters of the overlapped mode raised
     CU(cudaMemset(c->d_ready, 0, (OVERLAP_MAX_TOKENS + 1) * sizeof(unsigned long long)));    // not the sequence word
+    CU(cudaMemset(c->d_ready + OVERLAP_MAX_TOKENS + 2, 0, sizeof(unsigned long long)));      // arrivals after the last token
+    c->host_status = 0;
     return AVSG_OK;
 }
 

@@ -12,7 +12,7 @@ enum : uint32_t {
     ST_NO_DEAD_SLOTS   = 1u << 1,   // fewer reclaimable slots than misses (Eq. 7 violated)
     ST_BAD_SLOT        = 1u << 2,   // slot / position index out of range
     ST_BAD_SEGMENT     = 1u << 3,   // transfer kernel could not resolve a miss
-    ST_BAD_ID          = 1u << 4,   // direct index: an id beyond max_context (treated as padding)
+    ST_BAD_ID          = 1u << 4,   // an id beyond the table's host rows or the direct index (treated as padding)
     ST_WAIT_TIMEOUT    = 1u << 5,   // overlapped Stage Two: a bounded wait for Stage One ran out
 };
 
@@ -103,11 +103,13 @@ struct S1ParamsT {
     // calls with host buffers in that mode (null otherwise): the table that places the call's last token last
     // writes the call's sequence number to *done_seq, which the output download waits for
     unsigned long long* done_seq = nullptr;
+    uint32_t*           done_ctr = nullptr;     // arrivals after the call's last token; wraps to zero at `expect`
     unsigned long long  host_seq = 0;
     uint32_t            expect = 0;             // tables of the call
     const int32_t* verified_len_dev = nullptr;  // [n] of the call: read instead of verified_len[] when set
     uint32_t table_id[CAP];
     int32_t  verified_len[CAP];
+    uint32_t id_limit[CAP];      // ids >= this are not looked up or fetched (host rows of the table; direct index size)
     uint64_t kv_base[CAP];
     uint64_t kv_stride[CAP];
 };
@@ -157,8 +159,10 @@ struct AllKParams {
     SegDesc*       seg;
     TableStats*    stats;
     uint8_t*       buffer;
+    uint32_t*      status;
     uint32_t S, row_bytes, K, n_q, first, list_stride;
     uint32_t table_id[S1_MAX_TABLES];
+    uint32_t id_limit[S1_MAX_TABLES];
     uint64_t kv_base[S1_MAX_TABLES];
     uint64_t kv_stride[S1_MAX_TABLES];
 };
@@ -177,6 +181,12 @@ uint32_t stage_one_threads(uint32_t S, uint32_t K);
 cudaError_t stage_one_prepare(size_t max_smem);
 cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream);
 cudaError_t launch_stage_one(const S1ParamsBig& p, uint32_t n_tables, cudaStream_t stream);   // hash / direct index only
+// Stage One with one table per thread-block cluster of C blocks (C = 2, 4 or 8; hash / direct index only)
+uint32_t stage_one_cluster_threads(uint32_t S, uint32_t C);
+size_t stage_one_cluster_smem_bytes(uint32_t S, uint32_t K, uint32_t L, uint32_t C, bool direct);
+cudaError_t stage_one_cluster_prepare(size_t max_smem);
+cudaError_t launch_stage_one_cluster(const S1Params& p, uint32_t n_tables, uint32_t C, cudaStream_t stream);
+cudaError_t launch_stage_one_cluster(const S1ParamsBig& p, uint32_t n_tables, uint32_t C, cudaStream_t stream);
 cudaError_t launch_direct_index_from_state(const int32_t* tok, uint16_t* where, uint32_t first_table, uint32_t n_tables,
                                            uint32_t S, uint32_t max_context, cudaStream_t stream);
 cudaError_t launch_all_k_prepare(const AllKParams& p, uint32_t n_tables, cudaStream_t stream);

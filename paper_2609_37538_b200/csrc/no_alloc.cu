@@ -101,6 +101,8 @@ extern "C" int avsg_step_noalloc(const avsg_noalloc_args* a, void* cuda_stream)
         const void* base = a->kv_base[i];
         if (!base || (reinterpret_cast<uint64_t>(base) & 15u)) return AVSG_EINVAL;
         if (a->row_stride && (a->row_stride[i] % 16 || a->row_stride[i] < a->row_bytes)) return AVSG_EINVAL;
+        if (a->kv_rows && a->kv_rows[i] > 0x80000000u) return AVSG_EINVAL;
+        p.id_limit[i] = a->kv_rows ? a->kv_rows[i] : 0x80000000u;
         cudaPointerAttributes at;
         if (cudaPointerGetAttributes(&at, base) != cudaSuccess) { cudaGetLastError(); return AVSG_EINVAL; }
         if (at.type == cudaMemoryTypeUnregistered || !at.devicePointer) return AVSG_EINVAL;

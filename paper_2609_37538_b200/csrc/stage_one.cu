@@ -36,17 +36,10 @@
 // When Stage Two overlaps Stage One (S1Params::ready set), the block announces
 // every token as soon as its misses are placed: see publish_token().
 #include "avsg_kernels.cuh"
+#include "stage_one_common.cuh"
 
 namespace avsg {
 namespace {
-
-constexpr int32_t EMPTY = -1;
-constexpr int32_t PRIV_HIST_MAX_L = 30;   // private byte-counter histogram up to this L (32 rows)
-
-__device__ __forceinline__ uint32_t hash_id(int32_t x, uint32_t logH)
-{
-    return ((uint32_t)x * 2654435769u) >> (32u - logH);
-}
 
 struct Index {
     int32_t*  key;
@@ -82,34 +75,6 @@ __device__ __forceinline__ void index_insert(const Index& ix, int32_t x, uint32_
         b = (b + 1u) & ix.mask;
     }
     atomicOr(status, ST_PROBE_EXHAUSTED);
-}
-
-// The lifetimes of the slots a thread owns, packed one signed byte each into
-// two words; unused lanes carry 0x7F (never counted, never dead).
-__device__ __forceinline__ void life_load(const int8_t* base, uint32_t j0, uint32_t spt, bool own,
-                                          uint32_t& w0, uint32_t& w1)
-{
-    w0 = w1 = 0x7F7F7F7Fu;
-    if (!own) return;
-    if (spt == 8) { const uint2 v = *reinterpret_cast<const uint2*>(base + j0); w0 = v.x; w1 = v.y; }
-    else if (spt == 4) { w0 = *reinterpret_cast<const uint32_t*>(base + j0); }
-    else if (spt == 2) { w0 = 0x7F7F0000u | *reinterpret_cast<const uint16_t*>(base + j0); }
-    else { w0 = 0x7F7F7F00u | (uint8_t)base[j0]; }
-}
-
-__device__ __forceinline__ void life_store(int8_t* base, uint32_t j0, uint32_t spt, bool own, uint32_t w0, uint32_t w1)
-{
-    if (!own) return;
-    if (spt == 8) { *reinterpret_cast<uint2*>(base + j0) = make_uint2(w0, w1); }
-    else if (spt == 4) { *reinterpret_cast<uint32_t*>(base + j0) = w0; }
-    else if (spt == 2) { *reinterpret_cast<uint16_t*>(base + j0) = (uint16_t)w0; }
-    else { base[j0] = (int8_t)(w0 & 0xFFu); }
-}
-
-// life <- max(life - d, -1) on four packed signed bytes
-__device__ __forceinline__ uint32_t decay4(uint32_t w, uint32_t d)
-{
-    return __vmaxs4(__vsubss4(w, d * 0x01010101u), 0xFFFFFFFFu);
 }
 
 // Inserts the ids of the slots a thread owns.  The first compare-and-swap of every id is issued
@@ -148,102 +113,6 @@ __device__ __forceinline__ void build_index(const Index& ix, const int32_t* s_to
     }
     live = __reduce_add_sync(0xffffffffu, live);
     if ((threadIdx.x & 31u) == 0 && live) atomicAdd(s_fill, live);
-}
-
-// The ids a thread handles for one token: positions i0 .. i0+ipt-1.
-__device__ __forceinline__ void load_ids(const int32_t* X, uint32_t i0, uint32_t ipt, uint32_t K, int32_t (&xs)[MAX_IPT])
-{
-    if ((ipt & 3u) == 0 && (K & 3u) == 0 && ((reinterpret_cast<uintptr_t>(X) & 15u) == 0)) {
-#pragma unroll
-        for (uint32_t q = 0; q < (uint32_t)MAX_IPT / 4; ++q) {
-            if (4 * q < ipt && i0 + 4 * q < K) {
-                const int4 v = __ldg(reinterpret_cast<const int4*>(X + i0) + q);
-                xs[4 * q] = v.x; xs[4 * q + 1] = v.y; xs[4 * q + 2] = v.z; xs[4 * q + 3] = v.w;
-            }
-        }
-    } else if (ipt == 2 && (K & 1u) == 0 && ((reinterpret_cast<uintptr_t>(X) & 7u) == 0)) {
-        if (i0 < K) {
-            const int2 v = __ldg(reinterpret_cast<const int2*>(X + i0));
-            xs[0] = v.x; xs[1] = v.y;
-        }
-    } else {
-#pragma unroll
-        for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k)
-            if (k < ipt && i0 + k < K) xs[k] = __ldg(X + i0 + k);
-    }
-}
-
-// Lifetime histogram of the table: s_hist[v + 1] = number of slots with lifetime v, v = -1 .. L.
-// s_hist must be zero on entry.  w0/w1 are the thread's packed lifetimes (life_load).
-__device__ __forceinline__ void count_lifetimes(uint32_t w0, uint32_t w1, uint32_t spt, bool own, int32_t L,
-                                                uint8_t* s_priv, uint32_t priv_stride, uint32_t* s_hist)
-{
-    const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31u;
-    if (s_priv) {
-        // private byte counters: row = lifetime value + 1, column = thread; no atomics
-        if (own) {
-#pragma unroll
-            for (uint32_t k = 0; k < (uint32_t)MAX_SPT; ++k) {
-                if (k < spt) {
-                    const uint32_t byte = ((k < 4 ? w0 >> (8 * k) : w1 >> (8 * (k - 4))) + 1u) & 0xFFu;   // value + 1
-                    s_priv[byte * priv_stride + tid] += 1;
-                }
-            }
-        }
-        __syncthreads();
-        // one warp per row: sum nt byte counters with dp4a and clear them for the next use
-        const uint32_t words = nt >> 2;
-        for (uint32_t row = tid >> 5; row <= (uint32_t)L + 1u; row += nt >> 5) {
-            uint32_t* r = reinterpret_cast<uint32_t*>(s_priv + row * priv_stride);
-            uint32_t acc = 0;
-            for (uint32_t i = lane; i < words; i += 32u) {
-                acc = __dp4a(r[i], 0x01010101u, acc);
-                r[i] = 0;
-            }
-            acc = __reduce_add_sync(0xffffffffu, acc);
-            if (lane == 0) s_hist[row] = acc;
-        }
-    } else {
-        for (int32_t v = -1; v <= L; ++v) {
-            const uint32_t vv = (uint32_t)(v & 0xFF) * 0x01010101u;
-            uint32_t c = (__popc(__vcmpeq4(w0, vv)) + __popc(__vcmpeq4(w1, vv))) >> 3;
-            c = __reduce_add_sync(0xffffffffu, c);
-            if (lane == 0 && c) atomicAdd(&s_hist[v + 1], c);
-        }
-    }
-}
-
-// Overlapped Stage Two only (p.ready set): tells the transfer kernel, which is already resident, that token g of
-// this table is placed - `count` more entries of the table's miss list are final.  Called by every thread of the
-// block: the block meets after its list writes; one thread then fences (the barrier makes the fence cover the whole
-// block's earlier writes, as in a grid-wide barrier) and raises the counter of token g.
-template <typename P>
-__device__ __forceinline__ void publish_token(const P& p, uint32_t ti, uint32_t table, uint32_t g, uint32_t count)
-{
-    if (!p.ready) return;
-    const uint32_t tid = threadIdx.x;
-    if (tid == 0) {
-        p.tcount[(size_t)ti * p.n_q + g] = count;
-        if (g == 0) {
-            SegDesc sd;
-            sd.src_base = p.kv_base[blockIdx.x];
-            sd.src_stride = p.kv_stride[blockIdx.x];
-            sd.dst_base = reinterpret_cast<uint64_t>(p.buffer + (size_t)table * p.S * p.row_bytes);
-            sd.count = 0;
-            sd.pad = 0;
-            p.seg[ti] = sd;
-        }
-    }
-    __syncthreads();
-    if (tid == 0) {
-        __threadfence();
-        const unsigned long long before = atomicAdd(p.ready + g, 1ull);
-        if (p.done_seq && g + 1 == p.n_q && before + 1ull == p.expect) {
-            // every table of the call has written its slot table, hit mask and miss counts
-            __threadfence();
-            *reinterpret_cast<volatile unsigned long long*>(p.done_seq) = p.host_seq;
-        }
-    }
 }
 
 template <bool DIRECT, int CAP>
@@ -307,6 +176,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
     life_load(g_life, j0, spt, own, lw0, lw1);
     int32_t xs[MAX_IPT];
     load_ids(p.indices + (size_t)ti * p.n_q * K, i0, ipt, K, xs);
+    const uint32_t id_limit = p.id_limit[blockIdx.x];
 
     if constexpr (!DIRECT) {
         for (uint32_t i = tid; i < H / 4; i += nt)
@@ -350,14 +220,12 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
         // ---- Probe, refresh hits to L, emit hit slots (Pass 1 + Pass 2) ----
         uint32_t missmask = 0, nmiss = 0, nvalid = 0;
         uint32_t cand[MAX_IPT];                             // direct index: candidate slot per id
+        check_ids(xs, i0, ipt, K, id_limit, p.status);      // out-of-range ids become padding (id_limit <= max_context)
         if (DIRECT) {
 #pragma unroll
             for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {   // all loads are issued before any is used
                 cand[k] = 0xFFFFFFFFu;
-                if (k < ipt && i0 + k < K && xs[k] >= 0) {
-                    if ((uint32_t)xs[k] < p.max_context) cand[k] = __ldcg(where + xs[k]) & (S - 1u);
-                    else atomicOr(p.status, ST_BAD_ID);
-                }
+                if (k < ipt && i0 + k < K && xs[k] >= 0) cand[k] = __ldcg(where + xs[k]) & (S - 1u);
             }
         }
 #pragma unroll
@@ -401,7 +269,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
         // the next token's ids travel while this token's misses are placed
         if (g + 1 < p.n_q) load_ids(p.indices + row + K, i0, ipt, K, xs);
         if (tid == 0 && p.miss_count) p.miss_count[(size_t)ti * p.n_q + g] = (int32_t)n_g;
-        if (n_g == 0) { __syncthreads(); publish_token(p, ti, table, g, 0); continue; }
+        if (n_g == 0) { __syncthreads(); publish_token(p, ti, table, g, 0, blockIdx.x); continue; }
         __syncthreads();
 
         // ---- Pass 3: CollectDead; if fewer than n_g slots are dead, decay until enough are ----
@@ -475,7 +343,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
             __syncthreads();
             fill_bound = *s_fill;
         }
-        publish_token(p, ti, table, g, n_take);
+        publish_token(p, ti, table, g, n_take, blockIdx.x);
     }
 
     // ---- write the table back; speculative entries (id >= N) become empty (Alg. 4) ----
@@ -649,6 +517,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_paper_kernel(const __g
 
         // ---- Probe (Eq. 8-11): at most R + 1 buckets; the full id is compared ----
         uint32_t missmask = 0, nmiss = 0, nvalid = 0;
+        check_ids(xs, i0, ipt, K, p.id_limit[blockIdx.x], p.status);
 #pragma unroll
         for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {
             const uint32_t i = i0 + k;
@@ -693,7 +562,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_paper_kernel(const __g
         }
         if (g + 1 < p.n_q) load_ids(p.indices + row + K, i0, ipt, K, xs);
         if (tid == 0 && p.miss_count) p.miss_count[(size_t)ti * p.n_q + g] = (int32_t)n_g;
-        if (n_g == 0) { __syncthreads(); publish_token(p, ti, table, g, 0); continue; }
+        if (n_g == 0) { __syncthreads(); publish_token(p, ti, table, g, 0, blockIdx.x); continue; }
         __syncthreads();
 
         // ---- CollectDead / decay until n_g slots are dead ----
@@ -775,7 +644,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_paper_kernel(const __g
         list_off += n_take;
         sum_decay += d;
         __syncthreads();
-        publish_token(p, ti, table, g, n_take);
+        publish_token(p, ti, table, g, n_take, blockIdx.x);
     }
 
     // ---- write back; speculative entries (id >= N) become empty ----
@@ -821,7 +690,11 @@ __global__ void __launch_bounds__(256) avsg_all_k_prepare_kernel(const __grid_co
     int2* list = p.miss_list + (size_t)ti * p.list_stride + (size_t)g * K;
     uint32_t valid = 0;
     for (uint32_t i = threadIdx.x; i < K; i += blockDim.x) {
-        const int32_t x = __ldg(p.indices + row + i);
+        int32_t x = __ldg(p.indices + row + i);
+        if (x >= 0 && (uint32_t)x >= p.id_limit[b]) {             // beyond the table's host rows: not fetched
+            atomicOr(p.status, ST_BAD_ID);
+            x = -1;
+        }
         const int32_t o = x >= 0 ? (int32_t)(g * K + i) : -1;
         p.slots[row + i] = o;
         if (p.hit) p.hit[row + i] = 0;

@@ -31,7 +31,7 @@ class HostKV:
 def run_parity(w: tr.Workload, *, tables: Optional[Sequence[int]] = None, mode: int = 0, host_io: bool = False,
                row_stride: Optional[int] = None, buffer_every: int = 1, oracle_tables: Optional[Sequence[int]] = None,
                n_iters: Optional[int] = None, threads: Optional[int] = None, xfer_geometry=None,
-               index_mode: int = 0, permute_seed: Optional[int] = None) -> Dict:
+               index_mode: int = 0, permute_seed: Optional[int] = None, cluster: int = 0) -> Dict:
     """Steps every call group of w for every iteration on the GPU; the tables in oracle_tables (default: all)
     are stepped by the oracle too and compared after EVERY step: hit mask, slot table, miss counts, (tok, life);
     the buffer rows every buffer_every iterations and at the end.  With permute_seed the K positions of every token
@@ -57,7 +57,8 @@ def run_parity(w: tr.Workload, *, tables: Optional[Sequence[int]] = None, mode: 
     local = {ti: k for k, ti in enumerate(ids)}                  # context table id of a workload table
     ctx = avsg.Context(num_tables=len(ids), buffer_slots=w.buffer_slots, row_bytes=w.row_bytes, max_topk=w.topk,
                        max_tokens=w.n_q, max_lifetime=w.max_lifetime, transfer_mode=mode, device=0,
-                       index_mode=index_mode, max_context=max(c.context for c in w.tables) + w.n_q)
+                       index_mode=index_mode, max_context=max(c.context for c in w.tables) + w.n_q,
+                       stage_one_cluster=cluster)
     if xfer_geometry:
         ctx.set_transfer_geometry(*xfer_geometry)
     orc = {ti: OracleTable(w.buffer_slots, w.row_bytes, w.max_lifetime) for ti in ids if ti in check}

@@ -25,9 +25,10 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_layouts_match_the_header():
-    assert ctypes.sizeof(avsg.AvsgConfig) == 52
-    assert ctypes.sizeof(avsg.AvsgStepArgs) == 88
+    assert ctypes.sizeof(avsg.AvsgConfig) == 56
+    assert ctypes.sizeof(avsg.AvsgStepArgs) == 96
     assert ctypes.sizeof(avsg.AvsgStats) == 88
+    assert ctypes.sizeof(avsg.AvsgNoAllocArgs) == 120
 
 
 def test_error_strings_and_argument_errors_need_no_gpu():
@@ -43,8 +44,10 @@ def test_error_strings_and_argument_errors_need_no_gpu():
     assert lib.avsg_create(ctypes.byref(bad), ctypes.byref(h)) == avsg.EINVAL
     bad = avsg.AvsgConfig(1, 1024, 656, 600, 2, 16, 0, 0)           # Eq. 7: 2 * 600 > 1024
     assert lib.avsg_create(ctypes.byref(bad), ctypes.byref(h)) == avsg.ECAPACITY
-    bad = avsg.AvsgConfig(1, 16384, 656, 2048, 2, 16, 0, 0)
+    bad = avsg.AvsgConfig(1, 65536, 656, 2048, 2, 16, 0, 0)         # more slots than a cluster holds
     assert lib.avsg_create(ctypes.byref(bad), ctypes.byref(h)) == avsg.EUNSUPPORTED
+    bad = avsg.AvsgConfig(1, 1024, 656, 16, 1, 16, 0, 0, 0, 0, 0, 0, 0, 3)       # cluster size not a power of two
+    assert lib.avsg_create(ctypes.byref(bad), ctypes.byref(h)) == avsg.EINVAL
     bad = avsg.AvsgConfig(1, 1024, 656, 16, 1, 200, 0, 0)
     assert lib.avsg_create(ctypes.byref(bad), ctypes.byref(h)) == avsg.EINVAL
     assert lib.avsg_step(None, None, None) == avsg.EINVAL

@@ -160,6 +160,49 @@ def test_unsorted_ids_differ_from_sorted(avsg):
     assert slot_of_a != slot_of_b
 
 
+# ---- Stage One across a thread-block cluster: the small shapes with forced cluster sizes, and tables above 8192
+# ---- slots, which only a cluster holds -----------------------------------------------------------------------
+@pytest.mark.parametrize("name,kw", SHAPES)
+@pytest.mark.parametrize("cluster", [2, 4, 8])
+@pytest.mark.parametrize("index", ["INDEX_HASH", "INDEX_DIRECT"])
+def test_cluster_shapes(avsg, name, kw, cluster, index):
+    w = tr.workload(name, **kw)
+    if w.buffer_slots // cluster < 32:
+        with pytest.raises(avsg.AvsgError) as e:
+            _parity(w, cluster=cluster, index_mode=getattr(avsg, index))
+        assert e.value.code == avsg.EUNSUPPORTED
+        return
+    mode = avsg.XFER_SM_OVERLAP if cluster == 4 else avsg.XFER_SM_BALANCED
+    _parity(w, cluster=cluster, index_mode=getattr(avsg, index), mode=mode, permute_seed=3 if cluster == 2 else None)
+
+
+BIG_TABLES = [
+    ("C2", dict(topk=2048, n_q=4, buffer_slots=16384, n_iters=14, context=131072)),           # MTP-3, S = 2 N_q K
+    ("C2", dict(topk=4096, n_q=2, buffer_slots=16384, n_iters=14, context=131072)),
+    ("C3", dict(topk=2048, n_q=4, buffer_slots=16384, n_iters=8, context=65536, requests=5, layers=2)),
+    ("C2", dict(topk=8192, n_q=2, buffer_slots=16384, n_iters=6, context=131072)),            # S = N_q K
+    ("C2", dict(topk=4096, n_q=4, buffer_slots=32768, n_iters=8, context=131072)),
+    ("C5", dict(topk=32768, buffer_slots=32768, n_iters=4, requests=2, ctx_lo=70000, ctx_hi=120000)),   # K = S = max
+    ("C2", dict(topk=2048, n_q=2, buffer_slots=32768, n_iters=40, context=131072, max_lifetime=3)),
+]
+
+
+@pytest.mark.parametrize("name,kw", BIG_TABLES)
+@pytest.mark.parametrize("index", ["INDEX_HASH", "INDEX_DIRECT"])
+@pytest.mark.parametrize("mode", ["XFER_SM_BALANCED", "XFER_SM_OVERLAP"])
+def test_tables_above_8192_slots(avsg, name, kw, index, mode):
+    r = _parity(tr.workload(name, **kw), index_mode=getattr(avsg, index), mode=getattr(avsg, mode), buffer_every=4)
+    assert r["gpu"]["rows_copied"] == r["oracle"]["rows_copied"] > 0
+
+
+def test_cluster_full_c2_c3_and_unsorted(avsg):
+    _parity(tr.workload("C2"), cluster=4, index_mode=avsg.INDEX_DIRECT, mode=avsg.XFER_SM_OVERLAP, buffer_every=8)
+    _parity(tr.workload("C2", n_iters=48), cluster=2, index_mode=avsg.INDEX_HASH, permute_seed=4, buffer_every=8)
+    _parity(tr.workload("C3", n_iters=24), cluster=4, index_mode=avsg.INDEX_DIRECT, mode=avsg.XFER_SM_OVERLAP,
+            buffer_every=8)
+    _parity(tr.workload("C4", n_iters=16), cluster=4, index_mode=avsg.INDEX_HASH, buffer_every=8, host_io=True)
+
+
 # ---- Stage Two overlapping Stage One (latency hiding, App. G) ---------------------------------------------------
 @pytest.mark.parametrize("name,kw,index", [
     ("C1", {}, "INDEX_HASH"), ("C2", {}, "INDEX_HASH"), ("C2", {}, "INDEX_DIRECT"), ("C3", {}, "INDEX_DIRECT"),
