@@ -230,7 +230,7 @@ def run_cuda(args):
     ctx = avsg.Context(num_tables=w.num_tables, buffer_slots=w.buffer_slots, row_bytes=w.row_bytes,
                        max_topk=w.topk, max_tokens=w.n_q, max_lifetime=w.max_lifetime, device=local,
                        index_mode=avsg.INDEX_DIRECT if direct else avsg.INDEX_HASH,
-                       max_context=max(c.context for c in w.tables) + w.n_q,
+                       max_context=max(c.context for c in w.tables) + w.n_q, stage_one_cluster=args.cluster,
                        transfer_mode=avsg.XFER_SM_OVERLAP if args.stage_two == "overlap" else avsg.XFER_SM_BALANCED)
     ncalls = len(w.calls)
     calls = [ctx.prepare(grp, [kv[t] for t in grp], w.n_q, w.topk,
@@ -406,7 +406,8 @@ def run_cuda(args):
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms_j / K, "ms_per_step_without_l2_flush": tmax["warm_ms"] / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int32/u8", "data": "synthetic", "config": dict(_config(w), host_row_stride=stride, stage_one_index=args.index, stage_two=args.stage_two),
+        "dtype": "int32/u8", "data": "synthetic", "config": dict(_config(w), host_row_stride=stride, stage_one_index=args.index, stage_two=args.stage_two,
+                                                       stage_one_cluster=args.cluster),
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "GB/s",
                 "h2d_bytes_per_step": int(ids_bytes + rows_timed * rb / K), "d2h_bytes_per_step": int(ids_bytes + mc_bytes),
@@ -806,6 +807,8 @@ def main():
                     help="overlap: Stage Two starts on token g's misses while Stage One places token g+1; balanced: it "
                          "starts when Stage One is complete (the per-kernel figures are always taken in balanced mode, "
                          "where an event can separate the two kernels; the copy loop is the same)")
+    ap.add_argument("--cluster", type=int, default=0, choices=[0, 1, 2, 4, 8],
+                    help="thread blocks per table in Stage One (0 = the library's choice)")
     ap.add_argument("--row-stride", type=int, default=0,
                     help="bytes between host KV rows (0 = packed, 656); e.g. 768 pads rows to 128-byte lines")
     ap.add_argument("--table3", action="store_true",

@@ -198,8 +198,9 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_cluster_kernel(const _
     };
     // (re)builds the index from the cached ids; returns the cluster-wide number of occupied buckets
     auto build = [&]() -> uint32_t {
-        for (uint32_t i = tid; i < Hc / 4; i += nt)
-            reinterpret_cast<int4*>(s_key)[i] = make_int4(EMPTY, EMPTY, EMPTY, EMPTY);
+        if constexpr (!DIRECT)
+            for (uint32_t i = tid; i < Hc / 4; i += nt)
+                reinterpret_cast<int4*>(s_key)[i] = make_int4(EMPTY, EMPTY, EMPTY, EMPTY);
         if (tid == 0) *s_fill = 0;
         cluster_sync();                                   // every block's buckets are empty, every block's ids in place
         uint32_t live = 0;

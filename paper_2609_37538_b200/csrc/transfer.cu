@@ -255,7 +255,8 @@ __global__ void __launch_bounds__(1024) avsg_transfer_positions_kernel(const __g
         const int32_t x = __ldg(p.indices + q);
         if (x < 0 || __ldg(p.hit + q)) continue;                 // padding or hit: nothing to move
         const int32_t o = __ldg(p.slots + q);
-        if (o < 0 || (uint32_t)o >= p.S) {
+        if (o < 0) continue;                                     // an id Stage One refused (beyond the host rows)
+        if ((uint32_t)o >= p.S) {
             if (lane == 0) atomicOr(p.status, ST_BAD_SLOT);
             continue;
         }

@@ -607,6 +607,51 @@ def test_direct_index_import_restore_and_bad_ids(avsg):
         avsg.Context(1, S, rb, K, 1, 4, index_mode=avsg.INDEX_DIRECT, max_context=0)
 
 
+@pytest.mark.parametrize("index,cluster,mode", [
+    ("INDEX_HASH", 0, "XFER_SM_BALANCED"), ("INDEX_DIRECT", 0, "XFER_SM_OVERLAP"), ("INDEX_PAPER", 0, "XFER_SM_BALANCED"),
+    ("INDEX_HASH", 2, "XFER_SM_OVERLAP"), ("INDEX_DIRECT", 4, "XFER_SM_BALANCED"), ("INDEX_HASH", 0, "XFER_ALL_K"),
+    ("INDEX_HASH", 0, "XFER_POSITION_LEVEL"),
+])
+def test_ids_beyond_the_host_rows_are_not_fetched(avsg, index, cluster, mode):
+    """With kv_rows stated, an id at or beyond a table's host rows is taken as padding (slot -1, nothing read from
+    host memory) and reported in the status word; everything else goes on as if the id had been padding."""
+    import torch
+    from oracle import LiteralOracleTable
+    rb, S, K, rows, n = 48, 256, 24, 3000, 3
+    kv = avsg.pinned_empty(rows * rb)                     # exactly `rows` rows: an unchecked id beyond it would read
+    tr.fill_kv(kv.data_ptr(), 6, 0, rows, rb)             # outside the allocation
+    literal = index == "INDEX_PAPER"
+    all_k = mode == "XFER_ALL_K"
+    ctx = avsg.Context(n, S, rb, K, 2, 4, index_mode=getattr(avsg, index), max_context=1 << 20,
+                       stage_one_cluster=cluster, transfer_mode=getattr(avsg, mode))
+    orc = [LiteralOracleTable(S, rb, 4) if literal else OracleTable(S, rb, 4) for _ in range(n)]
+    rng = np.random.default_rng(9)
+    saw_bad = False
+    for t in range(12):
+        X = np.stack([np.stack([rng.permutation(rows)[:K] for _ in range(2)]) for _ in range(n)]).astype(np.int32)
+        if t % 3 == 1:                                    # some calls carry ids the host KV does not have
+            X[0, 0, 3] = rows
+            X[1, 1, 7] = rows + 123456
+            X[2, 0, 0] = 0x7FFFFFFF
+            saw_bad = True
+        out = ctx.step(list(range(n)), torch.from_numpy(X).cuda(), [kv] * n, [rows] * n, kv_rows=[rows] * n)
+        torch.cuda.synchronize()
+        Xo = np.where(X >= rows, -1, X)                   # what the operator must have seen
+        for i in range(n):
+            if all_k:
+                want = orc[i].step_all_k(Xo[i], kv.numpy(), rb)
+                assert (out.slots[i].cpu().numpy() == want).all(), (t, i)
+                continue
+            r = orc[i].step(Xo[i], rows, kv.numpy(), rb)
+            assert (out.slots[i].cpu().numpy() == r.O).all() and (out.hit[i].cpu().numpy() == r.M).all(), (t, i)
+            assert (out.miss_count[i].cpu().numpy() == r.n).all(), (t, i)
+            assert (ctx.buffer(i).cpu().numpy() == orc[i].rows()).all(), (t, i)
+        status = ctx.sync_status()
+        assert status == (avsg.STATUS_BAD_ID if saw_bad else 0), (t, status)
+    ctx.clear_status()
+    assert ctx.sync_status() == 0
+
+
 # ---- degenerate selections --------------------------------------------------------------------------------------
 @pytest.mark.parametrize("index_mode", [0, 1])
 def test_degenerate_selections(avsg, index_mode):

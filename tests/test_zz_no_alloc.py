@@ -66,6 +66,39 @@ def test_noalloc_matches_context_path_on_consecutive_calls():
                                   hot_size=32, hot_range=512, max_lifetime=3), 6)
 
 
+def test_noalloc_at_its_documented_limits():
+    """32 tables x 2 tokens x 2048 ids = 131072 ids on 8192-slot tables: the largest call the fixed scratch takes.
+    The first (cold) step writes every entry of the scratch's miss list, the following ones are steady steps."""
+    import torch
+    import paper_2609_37538_b200 as avsg
+    avsg.load_library()
+    w = tr.workload("C3", requests=avsg.NOALLOC_MAX_TABLES, layers=1, n_iters=3, context=32768)
+    assert w.num_tables * w.n_q * w.topk == avsg.NOALLOC_MAX_IDS and w.buffer_slots == 8192
+    _run(avsg, torch, w, 3)
+
+
+def test_noalloc_checks_ids_against_the_stated_host_rows():
+    import torch
+    import paper_2609_37538_b200 as avsg
+    from oracle import OracleTable
+    rb, S, K, rows = 32, 64, 8, 500
+    kv = avsg.pinned_empty(rows * rb)
+    tr.fill_kv(kv.data_ptr(), 3, 0, rows, rb)
+    tok = torch.full((1, S), -1, dtype=torch.int32, device="cuda")
+    life = torch.full((1, S), -1, dtype=torch.int8, device="cuda")
+    buf = torch.zeros((1, S, rb), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    X = np.array([[[5, 499, 500, 17, 100000, 3, 8, 9]]], dtype=np.int32)
+    slots = torch.full((1, 1, K), -7, dtype=torch.int32, device="cuda")
+    avsg.step_noalloc(tok, life, buf, torch.from_numpy(X).cuda(), [kv], [rows], max_lifetime=4, slots=slots,
+                      status=status, kv_rows=[rows])
+    torch.cuda.synchronize()
+    orc = OracleTable(S, rb, 4)
+    r = orc.step(np.where(X[0] >= rows, -1, X[0]), rows, kv.numpy(), rb)
+    assert (slots[0].cpu().numpy() == r.O).all() and (buf[0].cpu().numpy() == orc.rows()).all()
+    assert int(status.item()) == avsg.STATUS_BAD_ID
+
+
 def test_noalloc_rejects_what_the_fixed_scratch_cannot_hold():
     import torch
     import paper_2609_37538_b200 as avsg
