@@ -103,12 +103,25 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def _workload(rank: int, n_iters: int, args=None):
+def _workload(rank: int, n_iters: int, args=None, world: int = 1):
+    """C3 for this rank.  Weak scaling (default): every rank has its own full set of tables (its own seed).
+    Strong scaling: the ONE set of tables of a single-GPU run is split by request over the ranks
+    (sharding.tables_of_rank), every rank keeping all layers of its requests."""
+    import dataclasses
     import avsg_traces as tr
+    from paper_2609_37538_b200.sharding import tables_of_rank
     kw = {}
     if args is not None:
         kw = {"requests": args.requests, "layers": args.layers}
-    return tr.workload("C3", seed=3 + 1000 * rank, n_iters=n_iters, **kw)
+    if args is None or getattr(args, "scaling", "weak") == "weak" or world == 1:
+        return tr.workload("C3", seed=3 + 1000 * rank, n_iters=n_iters, **kw)
+    w = tr.workload("C3", seed=3, n_iters=n_iters, **kw)
+    n_req = len(w.calls[0])
+    mine = tables_of_rank(n_req, world, rank)                 # requests of this rank
+    keep = [grp[r] for grp in w.calls for r in mine]          # their tables, layer by layer
+    local = {t: i for i, t in enumerate(keep)}
+    calls = [[local[grp[r]] for r in mine] for grp in w.calls]
+    return dataclasses.replace(w, tables=[w.tables[t] for t in keep], calls=[c for c in calls if c])
 
 
 def _gen_traces(w, threads):
@@ -204,6 +217,12 @@ def run_cuda(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
+    # the rank's threads (trace generation, the fill of the pinned host KV: first touch decides where its pages
+    # live) run on the CPUs of the GPU's NUMA node; on by default when there are several ranks
+    from paper_2609_37538_b200.sharding import bind_to_numa_node_of, pci_address
+    props = torch.cuda.get_device_properties(local)
+    bdf = pci_address(getattr(props, "pci_domain_id", 0), getattr(props, "pci_bus_id", 0), getattr(props, "pci_device_id", 0))
+    numa = bind_to_numa_node_of(bdf, apply=args.numa_bind == "on" or (args.numa_bind == "auto" and world > 1))
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     if rank == 0:
@@ -213,11 +232,11 @@ def run_cuda(args):
     import paper_2609_37538_b200 as avsg
     avsg.load_library()
 
-    cores = os.cpu_count() or 1
-    threads = max(1, cores // world)
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    threads = max(1, cores if numa["bound"] else cores // world)
     W, K = args.warmup, args.steps
     n_iters = max(64, W + K)
-    w = _workload(rank, n_iters, args)
+    w = _workload(rank, n_iters, args, world)
     traces = _gen_traces(w, threads)
     kv = []
     stride = args.row_stride or w.row_bytes
@@ -391,7 +410,7 @@ def run_cuda(args):
         roofline = {"bound": "host_link", "kernel": "avsg_transfer_overlap_kernel", "achieved": call_gbs,
                     "peak": link_peak, "unit": "GB/s", "frac": call_gbs / link_peak,
                     "traffic": NCU_XFER_DRAM_BYTES_PER_ROW * call_bytes / rb,
-                    "peak_kind": "measured in this run (pinned cudaMemcpyAsync H2D)",
+                    "peak_kind": "measured in this run (pinned cudaMemcpyAsync H2D, 1 GiB, best of 4 after one warm-up copy)", "peak_repeats": 4,
                     "duration_us": call_us,
                     "note": "algorithmic bytes = row_bytes x missed rows per launch; duration = CUDA events around the "
                             "timed steps / launches, i.e. the whole call, the part of Stage One that is not hidden "
@@ -401,11 +420,12 @@ def run_cuda(args):
         roofline = {"bound": "host_link", "kernel": "avsg_transfer_kernel", "achieved": x_gbs, "peak": link_peak,
                     "unit": "GB/s", "frac": x_gbs / link_peak,
                     "traffic": NCU_XFER_DRAM_BYTES_PER_ROW * sum(x_rows) / n_launch,
-                    "peak_kind": "measured in this run (pinned cudaMemcpyAsync H2D)", "duration_us": x_avg_us,
+                    "peak_kind": "measured in this run (pinned cudaMemcpyAsync H2D, 1 GiB, best of 4 after one warm-up copy)", "peak_repeats": 4, "duration_us": x_avg_us,
                     "note": "same object as roofline_transfer_alone"}
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W,
-        "ms_per_step": total_ms_j / K, "ms_per_step_without_l2_flush": tmax["warm_ms"] / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": total_ms_j / K, "ms_per_step_without_l2_flush": tmax["warm_ms"] / K, "higher_is_better": True,
+        "scaling": args.scaling if world > 1 else "weak", "vs_baseline": None,
         "dtype": "int32/u8", "data": "synthetic", "config": dict(_config(w), host_row_stride=stride, stage_one_index=args.index, stage_two=args.stage_two,
                                                        stage_one_cluster=args.cluster),
         "clocks": clocks,
@@ -415,6 +435,8 @@ def run_cuda(args):
                 "note": "avsg_step_host: ids uploaded from pinned host memory, slot table and miss counts "
                         "downloaded; h2d bytes = ids + missed KV rows"},
         "gpu_launches": 2 * ncalls * K,
+        "numa": {"gpu_pci": bdf, "numa_node": numa["numa_node"], "bound": numa["bound"], "cpus": len(numa["cpus"]),
+                 "note": "rank 0; the pinned host KV is allocated and filled by threads bound to these CPUs when bound"},
         "hit_rate": hits_j / max(1.0, hits_j + miss_j),
         "hit_rate_request_macro": tsum["req_rate_sum"] / max(1.0, tsum["req_n"]),
         "miss_rows_per_step": rows_j / K / world,
@@ -436,7 +458,7 @@ def run_cuda(args):
         "roofline_transfer_alone": {"bound": "host_link", "kernel": "avsg_transfer_kernel", "achieved": x_gbs, "peak": link_peak,
                      "unit": "GB/s", "frac": x_gbs / link_peak,
                      "traffic": NCU_XFER_DRAM_BYTES_PER_ROW * sum(x_rows) / n_launch,
-                     "peak_kind": "measured in this run (pinned cudaMemcpyAsync H2D)",
+                     "peak_kind": "measured in this run (pinned cudaMemcpyAsync H2D, 1 GiB, best of 4 after one warm-up copy)", "peak_repeats": 4,
                      "note": "algorithmic bytes = row_bytes x missed rows per launch; the rows cross the host link and stay "
                              "in L2 after the write, so DRAM traffic (scaled from the ncu capture of the one-layer case) is small; "
                              "timed in balanced mode (one kernel at a time); with --stage-two overlap the timed steps run "
@@ -462,6 +484,12 @@ def run_cuda(args):
             "single_thread": {"value": sum(rows1) * rb / 1e9 / sum(secs1), "unit": "GB/s",
                               "ms_per_table_iteration": 1e3 * sum(secs1) / len(secs1) / len(one_tables),
                               "sample": "%d tables, 4 iterations after %d warm-up, one thread" % (len(one_tables), W)}}
+    if world == 1 and not args.no_comparators:
+        # the three-way comparison of the evaluation on C5, inside the same run: free C3 first
+        ctx.close()
+        del calls, ctx, kv, Xd, Xp
+        torch.cuda.empty_cache()
+        line["comparators_c5"] = comparators_c5(avsg, torch, tr, link_peak, tiny=args.tiny)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -510,6 +538,7 @@ def _suite_one(avsg, torch, tr, name, mode, mode_name, link_peak, needed_rows=No
     xf_us = sum(x for _, x, _ in steady)
     out = {
         "suite": name, "transfer_mode": mode_name, "tables": w.num_tables, "calls_per_iter": len(w.calls),
+        "host_kv_gb": round(w.host_kv_bytes() / 1e9, 2),
         "iters": w.n_iters, "hit_rate": st["hits"] / max(1, st["hits"] + st["misses"]),
         "cold_iter": {"rows": cold[2], "transfer_us": cold[1], "gbs": cold[2] * rb / 1e3 / max(cold[1], 1e-9),
                       "match_reserve_us": cold[0]},
@@ -563,6 +592,55 @@ def _suite_modes(avsg, torch, tr, name, **kw):
     return out
 
 
+# shrunk shapes for --tiny (K <= 256, at most 4 tables, 6 iterations): what the GPU tests run so that this code
+# cannot rot; the numbers they give are not measurements of anything
+TINY = {
+    "C1": dict(topk=64, buffer_slots=256, n_iters=6, context=2048),
+    "C2": dict(topk=256, buffer_slots=1024, n_iters=6, context=8192, recent_window=512),
+    "C3": dict(topk=256, buffer_slots=1024, n_iters=6, context=8192, requests=2, layers=2, recent_window=512),
+    "C4": dict(topk=256, buffer_slots=1024, n_iters=6, context=16384, requests=4, hot_size=64, hot_range=1024),
+    "C5": dict(topk=256, buffer_slots=1024, n_iters=6, requests=4, ctx_lo=512, ctx_hi=8192),
+}
+
+
+def _link_peak(torch, nbytes=1 << 30, repeats=4):
+    """Best of `repeats` pinned host -> device copies of nbytes (after one warm-up copy), GB/s."""
+    big_h = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+    big_d = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    best = 0.0
+    for i in range(repeats + 1):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); big_d.copy_(big_h, non_blocking=True); e1.record()
+        torch.cuda.synchronize()
+        if i:
+            best = max(best, nbytes / 1e9 / (e0.elapsed_time(e1) / 1e3))
+    return best
+
+
+def comparators_c5(avsg, torch, tr, link_peak, tiny=False):
+    """Configuration C5 (load-imbalance stress) under the operator's balanced Stage Two and the two comparators the
+    evaluation names: request-level assignment (App. D, S1: one block per request) and transfer-all-K (Sec. 4.1,
+    no reuse).  Same traces for all three; steady iterations after the cold one; effective GB/s = bytes of the
+    rows the operator NEEDS (the balanced run's misses) over the Stage Two time of the mode."""
+    kw = dict(TINY["C5"]) if tiny else dict(n_iters=9)
+    out = {"workload": "C5: %s" % ("tiny" if tiny else "64 requests, contexts log-uniform in [4096, 524288], cold + 8 steps")}
+    need = None
+    for mode, mn in ((avsg.XFER_SM_BALANCED, "balanced"), (avsg.XFER_REQUEST_LEVEL, "request_level"),
+                     (avsg.XFER_ALL_K, "transfer_all_k")):
+        r = _suite_one(avsg, torch, tr, "C5", mode, mn, link_peak, needed_rows=need, **kw)
+        if need is None:
+            need = r["rows_per_iter_list"]
+            out["host_kv_gb"] = r["host_kv_gb"]
+            out["hit_rate"] = r["hit_rate"]
+            out["rows_needed_per_iter"] = r["steady"]["rows_per_iter"]
+        out[mn] = {"stage_two_us_per_iter": r["steady"]["transfer_us_per_iter"],
+                   "effective_gbs": r["steady"]["effective_gbs"], "raw_gbs": r["steady"]["raw_gbs"],
+                   "pct_of_link_peak": 100.0 * r["steady"]["effective_gbs"] / link_peak}
+    out["balanced_over_request_level"] = out["balanced"]["effective_gbs"] / out["request_level"]["effective_gbs"]
+    out["balanced_over_transfer_all_k"] = out["balanced"]["effective_gbs"] / out["transfer_all_k"]["effective_gbs"]
+    return out
+
+
 def run_suite(args):
     import torch
     import __graft_entry__
@@ -570,34 +648,27 @@ def run_suite(args):
     __graft_entry__.build()
     import paper_2609_37538_b200 as avsg
     torch.cuda.set_device(0)
-    big_h = torch.empty(1 << 30, dtype=torch.uint8, pin_memory=True)
-    big_d = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
-    best = 0.0
-    for i in range(5):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(); big_d.copy_(big_h, non_blocking=True); e1.record()
-        torch.cuda.synchronize()
-        if i:
-            best = max(best, (1 << 30) / 1e9 / (e0.elapsed_time(e1) / 1e3))
-    del big_h, big_d
+    tiny = args.tiny
+    best = _link_peak(torch, (64 << 20) if tiny else (1 << 30))
     print(json.dumps({"suite": "link", "link_peak_gbs": best}), flush=True)
     M = avsg
     for name in ("C1", "C2", "C3", "C4", "C5"):
-        r = _suite_one(avsg, torch, tr, name, M.XFER_SM_BALANCED, "sm_balanced", best)
+        kw = dict(TINY[name]) if tiny else {}
+        r = _suite_one(avsg, torch, tr, name, M.XFER_SM_BALANCED, "sm_balanced", best, **kw)
         need = r.pop("rows_per_iter_list")
         print(json.dumps(r), flush=True)
         if name == "C5":      # the load-imbalance stress: same traces under the comparators
             for mode, mn in ((M.XFER_REQUEST_LEVEL, "request_level"), (M.XFER_ALL_K, "transfer_all_k")):
-                r2 = _suite_one(avsg, torch, tr, name, mode, mn, best, needed_rows=need)
+                r2 = _suite_one(avsg, torch, tr, name, mode, mn, best, needed_rows=need, **kw)
                 r2.pop("rows_per_iter_list")
                 print(json.dumps(r2), flush=True)
         if name == "C3":      # copy-engine comparator on a few iterations (one async copy per run of rows)
-            r2 = _suite_one(avsg, torch, tr, name, M.XFER_COPY_ENGINE, "copy_engine", best, needed_rows=need[:6],
-                            n_iters=6)
+            kw2 = dict(kw, n_iters=6)
+            r2 = _suite_one(avsg, torch, tr, name, M.XFER_COPY_ENGINE, "copy_engine", best, needed_rows=need[:6], **kw2)
             r2.pop("rows_per_iter_list")
             print(json.dumps(r2), flush=True)
     for name, kw in (("C1", {}), ("C2", {}), ("C3", {"n_iters": 32}), ("C4", {"n_iters": 32}), ("C5", {})):
-        print(json.dumps(_suite_modes(avsg, torch, tr, name, **kw)), flush=True)
+        print(json.dumps(_suite_modes(avsg, torch, tr, name, **(dict(TINY[name]) if tiny else kw))), flush=True)
 
 
 # ------------------------------------------------------------------------------------------------------------
@@ -610,7 +681,7 @@ def run_table3(args):
     __graft_entry__.build()
     import paper_2609_37538_b200 as avsg
     torch.cuda.set_device(0)
-    K, S, RB, CTX, B_MAX = 2048, 8192, 1152, 131072, 32
+    K, S, RB, CTX, B_MAX = (256, 1024, 1152, 8192, 4) if args.tiny else (2048, 8192, 1152, 131072, 32)
     rng = np.random.default_rng(20260937)
     kv = []
     for ti in range(B_MAX):
@@ -621,7 +692,7 @@ def run_table3(args):
     stream = torch.cuda.current_stream()
     modes = (("S1_request_level", avsg.XFER_REQUEST_LEVEL), ("S2_position_level", avsg.XFER_POSITION_LEVEL),
              ("S3_miss_level", avsg.XFER_SM_BALANCED))
-    for B in (1, 2, 4, 8, 16, 32):
+    for B in ((1, 4) if args.tiny else (1, 2, 4, 8, 16, 32)):
         ctx = avsg.Context(num_tables=B, buffer_slots=S, row_bytes=RB, max_topk=K, max_tokens=1, max_lifetime=16)
         ctx.set_timing(True)
         call = ctx.prepare(list(range(B)), kv[:B], 1, K)
@@ -631,7 +702,7 @@ def run_table3(args):
         call.run(Xa, [CTX] * B, slots, None, None, stream)          # cold step: the first selection becomes resident
         ctx.save_state()
         torch.cuda.synchronize()
-        for reuse in (0.0, 0.25, 0.5, 0.75):
+        for reuse in ((0.0, 0.5) if args.tiny else (0.0, 0.25, 0.5, 0.75)):
             keep = int(round(reuse * K))
             sel = []
             for b in range(B):
@@ -708,74 +779,90 @@ def run_sweeps(args):
     __graft_entry__.build()
     import paper_2609_37538_b200 as avsg
     torch.cuda.set_device(0)
+    tiny = args.tiny
+    CTX = 8192 if tiny else 131072
+    KB = 256 if tiny else 2048                 # the top-K of the DSA-shaped sweeps
+    SB = 1024 if tiny else 8192                # their pool
+    NT = 4 if tiny else 16                     # tables
+    WIN = 512 if tiny else 4096
 
-    def recipe(table, K, n_q, T, ctx=131072, seed=77, **kw):
-        base = dict(beta=(18, 2), p_recent=0.5, recent_window=4096)
+    def recipe(table, K, n_q, T, ctx=CTX, seed=77, **kw):
+        base = dict(beta=(18, 2), p_recent=0.5, recent_window=WIN)
         base.update(kw)
         return tr.TraceConfig(seed=seed, table=table, topk=K, n_q=n_q, n_iters=T, context=ctx, **base)
 
-    # (a) Stage One latency: S = K = N; K at S = 4096; S at K = 512.  Median of 300 replays of a steady step.
-    shapes = [("S=K=N", k, k) for k in (256, 512, 1024, 2048)]
-    shapes += [("K at S=4096", k, 4096) for k in (256, 512, 1024, 2048)]
-    shapes += [("S at K=512", 512, sz) for sz in (512, 1024, 2048, 4096, 8192)]
+    # (a) Stage One latency: S = K = N; K at S = 4096; S at K = 512 (the shapes of the paper's Fig. 3); pools above
+    #     8192 slots at K = 2048 (one thread-block cluster per table).  Median of the replays of a steady step.
+    if tiny:
+        shapes = [("S=K=N", 64, 64), ("K at S=4096", 128, 4096), ("S at K=512", 512, 1024), ("S at K=2048", 2048, 16384)]
+    else:
+        shapes = [("S=K=N", k, k) for k in (256, 512, 1024, 2048)]
+        shapes += [("K at S=4096", k, 4096) for k in (256, 512, 1024, 2048)]
+        shapes += [("S at K=512", 512, sz) for sz in (512, 1024, 2048, 4096, 8192)]
+        shapes += [("S at K=2048", 2048, sz) for sz in (8192, 16384, 32768)]
     for label, K, S in shapes:
-        for B in (1, 32):
-            _, med = _run_tables(avsg, torch, tr, [recipe(i, K, 1, 24) for i in range(B)], S, 16, replay=300)
+        for B in ((1, 3) if tiny else (1, 32)):
+            _, med = _run_tables(avsg, torch, tr, [recipe(i, K, 1, 6 if tiny else 24, ctx=max(CTX, 4 * K)) for i in range(B)],
+                                 S, 16, replay=5 if tiny else 300)
             print(json.dumps({"sweep": "stage_one_latency", "series": label, "K": K, "S": S, "tables": B,
                               "match_reserve_us_median": med}), flush=True)
     # (b) lifetime ablation: K = 2048, 8K pool, MTP-0, 16 tables, 200 steps, steady steps only
-    for L in (1, 2, 4, 8, 16, 32):
-        per, med = _run_tables(avsg, torch, tr, [recipe(i, 2048, 1, 200) for i in range(16)], 8192, L, replay=100)
-        h = sum(a for a, _ in per[40:]); m = sum(b for _, b in per[40:])
+    T, skip = (6, 2) if tiny else (200, 40)
+    for L in ((1, 16) if tiny else (1, 2, 4, 8, 16, 32)):
+        per, med = _run_tables(avsg, torch, tr, [recipe(i, KB, 1, T) for i in range(NT)], SB, L, replay=3 if tiny else 100)
+        h = sum(a for a, _ in per[skip:]); m = sum(b for _, b in per[skip:])
         print(json.dumps({"sweep": "lifetime", "L": L, "hit_rate": h / (h + m), "match_reserve_us_median": med}),
               flush=True)
     # (c) capacity study: max KV 16K, K = 2048, L = 8, MTP-0, adjacent-step similarity gamma fixed, historical
     #     recall ~ N(mu, 0.01^2); 4K and 8K pools; 5 seeds (one table each); 300 steps, the first 60 not counted
-    for gamma in (0.5, 0.7, 0.9):
-        for mu in (0.5, 0.7, 0.9):
+    T, skip = (8, 2) if tiny else (300, 60)
+    for gamma in ((0.7,) if tiny else (0.5, 0.7, 0.9)):
+        for mu in ((0.7,) if tiny else (0.5, 0.7, 0.9)):
             row = {"sweep": "capacity", "gamma": gamma, "mu_hist": mu}
-            for S in (4096, 8192):
-                cfgs = [tr.TraceConfig(seed=900 + sd, table=sd, topk=2048, n_q=1, n_iters=300, context=16384,
-                                       rho_fixed=gamma, p_hist=mu, hist_sigma=0.01) for sd in range(5)]
+            for S in ((512, 1024) if tiny else (4096, 8192)):
+                cfgs = [tr.TraceConfig(seed=900 + sd, table=sd, topk=KB, n_q=1, n_iters=T, context=8 * KB,
+                                       rho_fixed=gamma, p_hist=mu, hist_sigma=0.01) for sd in range(2 if tiny else 5)]
                 per, _ = _run_tables(avsg, torch, tr, cfgs, S, 8)
-                h = sum(a for a, _ in per[60:]); m = sum(b for _, b in per[60:])
-                row["hit_rate_%dK" % (S // 1024)] = h / (h + m)
+                h = sum(a for a, _ in per[skip:]); m = sum(b for _, b in per[skip:])
+                row["hit_rate_%dK" % (S // 1024) if S >= 1024 else "hit_rate_%d" % S] = h / (h + m)
             print(json.dumps(row), flush=True)
     # (e) the paper's Hash-State table as printed (bounded probing, lossy) against the exact indexes
-    for n_q in (1, 2):
-        cfgs = [recipe(i, 2048, n_q, 200) for i in range(16)]
+    T, skip = (6, 2) if tiny else (200, 40)
+    for n_q in ((2,) if tiny else (1, 2)):
+        cfgs = [recipe(i, KB, n_q, T) for i in range(NT)]
         for label, mode, R in (("exact_hash", avsg.INDEX_HASH, 0), ("exact_direct", avsg.INDEX_DIRECT, 0),
                                ("paper_R1", avsg.INDEX_PAPER, 1), ("paper_R3", avsg.INDEX_PAPER, 3),
                                ("paper_R7", avsg.INDEX_PAPER, 7)):
-            per, med = _run_tables(avsg, torch, tr, cfgs, 8192, 16, replay=100, index_mode=mode, probe_retries=R)
-            h = sum(a for a, _ in per[40:]); m = sum(b for _, b in per[40:])
+            per, med = _run_tables(avsg, torch, tr, cfgs, SB, 16, replay=3 if tiny else 100, index_mode=mode, probe_retries=R)
+            h = sum(a for a, _ in per[skip:]); m = sum(b for _, b in per[skip:])
             print(json.dumps({"sweep": "index_mode", "n_tokens": n_q, "index": label, "hit_rate": h / (h + m),
-                              "rows_copied_per_table_iter": m / 16 / 160, "match_reserve_us_median": med}), flush=True)
+                              "rows_copied_per_table_iter": m / NT / (T - skip), "match_reserve_us_median": med}), flush=True)
     # (f) what the overlapped Stage Two buys as the MTP degree grows: one 32-table call per iteration, K = 2048,
     #     8K pool, direct index; device time per call (CUDA events, L2 flushed before each), steady iterations
-    kvs = [avsg.pinned_empty(131072 * 656) for _ in range(32)]
+    NB, T, skip = (3, 6, 2) if tiny else (32, 40, 10)
+    kvs = [avsg.pinned_empty(CTX * 656) for _ in range(NB)]
     for i, b in enumerate(kvs):
-        tr.fill_kv(b.data_ptr(), 77, i, 131072, 656)
+        tr.fill_kv(b.data_ptr(), 77, i, CTX, 656)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
-    for n_q in (1, 2, 3, 4):
-        cfgs = [recipe(i, 2048, n_q, 40) for i in range(32)]
+    for n_q in ((1, 3) if tiny else (1, 2, 3, 4)):
+        cfgs = [recipe(i, KB, n_q, T) for i in range(NB)]
         traces = [tr.generate(c) for c in cfgs]
-        X = [torch.from_numpy(np.stack([traces[i][0][t] for i in range(32)])).cuda() for t in range(40)]
-        V = [[int(traces[i][1][t]) for i in range(32)] for t in range(40)]
+        X = [torch.from_numpy(np.stack([traces[i][0][t] for i in range(NB)])).cuda() for t in range(T)]
+        V = [[int(traces[i][1][t]) for i in range(NB)] for t in range(T)]
         slots = torch.empty_like(X[0])
         row = {"sweep": "overlap_vs_tokens", "n_tokens": n_q}
         for mode, mname in ((avsg.XFER_SM_BALANCED, "balanced"), (avsg.XFER_SM_OVERLAP, "overlap")):
-            ctx = avsg.Context(num_tables=32, buffer_slots=8192, row_bytes=656, max_topk=2048, max_tokens=n_q,
-                               max_lifetime=16, transfer_mode=mode, index_mode=avsg.INDEX_DIRECT, max_context=131072 + n_q)
-            call = ctx.prepare(list(range(32)), kvs, n_q, 2048)
+            ctx = avsg.Context(num_tables=NB, buffer_slots=SB, row_bytes=656, max_topk=KB, max_tokens=n_q,
+                               max_lifetime=16, transfer_mode=mode, index_mode=avsg.INDEX_DIRECT, max_context=CTX + n_q)
+            call = ctx.prepare(list(range(NB)), kvs, n_q, KB)
             us = []
-            for t in range(40):
+            for t in range(T):
                 flush.fill_(t)
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(); call.run(X[t], V[t], slots, None, None, stream); e1.record()
                 torch.cuda.synchronize()
-                if t >= 10:
+                if t >= skip:
                     us.append(e0.elapsed_time(e1) * 1e3)
             st = ctx.stats()
             row[mname + "_us"] = sum(us) / len(us)
@@ -784,11 +871,11 @@ def run_sweeps(args):
         print(json.dumps(row), flush=True)
     del kvs
     # (d) MTP cold start: reuse inside the first iteration from an empty buffer, degrees 0..3, 32 tables
-    for deg in range(4):
-        per, _ = _run_tables(avsg, torch, tr, [recipe(i, 2048, deg + 1, 1) for i in range(32)], 8192, 16)
+    for deg in ((0, 3) if tiny else range(4)):
+        per, _ = _run_tables(avsg, torch, tr, [recipe(i, KB, deg + 1, 1) for i in range(NB)], SB, 16)
         h, m = per[0]
         print(json.dumps({"sweep": "mtp_cold_start", "n_mtp": deg, "reuse": h / (h + m),
-                          "rows_copied_per_request": m / 32}), flush=True)
+                          "rows_copied_per_request": m / NB}), flush=True)
 
 
 def main():
@@ -807,6 +894,16 @@ def main():
                     help="overlap: Stage Two starts on token g's misses while Stage One places token g+1; balanced: it "
                          "starts when Stage One is complete (the per-kernel figures are always taken in balanced mode, "
                          "where an event can separate the two kernels; the copy loop is the same)")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="N > 1: weak = every rank has its own 128 tables (default); strong = the 128 tables of the "
+                         "single-GPU run are split by request over the ranks")
+    ap.add_argument("--numa-bind", default="auto", choices=["auto", "on", "off"],
+                    help="bind the rank to the CPUs of its GPU's NUMA node before the host KV is allocated "
+                         "(auto = when there are several ranks)")
+    ap.add_argument("--tiny", action="store_true",
+                    help="with --suite / --table3 / --sweeps: shrunk shapes that finish in seconds (what the tests run)")
+    ap.add_argument("--no-comparators", action="store_true",
+                    help="skip the comparators_c5 object (balanced / request-level / transfer-all-K on C5)")
     ap.add_argument("--cluster", type=int, default=0, choices=[0, 1, 2, 4, 8],
                     help="thread blocks per table in Stage One (0 = the library's choice)")
     ap.add_argument("--row-stride", type=int, default=0,

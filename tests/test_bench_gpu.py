@@ -13,7 +13,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 @pytest.mark.parametrize("extra", [[], ["--stage-two", "balanced", "--index", "hash"]])
 def test_bench_line(extra):
     cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--requests", "4", "--layers", "2", "--steps", "4", "--warmup", "3",
-           "--replays", "20"] + extra
+           "--replays", "20", "--tiny"] + extra
     out = subprocess.run(cmd, cwd=ROOT, capture_output=True, text=True, timeout=900, check=True).stdout
     lines = [l for l in out.splitlines() if l.startswith("{")]
     assert len(lines) == 1
@@ -31,3 +31,55 @@ def test_bench_line(extra):
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["value"] > 0
     assert d["clocks"]["sm_max_mhz"] >= d["clocks"]["sm_mhz"] > 0
     assert 0.5 < d["hit_rate"] < 1.0 and d["config"]["workload"].startswith("C3")
+    assert r["peak_repeats"] == 4 and "numa_node" in d["numa"]
+    c5 = d["comparators_c5"]
+    for mode in ("balanced", "request_level", "transfer_all_k"):
+        assert c5[mode]["effective_gbs"] > 0 and c5[mode]["stage_two_us_per_iter"] > 0
+    assert c5["transfer_all_k"]["raw_gbs"] > c5["transfer_all_k"]["effective_gbs"]      # it moves rows nobody needs
+
+
+def _json_lines(args, timeout=900):
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py")] + args
+    out = subprocess.run(cmd, cwd=ROOT, capture_output=True, text=True, timeout=timeout, check=True).stdout
+    return [json.loads(l) for l in out.splitlines() if l.startswith("{")]
+
+
+def test_suite_report_tiny():
+    """bench.py --suite on shrunk shapes: every configuration reports, and so do the comparators."""
+    rows = _json_lines(["--suite", "--tiny"])
+    assert rows[0]["suite"] == "link" and rows[0]["link_peak_gbs"] > 1
+    by = {(r["suite"], r.get("transfer_mode")): r for r in rows if "transfer_mode" in r}
+    for name in ("C1", "C2", "C3", "C4", "C5"):
+        r = by[(name, "sm_balanced")]
+        assert 0 <= r["hit_rate"] <= 1 and r["cold_iter"]["rows"] > 0 and r["steady"]["transfer_us_per_iter"] > 0
+    assert by[("C5", "request_level")]["steady"]["rows_per_iter"] == by[("C5", "sm_balanced")]["steady"]["rows_per_iter"]
+    assert by[("C5", "transfer_all_k")]["steady"]["rows_per_iter"] > by[("C5", "sm_balanced")]["steady"]["rows_per_iter"]
+    assert ("C3", "copy_engine") in by
+    modes = [r for r in rows if r["suite"] == "stage_two_modes"]
+    assert len(modes) == 5 and all(set(m["us_per_iteration"]) == {"direct/balanced", "direct/overlap", "hash/balanced",
+                                                                   "hash/overlap"} for m in modes)
+
+
+def test_table3_report_tiny():
+    """bench.py --table3 on a shrunk grid: with ONE request the miss-level split (S3) cannot be slower than one
+    block serving the request alone (S1), which is the point of Eq. 6."""
+    rows = _json_lines(["--table3", "--tiny", "--replays-table3", "1"])
+    assert {(r["B"], r["reuse_pct"]) for r in rows} == {(1, 0), (1, 50), (4, 0), (4, 50)}
+    for r in rows:
+        assert r["rows"] == r["B"] * 256 * (100 - r["reuse_pct"]) // 100
+        for k in ("S1_request_level_gbs", "S2_position_level_gbs", "S3_miss_level_gbs"):
+            assert r[k] > 0
+    one = [r for r in rows if r["B"] == 1 and r["reuse_pct"] == 0][0]
+    assert one["S3_miss_level_gbs"] >= one["S1_request_level_gbs"]
+
+
+def test_sweeps_report_tiny():
+    rows = _json_lines(["--sweeps", "--tiny"])
+    kinds = {r["sweep"] for r in rows}
+    assert kinds == {"stage_one_latency", "lifetime", "capacity", "index_mode", "overlap_vs_tokens", "mtp_cold_start"}
+    big = [r for r in rows if r["sweep"] == "stage_one_latency" and r["S"] == 16384]
+    assert big and all(r["match_reserve_us_median"] > 0 for r in big)          # a pool only a cluster holds
+    cold = {r["n_mtp"]: r["reuse"] for r in rows if r["sweep"] == "mtp_cold_start"}
+    assert cold[0] == 0 and cold[3] > 0                                          # later tokens reuse earlier ones' rows
+    idx = {r["index"]: r["hit_rate"] for r in rows if r["sweep"] == "index_mode"}
+    assert idx["exact_hash"] == idx["exact_direct"] >= idx["paper_R3"]

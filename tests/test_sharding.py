@@ -9,7 +9,9 @@ import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
 
-from paper_2609_37538_b200.sharding import aggregate, tables_of_rank, whole_job_gbs
+from paper_2609_37538_b200.sharding import (aggregate, bind_to_numa_node_of, cpus_of_numa_node,
+                                            numa_node_of_pci_device, parse_cpulist, pci_address, tables_of_rank,
+                                            whole_job_gbs)
 
 
 def test_tables_of_rank_partitions_exactly():
@@ -26,6 +28,39 @@ def test_aggregate_without_process_group_is_identity():
     t, w = aggregate({"step_ms": 1.5}, {"rows": 10})
     assert t == {"step_ms": 1.5} and w == {"rows": 10}
     assert whole_job_gbs(2e9, 1000.0) == 2.0
+
+
+def test_numa_helpers_against_a_fake_sysfs_tree(tmp_path):
+    """A two-socket host written out as files: GPU 0000:1b:00.0 on node 0, GPU 0000:9c:00.0 on node 1."""
+    allowed = sorted(os.sched_getaffinity(0))
+    half = max(1, len(allowed) // 2)
+    node_cpus = {0: allowed[:half], 1: allowed[half:] or allowed[:1]}
+    for bdf, node in (("0000:1b:00.0", 0), ("0000:9c:00.0", 1), ("0000:aa:00.0", -1)):
+        d = tmp_path / "bus" / "pci" / "devices" / bdf
+        d.mkdir(parents=True)
+        (d / "numa_node").write_text("%d\n" % node)
+    for node, cpus in node_cpus.items():
+        d = tmp_path / "devices" / "system" / "node" / ("node%d" % node)
+        d.mkdir(parents=True)
+        (d / "cpulist").write_text(",".join(str(c) for c in cpus) + "\n")
+    root = str(tmp_path)
+    assert pci_address(0, 0x1b, 0) == "0000:1b:00.0" and pci_address(0, 0x9c, 0) == "0000:9c:00.0"
+    assert numa_node_of_pci_device("0000:1B:00.0", root) == 0            # sysfs names are lower case
+    assert numa_node_of_pci_device("0000:9c:00.0", root) == 1
+    assert numa_node_of_pci_device("0000:aa:00.0", root) == -1 and numa_node_of_pci_device("0000:ff:00.0", root) == -1
+    assert parse_cpulist("0-3,8,10-11\n") == [0, 1, 2, 3, 8, 10, 11] and parse_cpulist("") == []
+    assert cpus_of_numa_node(1, root) == sorted(node_cpus[1]) and cpus_of_numa_node(-1, root) == []
+    before = sorted(os.sched_getaffinity(0))
+    try:
+        info = bind_to_numa_node_of("0000:9c:00.0", root, apply=False)
+        assert info == {"numa_node": 1, "cpus": sorted(node_cpus[1]), "bound": False}
+        assert sorted(os.sched_getaffinity(0)) == before                  # apply=False only reports
+        info = bind_to_numa_node_of("0000:1b:00.0", root)
+        assert info["bound"] and sorted(os.sched_getaffinity(0)) == sorted(node_cpus[0])
+        info = bind_to_numa_node_of("0000:aa:00.0", root)                 # unknown node: nothing changes
+        assert not info["bound"] and sorted(os.sched_getaffinity(0)) == sorted(node_cpus[0])
+    finally:
+        os.sched_setaffinity(0, before)
 
 
 def _free_port():
