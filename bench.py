@@ -672,6 +672,185 @@ def run_suite(args):
 
 
 # ------------------------------------------------------------------------------------------------------------
+# --link-model: what the host link gives SM-issued reads of scattered rows, by row size and alignment.  Every case is
+# an all-miss step of the operator itself (32 tables x 2048 rows), Stage Two timed from inside the kernel, so the
+# figures are the ceiling of the gather for that row geometry on this machine.  Next to each measurement: the 32-byte
+# sectors and 128-byte lines a row touches (computed from the addresses) and the prediction of a packet model of
+# the link fitted to two of the cases (see LINK_MODEL below).
+# ------------------------------------------------------------------------------------------------------------
+LINK_MODEL = {
+    "text": "time per row = (payload + H x packets) / R.  A read request of an SM covers at most one 128-byte line of host "
+            "memory and is answered by its own completion packet(s); a request for part of a line that spans the line's "
+            "64-byte midpoint is answered by two.  payload = 32-byte sectors fetched.  H (bytes per packet) and R (raw "
+            "rate) are fitted so that aligned full lines (one 128-byte packet each) and one large pinned cudaMemcpyAsync "
+            "(256-byte packets) are both reproduced.",
+}
+
+
+def _row_wire_bytes(offset, row_bytes, header):
+    """Payload sectors, lines and modelled bytes on the wire for a row at byte `offset` of a 128-byte-aligned buffer."""
+    a, b = offset, offset + row_bytes
+    sectors = lines = packets = 0
+    line = a // 128
+    while line * 128 < b:
+        lo, hi = max(a, line * 128), min(b, line * 128 + 128)
+        s0, s1 = (lo % 128) // 32, ((hi - 1) % 128) // 32           # first and last sector of the line that is read
+        sectors += s1 - s0 + 1
+        lines += 1
+        packets += 1 if (s0 == 0 and s1 == 3) or (s0 // 2 == s1 // 2) else 2
+        line += 1
+    return sectors, lines, sectors * 32 + header * packets
+
+
+def run_link_model(args):
+    import torch
+    import __graft_entry__
+    import avsg_traces as tr
+    __graft_entry__.build()
+    import paper_2609_37538_b200 as avsg
+    torch.cuda.set_device(0)
+    tiny = args.tiny
+    peak = _link_peak(torch, (64 << 20) if tiny else (1 << 30))
+    n_tab, K, S, steps = (3, 256, 1024, 3) if tiny else (32, 2048, 8192, 5)
+    geos = [(656, 656), (656, 672), (656, 704), (656, 768), (640, 640), (1152, 1152), (2048, 2048), (512, 512),
+            (256, 256), (128, 128)]
+    if tiny:
+        geos = [(656, 656), (656, 768), (1152, 1152)]
+    rows = []
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    rng = np.random.default_rng(12)
+    for rb, stride in geos:
+        ctx_len = (steps + 1) * K * (2 if tiny else 8)
+        kv = [avsg.pinned_empty(ctx_len * stride) for _ in range(n_tab)]
+        for i, b in enumerate(kv):
+            tr.fill_kv(b.data_ptr(), 21, i, ctx_len, rb, row_stride=stride)
+        ctx = avsg.Context(num_tables=n_tab, buffer_slots=S, row_bytes=rb, max_topk=K, max_tokens=1, max_lifetime=16,
+                           index_mode=avsg.INDEX_DIRECT, max_context=ctx_len)
+        ctx.set_timing(True)
+        call = ctx.prepare(list(range(n_tab)), kv, 1, K, [stride] * n_tab)
+        perm = [rng.permutation(ctx_len).astype(np.int32) for _ in range(n_tab)]
+        us_k, us_e, sect, line, wire = [], [], 0, 0, 0
+        for t in range(steps):
+            ids = np.stack([np.sort(perm[i][t * K:(t + 1) * K]) for i in range(n_tab)])[:, None, :]    # never seen: all miss
+            X = torch.from_numpy(np.ascontiguousarray(ids)).cuda()
+            slots = torch.empty_like(X)
+            flush.fill_(t)
+            call.run(X, [ctx_len] * n_tab, slots, None, None, stream)
+            st = ctx.stats()
+            assert st["last_rows"] == n_tab * K
+            if t:
+                us_k.append(st["last_transfer_kernel_us"]); us_e.append(st["last_transfer_us"])
+                for x in ids.ravel()[:: max(1, ids.size // 4096)]:
+                    a, b, c = _row_wire_bytes(int(x) * stride % 128, rb, 24)
+                    sect += a; line += b; wire += c
+        n_s = len(ids.ravel()[:: max(1, ids.size // 4096)]) * (steps - 1)
+        ctx.close()
+        del kv
+        k_us = sum(us_k) / len(us_k)
+        rows.append({"link_model": True, "row_bytes": rb, "row_stride": stride, "rows_per_launch": n_tab * K,
+                     "in_kernel_us": k_us, "event_us": sum(us_e) / len(us_e), "ns_per_row": 1e3 * k_us / (n_tab * K),
+                     "gbs": n_tab * K * rb / 1e3 / k_us, "pct_of_link_peak": 100.0 * n_tab * K * rb / 1e3 / k_us / peak,
+                     "sectors_per_row": sect / n_s, "lines_per_row": line / n_s, "wire_bytes_per_row_H24": wire / n_s})
+    # fit: R from aligned full lines (the 1152-byte rows: 9 packets of 128 + H), H from the memcpy peak (256 + H per 256)
+    full = [r for r in rows if r["row_bytes"] == 1152][0]
+    t_line = full["ns_per_row"] / 9.0                                  # ns per (128 + H) bytes
+    t_256 = 256.0 / peak                                               # ns per (256 + H) bytes of the copy engine
+    H = (128.0 * t_256 - 256.0 * t_line) / (t_line - t_256)
+    R = (128.0 + H) / t_line
+    print(json.dumps({"link_model": "fit", "link_peak_gbs": peak, "header_bytes_H": H, "raw_rate_gbs_R": R,
+                      "model": LINK_MODEL["text"]}), flush=True)
+    for r in rows:
+        wire = r["sectors_per_row"] * 32 + (r["wire_bytes_per_row_H24"] - r["sectors_per_row"] * 32) / 24.0 * H
+        r["model_gbs"] = r["row_bytes"] / (wire / R)
+        r["model_pct_of_link_peak"] = 100.0 * r["model_gbs"] / peak
+        del r["wire_bytes_per_row_H24"]
+        print(json.dumps(r), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------------------
+# --breakdown: where the time of ONE call goes, for calls of different sizes (time marks the kernels take on the
+# GPU's own clock when timing is on; the event time of the same call around it)
+# ------------------------------------------------------------------------------------------------------------
+def run_breakdown(args):
+    import torch
+    import __graft_entry__
+    import avsg_traces as tr
+    __graft_entry__.build()
+    import paper_2609_37538_b200 as avsg
+    torch.cuda.set_device(0)
+    tiny = args.tiny
+    link_peak = _link_peak(torch, (64 << 20) if tiny else (1 << 30))
+    print(json.dumps({"breakdown": "link", "link_peak_gbs": link_peak}), flush=True)
+    cases = [("C2", dict(TINY["C2"]) if tiny else dict(n_iters=40)),
+             ("C3", dict(TINY["C3"], layers=1) if tiny else dict(requests=5, layers=1, n_iters=40)),
+             ("C4", dict(TINY["C4"]) if tiny else dict(n_iters=40)),
+             ("C3", dict(TINY["C3"], layers=1, requests=3) if tiny else dict(requests=32, layers=1, n_iters=40))]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    for name, kw in cases:
+        w = tr.workload(name, **kw)
+        traces = _gen_traces(w, os.cpu_count() or 1)
+        kv = []
+        for ti, cfg in enumerate(w.tables):
+            buf = avsg.pinned_empty(cfg.context * w.row_bytes)
+            tr.fill_kv(buf.data_ptr(), w.seed, ti, cfg.context, w.row_bytes)
+            kv.append(buf)
+        grp = w.calls[0]
+        X = [torch.from_numpy(np.stack([traces[ti][0][t] for ti in grp])).cuda() for t in range(w.n_iters)]
+        V = [[int(traces[ti][1][t]) for ti in grp] for t in range(w.n_iters)]
+        slots = torch.empty_like(X[0])
+        for mode, mname in ((avsg.XFER_SM_OVERLAP, "overlap"), (avsg.XFER_SM_BALANCED, "balanced")):
+            ctx = avsg.Context(num_tables=w.num_tables, buffer_slots=w.buffer_slots, row_bytes=w.row_bytes,
+                               max_topk=w.topk, max_tokens=w.n_q, max_lifetime=w.max_lifetime, transfer_mode=mode,
+                               index_mode=avsg.INDEX_DIRECT, max_context=max(c.context for c in w.tables) + w.n_q)
+            call = ctx.prepare(grp, [kv[t] for t in grp], w.n_q, w.topk)
+            untimed, rows_per = [], []
+            prev = ctx.stats()
+            # pass 1: the call as it runs in production (no events inside the library), CUDA events around it
+            for t in range(w.n_iters):
+                flush.fill_(t & 0xFF)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); call.run(X[t], V[t], slots, None, None, stream); e1.record()
+                torch.cuda.synchronize()
+                st = ctx.stats()
+                if t >= w.n_iters // 4:
+                    untimed.append(e0.elapsed_time(e1) * 1e3)
+                    rows_per.append(st["rows_copied"] - prev["rows_copied"])
+                prev = st
+            ctx.close()
+            # pass 2: the same calls with the time marks on
+            ctx = avsg.Context(num_tables=w.num_tables, buffer_slots=w.buffer_slots, row_bytes=w.row_bytes,
+                               max_topk=w.topk, max_tokens=w.n_q, max_lifetime=w.max_lifetime, transfer_mode=mode,
+                               index_mode=avsg.INDEX_DIRECT, max_context=max(c.context for c in w.tables) + w.n_q)
+            ctx.set_timing(True)
+            call = ctx.prepare(grp, [kv[t] for t in grp], w.n_q, w.topk)
+            marks = {k: [] for k in ("last_copy_start_us", "last_first_row_us", "last_first_block_done_us",
+                                     "last_call_kernel_us", "last_stage_one_kernel_us")}
+            for t in range(w.n_iters):
+                flush.fill_(t & 0xFF)
+                call.run(X[t], V[t], slots, None, None, stream)
+                st = ctx.stats()
+                if t >= w.n_iters // 4 and st["last_rows"] > 0:
+                    for k in marks:
+                        marks[k].append(st[k])
+            ctx.close()
+            mean = lambda v: sum(v) / max(1, len(v))
+            rows = mean(rows_per)
+            ev, copy_start, first_row = mean(untimed), mean(marks["last_copy_start_us"]), mean(marks["last_first_row_us"])
+            first_done, call_k = mean(marks["last_first_block_done_us"]), mean(marks["last_call_kernel_us"])
+            print(json.dumps({
+                "breakdown": name, "tables": len(grp), "stage_two": mname, "rows_per_call": rows,
+                "mb_per_call": rows * w.row_bytes / 1e6, "event_us_per_call": ev,
+                "gbs": rows * w.row_bytes / 1e3 / ev, "pct_of_link_peak": 100.0 * rows * w.row_bytes / 1e3 / ev / link_peak,
+                "split_us": {"launch_and_event_gap": ev - call_k, "stage_one_exposed": copy_start,
+                             "first_row": first_row - copy_start, "copy": first_done - first_row,
+                             "tail": call_k - first_done},
+                "stage_one_kernel_us": mean(marks["last_stage_one_kernel_us"]), "call_kernel_us": call_k}), flush=True)
+        del kv
+
+
+# ------------------------------------------------------------------------------------------------------------
 # --table3: the Stage Two strategies of App. D on the paper's grid (B x reuse, K = 2048, N_mtp = 0, 1152-byte rows)
 # ------------------------------------------------------------------------------------------------------------
 def run_table3(args):
@@ -913,12 +1092,22 @@ def main():
     ap.add_argument("--replays-table3", type=int, default=9)
     ap.add_argument("--sweeps", action="store_true",
                     help="extra report: Stage One K/S latency sweep, lifetime ablation, capacity study, MTP cold start")
+    ap.add_argument("--link-model", action="store_true",
+                    help="extra report: Stage Two's rate on all-miss steps by row size and alignment, against a packet "
+                         "model of the host link (1 GPU)")
+    ap.add_argument("--breakdown", action="store_true",
+                    help="extra report: where the time of one call goes (Stage One exposed, first row, copy, tail, "
+                         "launch gap) for calls of 0.2 .. 6 MB (1 GPU)")
     ap.add_argument("--suite", action="store_true",
                     help="extra report: C1..C5 hit rates, per-call times and the Stage Two comparators (1 GPU)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.sweeps:
+    if args.link_model:
+        run_link_model(args)
+    elif args.breakdown:
+        run_breakdown(args)
+    elif args.sweeps:
         run_sweeps(args)
     elif args.table3:
         run_table3(args)

@@ -75,9 +75,11 @@ extern "C" {
                                        resident while Stage One runs and starts on token
                                        g's misses, cut evenly over all SMs per token,
                                        while token g+1 is being placed.  Same results.
-                                       Calls with more than 1024 tables (128 with
-                                       AVSG_INDEX_PAPER) or more than 8 tokens run as
-                                       AVSG_XFER_SM_BALANCED                             */
+                                       Calls with more than 8 tokens, or whose Stage One
+                                       blocks (tables x stage_one_cluster) would take
+                                       more than half of the SMs, run as
+                                       AVSG_XFER_SM_BALANCED: there the overlap costs
+                                       more than it hides                                */
 
 /* How Stage One finds the slot that holds an id (same results either way). */
 #define AVSG_INDEX_HASH   0u  /* open-addressing table in shared memory, rebuilt every step     */
@@ -169,6 +171,14 @@ typedef struct {
     float    last_transfer_start_us;   /* first transfer block's start after the first Stage One
                                   block's start, same clock: below last_stage_one_kernel_us
                                   when AVSG_XFER_SM_OVERLAP overlaps the two                */
+    float    last_copy_start_us;       /* more marks of the last timed call, all counted from the
+                                  first Stage One block's start on the GPU's clock: the first
+                                  transfer block enters its copy loop (what precedes it is the
+                                  part of Stage One the call cannot hide),                   */
+    float    last_first_row_us;        /* the first row has arrived from host memory,           */
+    float    last_first_block_done_us; /* the first transfer block has copied its share (the
+                                  tail of the copy starts here),                             */
+    float    last_call_kernel_us;      /* the last block of either grid has ended               */
     float    reserved;
 } avsg_stats_t;
 

@@ -53,7 +53,9 @@ class AvsgStats(ctypes.Structure):
                 ("extra_decays", ctypes.c_uint64), ("last_stage_one_us", ctypes.c_float),
                 ("last_transfer_us", ctypes.c_float), ("last_rows", ctypes.c_uint64),
                 ("last_stage_one_kernel_us", ctypes.c_float), ("last_transfer_kernel_us", ctypes.c_float),
-                ("last_transfer_start_us", ctypes.c_float), ("reserved", ctypes.c_float)]
+                ("last_transfer_start_us", ctypes.c_float), ("last_copy_start_us", ctypes.c_float),
+                ("last_first_row_us", ctypes.c_float), ("last_first_block_done_us", ctypes.c_float),
+                ("last_call_kernel_us", ctypes.c_float), ("reserved", ctypes.c_float)]
 
 
 class AvsgNoAllocArgs(ctypes.Structure):

@@ -31,7 +31,7 @@ struct avsg_ctx {
                                                    //   one word with the sequence number of the last host-buffer call
     uint32_t* d_tcount = nullptr;                  //   and per-(table of the call, token) miss counts
     S1ParamsBig* big_args = nullptr;               // host: the large Stage One argument block, built in place per call
-    unsigned long long* d_trange = nullptr;        // [4] grid spans of the last timed call, then [4] their initial values
+    unsigned long long* d_trange = nullptr;        // [8] time marks of the last timed call, then [8] their initial values
     unsigned long long* d_trange_init = nullptr;
     int2* d_list = nullptr;
     SegDesc* d_seg = nullptr;
@@ -217,13 +217,19 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
                                ? (uint32_t)S1_MAX_TABLES : (uint32_t)S1_BIG_TABLES;
     if (mode == AVSG_XFER_SM_OVERLAP && (n > chunk || n_q > (uint32_t)OVERLAP_MAX_TOKENS))
         mode = AVSG_XFER_SM_BALANCED;                  // the overlapped kernel pairs with ONE Stage One launch
+    // The overlapped transfer grid shares the GPU with the Stage One grid it waits for.  When Stage One's blocks
+    // take more than half of the SMs, many transfer blocks only find room once Stage One is over and their fixed
+    // shares (Eq. 6) finish late: measured, a 96- or 128-table call is 3-6 % slower overlapped than not (64: 2 %
+    // faster).  Such calls run Stage Two after Stage One.
+    if (mode == AVSG_XFER_SM_OVERLAP && (uint64_t)n * c->s1_cluster > (uint64_t)c->sm_count / 2)
+        mode = AVSG_XFER_SM_BALANCED;
     // host buffers in the overlapped mode: no event between the two grids, the download waits for a sequence number
     const bool wait_on_sequence = host_io && mode == AVSG_XFER_SM_OVERLAP && c->wait_value64 != nullptr;
     // the position-level comparator reads the hit mask: use the library's own buffer if the caller wants none
     if (mode == AVSG_XFER_POSITION_LEVEL && !hit) hit = c->d_hit_stage;
     if (c->timing) {
         // grid spans: [0] Stage One first start, [1] its last end, [2], [3] the same for Stage Two
-        CU(cudaMemcpyAsync(c->d_trange, c->d_trange_init, 4 * sizeof(unsigned long long), cudaMemcpyDeviceToDevice, stream));
+        CU(cudaMemcpyAsync(c->d_trange, c->d_trange_init, 8 * sizeof(unsigned long long), cudaMemcpyDeviceToDevice, stream));
         CU(cudaEventRecord(c->ev[0], stream));
     }
 
@@ -442,7 +448,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaMalloc(&c->d_life, T * S) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_buffer, T * S * cfg->row_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_stats, T * sizeof(TableStats)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->d_trange, 8 * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_trange, 16 * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_ready, (OVERLAP_MAX_TOKENS + 3) * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_tcount, (size_t)OVERLAP_MAX_TABLES * OVERLAP_MAX_TOKENS * sizeof(uint32_t)) == cudaSuccess;
     c->big_args = new (std::nothrow) S1ParamsBig();
@@ -484,8 +490,11 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaEventCreateWithFlags(&c->ev_ids_ready, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) { cudaGetLastError(); free_all(c); delete c; return AVSG_ENOMEM; }
     {
-        const unsigned long long never = ~0ull, init[8] = {never, 0, never, 0, never, 0, never, 0};
-        c->d_trange_init = c->d_trange + 4;
+        // [0] Stage One first start, [1] its last end; Stage Two: [2] first start, [3] last end, [4] first copy loop,
+        // [5] first row in, [6] first block done; minima start at "never", maxima at 0
+        const unsigned long long never = ~0ull;
+        const unsigned long long init[16] = {never, 0, never, 0, never, never, never, 0, never, 0, never, 0, never, never, never, 0};
+        c->d_trange_init = c->d_trange + 8;
         if (cudaMemcpy(c->d_trange, init, sizeof(init), cudaMemcpyHostToDevice) != cudaSuccess ||
             cudaMemset(c->d_ready, 0, (OVERLAP_MAX_TOKENS + 3) * sizeof(unsigned long long)) != cudaSuccess) {
             free_all(c); delete c; return AVSG_ECUDA;
@@ -582,11 +591,18 @@ int avsg_stats(avsg_ctx* c, avsg_stats_t* out)
         if (cudaEventElapsedTime(&a, c->ev[0], c->ev[1]) == cudaSuccess) out->last_stage_one_us = a * 1000.f;
         if (cudaEventElapsedTime(&b, c->ev[1], c->ev[2]) == cudaSuccess) out->last_transfer_us = b * 1000.f;
         cudaGetLastError();
-        unsigned long long r[4];
+        unsigned long long r[8];
         CU(cudaMemcpy(r, c->d_trange, sizeof(r), cudaMemcpyDeviceToHost));
         if (r[1] > r[0]) out->last_stage_one_kernel_us = (float)(r[1] - r[0]) * 1e-3f;
         if (r[3] > r[2]) out->last_transfer_kernel_us = (float)(r[3] - r[2]) * 1e-3f;
         if (r[3] > r[2] && r[1] > r[0] && r[2] >= r[0]) out->last_transfer_start_us = (float)(r[2] - r[0]) * 1e-3f;
+        const unsigned long long never = ~0ull;
+        if (r[1] > r[0] && r[3] > r[2]) {                 // the other marks, all measured from Stage One's first start
+            if (r[4] != never && r[4] >= r[0]) out->last_copy_start_us = (float)(r[4] - r[0]) * 1e-3f;
+            if (r[5] != never && r[5] >= r[0]) out->last_first_row_us = (float)(r[5] - r[0]) * 1e-3f;
+            if (r[6] != never && r[6] >= r[0]) out->last_first_block_done_us = (float)(r[6] - r[0]) * 1e-3f;
+            if (r[3] >= r[0]) out->last_call_kernel_us = (float)((r[3] > r[1] ? r[3] : r[1]) - r[0]) * 1e-3f;
+        }
     }
     out->last_rows = out->rows_copied - c->last_rows;
     c->last_rows = out->rows_copied;

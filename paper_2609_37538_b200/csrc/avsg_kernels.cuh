@@ -122,7 +122,9 @@ struct XferParams {
     const int2*    miss_list;
     uint32_t*      status;
     uint32_t n_seg, list_stride, row_bytes, request_level, S;
-    unsigned long long* t_range = nullptr;      // timing on: [0] earliest block start, [1] latest block end (ns)
+    // timing on: [0] earliest block start, [1] latest block end, [2] earliest start of a block's copy loop,
+    // [3] earliest arrival of a block's first row, [4] earliest end of a block that copied something (ns)
+    unsigned long long* t_range = nullptr;
 };
 
 constexpr int OVERLAP_MAX_TOKENS = 8;

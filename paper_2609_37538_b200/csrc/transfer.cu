@@ -104,6 +104,8 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_kernel(const __grid_con
     }
 
     const uint32_t cpr = p.row_bytes >> 4;                     // 16-byte chunks per row
+    bool first_row = p.t_range != nullptr;                     // timing: when the copy starts, when its first row is in
+    if (first_row && tid == 0 && m1 > m0) atomicMin(p.t_range + 2, global_ns());
     for (uint32_t m = m0 + (tid >> 5); m < m1; m += nt >> 5) {
         uint32_t lo = 0, hi = n_seg;                           // largest lo with s_pref[lo] <= m
         while (hi - lo > 1) {
@@ -124,10 +126,18 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_kernel(const __grid_con
         const uint64_t src = __ldg(&p.seg[lo].src_base) + (uint64_t)(uint32_t)e.x * __ldg(&p.seg[lo].src_stride);
         const uint64_t dst = __ldg(&p.seg[lo].dst_base) + (uint64_t)(uint32_t)e.y * p.row_bytes;
         copy_row(src, dst, cpr, lane);
+        if (first_row) {
+            if (tid == 0) atomicMin(p.t_range + 3, global_ns());
+            first_row = false;
+        }
     }
     if (p.t_range) {
         __syncthreads();
-        if (tid == 0) atomicMax(p.t_range + 1, global_ns());
+        if (tid == 0) {
+            const unsigned long long t = global_ns();
+            atomicMax(p.t_range + 1, t);
+            if (m1 > m0) atomicMin(p.t_range + 4, t);          // the earliest block to finish: the tail starts here
+        }
     }
 }
 
@@ -170,6 +180,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __
     __syncthreads();
 
     const uint32_t cpr = p.row_bytes >> 4;
+    bool first_row = p.t_range != nullptr, copied = false;
     for (uint32_t g = 0; g < p.n_q; ++g) {
         if (tid == 0) {
             uint32_t ok = 0;
@@ -210,6 +221,8 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __
         const uint32_t C = gridDim.x, cb = blockIdx.x, q = running / C, r = running % C;
         const uint32_t m0 = cb * q + (cb < r ? cb : r);
         const uint32_t m1 = m0 + q + (cb < r ? 1u : 0u);
+        if (first_row && tid == 0 && m1 > m0) atomicMin(p.t_range + 2, global_ns());
+        copied = copied || m1 > m0;
         for (uint32_t m = m0 + (tid >> 5); m < m1; m += nt >> 5) {
             uint32_t lo = 0, hi = n;                               // largest lo with s_pref[lo] <= m
             while (hi - lo > 1) {
@@ -230,16 +243,25 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __
             const uint64_t src = s_src[lo] + (uint64_t)(uint32_t)e.x * s_stride[lo];
             const uint64_t dst = s_dst[lo] + (uint64_t)(uint32_t)e.y * p.row_bytes;
             copy_row(src, dst, cpr, lane);
+            if (first_row) {
+                if (tid == 0) atomicMin(p.t_range + 3, global_ns());
+                first_row = false;
+            }
         }
         __syncthreads();
         for (uint32_t i = tid; i < n; i += nt) s_off[i] += s_pref[i + 1] - s_pref[i];
         __syncthreads();
     }
+    unsigned long long t_copied = 0;
     if (p.t_range) {
         __syncthreads();
-        if (tid == 0) atomicMax(p.t_range + 1, global_ns());
+        t_copied = global_ns();
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (p.t_range && tid == 0) {
+        atomicMax(p.t_range + 1, global_ns());                     // the block's end, the wait for Stage One included
+        if (copied) atomicMin(p.t_range + 4, t_copied);
+    }
 }
 
 // Comparator S2 (App. D, Eq. 14): the n * N_q * K selected positions of the call are flattened and cut into

@@ -83,3 +83,24 @@ def test_sweeps_report_tiny():
     assert cold[0] == 0 and cold[3] > 0                                          # later tokens reuse earlier ones' rows
     idx = {r["index"]: r["hit_rate"] for r in rows if r["sweep"] == "index_mode"}
     assert idx["exact_hash"] == idx["exact_direct"] >= idx["paper_R3"]
+
+
+def test_breakdown_report_tiny():
+    rows = [r for r in _json_lines(["--breakdown", "--tiny"]) if r["breakdown"] != "link"]
+    assert len(rows) == 8 and {r["stage_two"] for r in rows} == {"overlap", "balanced"}
+    for r in rows:
+        sp = r["split_us"]
+        assert r["rows_per_call"] > 0 and r["event_us_per_call"] > 0
+        assert sp["stage_one_exposed"] > 0 and sp["first_row"] >= 0 and sp["copy"] >= 0 and sp["tail"] >= 0
+        assert abs(sum(sp.values()) - r["event_us_per_call"]) < 0.05 * r["event_us_per_call"] + 1.0
+
+
+def test_link_model_report_tiny():
+    rows = _json_lines(["--link-model", "--tiny"])
+    fit = [r for r in rows if r["link_model"] == "fit"][0]
+    assert fit["link_peak_gbs"] > 1 and "raw_rate_gbs_R" in fit and "header_bytes_H" in fit    # (no fit at this size)
+    geo = {(r["row_bytes"], r["row_stride"]): r for r in rows if r["link_model"] is True}
+    assert set(geo) == {(656, 656), (656, 768), (1152, 1152)}
+    assert geo[(1152, 1152)]["sectors_per_row"] == 36 and geo[(1152, 1152)]["lines_per_row"] == 9
+    assert geo[(656, 768)]["sectors_per_row"] == 21 and geo[(656, 768)]["lines_per_row"] == 6
+    assert geo[(656, 656)]["lines_per_row"] == 6 and 21 <= geo[(656, 656)]["sectors_per_row"] <= 22

@@ -258,7 +258,9 @@ def test_overlap_mode_four_tokens_and_mode_switches(avsg):
     assert ctx.sync_status() == 0
 
 
-@pytest.mark.parametrize("n,n_q,K,S", [(128, 2, 64, 256),      # as many tables as the small argument block takes
+@pytest.mark.parametrize("n,n_q,K,S", [(74, 2, 64, 256),       # Stage One on half of a B200's SMs: still overlapped
+                                        (75, 2, 64, 256),       # one more table: runs as the balanced mode
+                                        (128, 2, 64, 256),      # as many tables as the small argument block takes
                                         (5, 8, 96, 1024),       # as many tokens as the overlapped kernel takes
                                         (3, 9, 100, 1024),      # one more: runs as the balanced mode
                                         (129, 1, 32, 64),       # more tables than the small argument block takes
