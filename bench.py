@@ -113,6 +113,10 @@ def _workload(rank: int, n_iters: int, args=None, world: int = 1):
     kw = {}
     if args is not None:
         kw = {"requests": args.requests, "layers": args.layers}
+        if getattr(args, "buffer_slots", 0):
+            kw["buffer_slots"] = args.buffer_slots
+        if getattr(args, "n_tokens", 0):
+            kw["n_q"] = args.n_tokens
     if args is None or getattr(args, "scaling", "weak") == "weak" or world == 1:
         return tr.workload("C3", seed=3 + 1000 * rank, n_iters=n_iters, **kw)
     w = tr.workload("C3", seed=3, n_iters=n_iters, **kw)
@@ -463,7 +467,8 @@ def run_cuda(args):
                              "in L2 after the write, so DRAM traffic (scaled from the ncu capture of the one-layer case) is small; "
                              "timed in balanced mode (one kernel at a time); with --stage-two overlap the timed steps run "
                              "avsg_transfer_overlap_kernel, the same copy loop started per token while Stage One still runs"},
-        "roofline_stage_one": {"bound": "hbm", "kernel": "avsg_stage_one_kernel<%s>" % args.index, "achieved": s1_gbs, "peak": hbm_peak,
+        "roofline_stage_one": {"bound": "hbm", "kernel": ("avsg_stage_one_cluster_kernel<%s>" if w.buffer_slots > 8192 or args.cluster > 1
+                                                          else "avsg_stage_one_kernel<%s>") % args.index, "achieved": s1_gbs, "peak": hbm_peak,
                                "unit": "GB/s", "frac": s1_gbs / hbm_peak, "traffic": NCU_S1_DRAM_BYTES_PER_TABLE[args.index] * n_tab,
                                "peak_kind": peak_kind,
                                "bytes_per_launch": s1_bytes},
@@ -716,6 +721,8 @@ def run_link_model(args):
             (256, 256), (128, 128)]
     if tiny:
         geos = [(656, 656), (656, 768), (1152, 1152)]
+    if args.case:                                            # one geometry only (what an ncu capture runs)
+        geos = [tuple(int(v) for v in args.case.split(":"))]
     rows = []
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     stream = torch.cuda.current_stream()
@@ -752,6 +759,11 @@ def run_link_model(args):
                      "in_kernel_us": k_us, "event_us": sum(us_e) / len(us_e), "ns_per_row": 1e3 * k_us / (n_tab * K),
                      "gbs": n_tab * K * rb / 1e3 / k_us, "pct_of_link_peak": 100.0 * n_tab * K * rb / 1e3 / k_us / peak,
                      "sectors_per_row": sect / n_s, "lines_per_row": line / n_s, "wire_bytes_per_row_H24": wire / n_s})
+    if not any(r["row_bytes"] == 1152 for r in rows):
+        for r in rows:
+            del r["wire_bytes_per_row_H24"]
+            print(json.dumps(r), flush=True)
+        return
     # fit: R from aligned full lines (the 1152-byte rows: 9 packets of 128 + H), H from the memcpy peak (256 + H per 256)
     full = [r for r in rows if r["row_bytes"] == 1152][0]
     t_line = full["ns_per_row"] / 9.0                                  # ns per (128 + H) bytes
@@ -1067,6 +1079,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--requests", type=int, default=32, help="requests per layer (32 = the full configuration)")
     ap.add_argument("--layers", type=int, default=4, help="layers (4 = the full configuration)")
+    ap.add_argument("--buffer-slots", type=int, default=0,
+                    help="slots per table (0 = the configuration's 8192); above 8192 Stage One runs one thread-block "
+                         "cluster per table, e.g. --buffer-slots 16384 --n-tokens 4 for an MTP-3 deployment")
+    ap.add_argument("--n-tokens", type=int, default=0, help="query tokens per iteration (0 = the configuration's 2)")
     ap.add_argument("--index", default="direct", choices=["hash", "direct"],
                     help="Stage One index: direct-address table in device memory (default) or shared-memory hash table")
     ap.add_argument("--stage-two", default="overlap", choices=["balanced", "overlap"],
@@ -1095,6 +1111,7 @@ def main():
     ap.add_argument("--link-model", action="store_true",
                     help="extra report: Stage Two's rate on all-miss steps by row size and alignment, against a packet "
                          "model of the host link (1 GPU)")
+    ap.add_argument("--case", default="", help="with --link-model: only this ROW_BYTES:STRIDE geometry")
     ap.add_argument("--breakdown", action="store_true",
                     help="extra report: where the time of one call goes (Stage One exposed, first row, copy, tail, "
                          "launch gap) for calls of 0.2 .. 6 MB (1 GPU)")
