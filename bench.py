@@ -286,7 +286,15 @@ def run_cuda(args):
     del big_h, big_d
 
     # ---- warm-up (cold start + W-1 iterations), then the timed steps ----
-    for t in range(W):
+    # the first warm-up step is the COLD step (empty buffers: every id misses); it is timed on its own
+    flush.fill_(0)
+    ce0, ce1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ce0.record()
+    device_step(0)
+    ce1.record()
+    torch.cuda.synchronize()
+    cold_ms, cold_rows = ce0.elapsed_time(ce1), ctx.stats()["rows_copied"]
+    for t in range(1, W):
         device_step(t)
     torch.cuda.synchronize()
     st0 = ctx.stats()
@@ -377,8 +385,9 @@ def run_cuda(args):
 
     # ---- aggregate over ranks: device time = max over ranks, work = sum over ranks ----
     from paper_2609_37538_b200.sharding import aggregate
-    tmax, tsum = aggregate({"total_ms": total_ms, "e2e_ms": e2e_ms, "xus": sum(x_us), "warm_ms": warm_ms},
+    tmax, tsum = aggregate({"total_ms": total_ms, "e2e_ms": e2e_ms, "xus": sum(x_us), "warm_ms": warm_ms, "cold_ms": cold_ms},
                            {"rows": rows_timed, "xrows": sum(x_rows), "hits": hits_timed, "misses": miss_timed,
+                            "cold_rows": cold_rows,
                             "req_rate_sum": sum(req_rates), "req_n": len(req_rates)})
     total_ms_j, e2e_ms_j, xus_j = tmax["total_ms"], tmax["e2e_ms"], tmax["xus"]
     rows_j, xrows_j, hits_j, miss_j = tsum["rows"], tsum["xrows"], tsum["hits"], tsum["misses"]
@@ -459,6 +468,20 @@ def run_cuda(args):
                         "note": "per_call_*: CUDA events around the launch (what the roofline uses); in_kernel_*: first "
                                 "block's start to last block's end on the GPU's clock, without the launch gap"},
         "roofline": roofline,
+        "target": {
+            "stated": "miss-only gather at >= 0.80 of the measured pinned H2D bandwidth",
+            "cold_step": {"rows": tsum["cold_rows"], "ms": tmax["cold_ms"],
+                          "gbs": tsum["cold_rows"] * rb / 1e6 / tmax["cold_ms"],
+                          "frac": tsum["cold_rows"] * rb / 1e6 / tmax["cold_ms"] / link_peak / world,
+                          "note": "first step, empty buffers, all ids miss; whole step (4 calls), CUDA events"},
+            "steady_call_stage_two_events": {"frac": x_gbs / link_peak},
+            "steady_call_stage_two_in_kernel": {"frac": x_bytes_per_launch / 1e3 / (sum(x_kus) / len(x_kus)) / link_peak},
+            "steady_whole_call": {"frac": value / link_peak / world},
+            "met": {"cold_step": tsum["cold_rows"] * rb / 1e6 / tmax["cold_ms"] / link_peak / world >= 0.8,
+                    "steady_call_stage_two_events": x_gbs / link_peak >= 0.8,
+                    "steady_call_stage_two_in_kernel": x_bytes_per_launch / 1e3 / (sum(x_kus) / len(x_kus)) / link_peak >= 0.8},
+            "ceiling_note": "SM-issued reads of packed 656-byte rows reach 85.5 % of the copy peak at most on this link "
+                            "(bench.py --link-model); an event pair around one launch costs 6-7 us beyond the kernel's span"},
         "roofline_transfer_alone": {"bound": "host_link", "kernel": "avsg_transfer_kernel", "achieved": x_gbs, "peak": link_peak,
                      "unit": "GB/s", "frac": x_gbs / link_peak,
                      "traffic": NCU_XFER_DRAM_BYTES_PER_ROW * sum(x_rows) / n_launch,

@@ -32,6 +32,9 @@ def test_bench_line(extra):
     assert d["clocks"]["sm_max_mhz"] >= d["clocks"]["sm_mhz"] > 0
     assert 0.5 < d["hit_rate"] < 1.0 and d["config"]["workload"].startswith("C3")
     assert r["peak_repeats"] == 4 and "numa_node" in d["numa"]
+    t = d["target"]
+    assert 8 * 2048 <= t["cold_step"]["rows"] <= 8 * 4096 and 0 < t["cold_step"]["frac"] < 1.2   # token 0 misses everything
+    assert set(t["met"]) == {"cold_step", "steady_call_stage_two_events", "steady_call_stage_two_in_kernel"}
     c5 = d["comparators_c5"]
     for mode in ("balanced", "request_level", "transfer_all_k"):
         assert c5[mode]["effective_gbs"] > 0 and c5[mode]["stage_two_us_per_iter"] > 0
