@@ -441,6 +441,12 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     if (stage_one_prepare((size_t)max_smem) != cudaSuccess || stage_one_cluster_prepare((size_t)max_smem) != cudaSuccess) {
         delete c; return AVSG_ECUDA;
     }
+    // a cluster shape that fits on paper may still find no home on the device (blocks of one cluster share a GPC)
+    if (c->s1_cluster > 1 &&
+        stage_one_cluster_max_active(cfg->buffer_slots, cfg->max_topk, (uint32_t)cfg->max_lifetime, c->s1_cluster,
+                                     cfg->index_mode == AVSG_INDEX_DIRECT) < 1) {
+        delete c; return AVSG_EUNSUPPORTED;
+    }
 
     const size_t n_ids = T * c->list_stride;
     bool ok = true;

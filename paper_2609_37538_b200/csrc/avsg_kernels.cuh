@@ -187,6 +187,7 @@ cudaError_t launch_stage_one(const S1ParamsBig& p, uint32_t n_tables, cudaStream
 uint32_t stage_one_cluster_threads(uint32_t S, uint32_t C);
 size_t stage_one_cluster_smem_bytes(uint32_t S, uint32_t K, uint32_t L, uint32_t C, bool direct);
 cudaError_t stage_one_cluster_prepare(size_t max_smem);
+int stage_one_cluster_max_active(uint32_t S, uint32_t K, uint32_t L, uint32_t C, bool direct);   // after ..._prepare
 cudaError_t launch_stage_one_cluster(const S1Params& p, uint32_t n_tables, uint32_t C, cudaStream_t stream);
 cudaError_t launch_stage_one_cluster(const S1ParamsBig& p, uint32_t n_tables, uint32_t C, cudaStream_t stream);
 cudaError_t launch_direct_index_from_state(const int32_t* tok, uint16_t* where, uint32_t first_table, uint32_t n_tables,

@@ -514,6 +514,28 @@ cudaError_t launch_cluster_t(const S1ParamsT<CAP>& p, uint32_t n_tables, uint32_
 }
 }  // namespace
 
+// How many clusters of this shape the device can hold at once (0: the shape cannot be launched at all).
+int stage_one_cluster_max_active(uint32_t S, uint32_t K, uint32_t L, uint32_t C, bool direct)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(C);
+    cfg.blockDim = dim3(stage_one_cluster_threads(S, C));
+    cfg.dynamicSmemBytes = stage_one_cluster_smem_bytes(S, K, L, C, direct);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = C;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    const cudaError_t e = direct
+        ? cudaOccupancyMaxActiveClusters(&n, avsg_stage_one_cluster_kernel<true, S1_MAX_TABLES>, &cfg)
+        : cudaOccupancyMaxActiveClusters(&n, avsg_stage_one_cluster_kernel<false, S1_MAX_TABLES>, &cfg);
+    if (e != cudaSuccess) { cudaGetLastError(); return 0; }
+    return n;
+}
+
 cudaError_t launch_stage_one_cluster(const S1Params& p, uint32_t n_tables, uint32_t C, cudaStream_t stream)
 {
     return launch_cluster_t(p, n_tables, C, stream);
