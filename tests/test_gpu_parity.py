@@ -293,8 +293,9 @@ def test_overlap_mode_limits(avsg, n, n_q, K, S):
     assert ctx.sync_status() == 0
 
 
+@pytest.mark.parametrize("cluster", [0, 2])
 @pytest.mark.parametrize("mode_name", ["XFER_SM_BALANCED", "XFER_SM_OVERLAP"])
-def test_a_captured_call_can_be_replayed(avsg, mode_name):
+def test_a_captured_call_can_be_replayed(avsg, mode_name, cluster):
     """One avsg_step call captured in a CUDA graph and replayed for the following iterations: the ids and the
     verified lengths (which grow every iteration here) sit in device tensors that are refreshed in place, and the
     kernel arguments hold nothing else that changes from call to call."""
@@ -310,7 +311,7 @@ def test_a_captured_call_can_be_replayed(avsg, mode_name):
         tr.fill_kv(b.data_ptr(), 11, i, ctxlen, rb)
         kv.append(b)
     ctx = avsg.Context(n, S, rb, K, n_q, 16, transfer_mode=getattr(avsg, mode_name), index_mode=avsg.INDEX_DIRECT,
-                       max_context=ctxlen + n_q)
+                       max_context=ctxlen + n_q, stage_one_cluster=cluster)
     orc = [OracleTable(S, rb, 16) for _ in range(n)]
     call = ctx.prepare(list(range(n)), kv, n_q, K, None)
     X = torch.empty((n, n_q, K), dtype=torch.int32, device="cuda")
@@ -360,7 +361,8 @@ def test_stream_ordered_reset(avsg, mode_name, index_name):
     kv = avsg.pinned_empty(ctxlen * rb)
     tr.fill_kv(kv.data_ptr(), 21, 0, ctxlen, rb)
     ctx = avsg.Context(n, S, rb, K, n_q, 16, transfer_mode=getattr(avsg, mode_name),
-                       index_mode=getattr(avsg, index_name), max_context=ctxlen + n_q)
+                       index_mode=getattr(avsg, index_name), max_context=ctxlen + n_q,
+                       stage_one_cluster=4 if index_name == "INDEX_HASH" else 0)     # the hash runs also cover a cluster
     orc = [OracleTable(S, rb, 16) for _ in range(n)]
     stream = torch.cuda.Stream()
     with torch.cuda.stream(stream):
