@@ -782,6 +782,36 @@ def run_link_model(args):
                      "in_kernel_us": k_us, "event_us": sum(us_e) / len(us_e), "ns_per_row": 1e3 * k_us / (n_tab * K),
                      "gbs": n_tab * K * rb / 1e3 / k_us, "pct_of_link_peak": 100.0 * n_tab * K * rb / 1e3 / k_us / peak,
                      "sectors_per_row": sect / n_s, "lines_per_row": line / n_s, "wire_bytes_per_row_H24": wire / n_s})
+    # the same 656-byte rows, the same number of rows per launch, spread over more and more host memory
+    if not args.case:
+        for n_t, ctx_len in ((3, 4096), (3, 16384)) if tiny else ((16, 16384), (16, 131072), (16, 1 << 20)):
+            rb = stride = 656
+            kv = [avsg.pinned_empty(ctx_len * stride) for _ in range(n_t)]
+            for i, b in enumerate(kv):
+                tr.fill_kv(b.data_ptr(), 22, i, ctx_len, rb)
+            ctx = avsg.Context(num_tables=n_t, buffer_slots=S, row_bytes=rb, max_topk=K, max_tokens=1, max_lifetime=16,
+                               index_mode=avsg.INDEX_DIRECT, max_context=ctx_len)
+            ctx.set_timing(True)
+            call = ctx.prepare(list(range(n_t)), kv, 1, K)
+            perm = [rng.permutation(ctx_len).astype(np.int32) for _ in range(n_t)]
+            us_k = []
+            for t in range(steps):
+                ids = np.stack([np.sort(perm[i][t * K:(t + 1) * K]) for i in range(n_t)])[:, None, :]
+                X = torch.from_numpy(np.ascontiguousarray(ids)).cuda()
+                slots = torch.empty_like(X)
+                flush.fill_(t)
+                call.run(X, [ctx_len] * n_t, slots, None, None, stream)
+                st = ctx.stats()
+                assert st["last_rows"] == n_t * K
+                if t:
+                    us_k.append(st["last_transfer_kernel_us"])
+            ctx.close()
+            del kv
+            k_us = sum(us_k) / len(us_k)
+            print(json.dumps({"link_model": "span", "row_bytes": rb, "tables": n_t, "host_rows_per_table": ctx_len,
+                              "host_span_gb": n_t * ctx_len * stride / 1e9, "rows_per_launch": n_t * K, "in_kernel_us": k_us,
+                              "ns_per_row": 1e3 * k_us / (n_t * K), "gbs": n_t * K * rb / 1e3 / k_us,
+                              "pct_of_link_peak": 100.0 * n_t * K * rb / 1e3 / k_us / peak}), flush=True)
     if not any(r["row_bytes"] == 1152 for r in rows):
         for r in rows:
             del r["wire_bytes_per_row_H24"]

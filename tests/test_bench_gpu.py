@@ -102,6 +102,7 @@ def test_link_model_report_tiny():
     rows = _json_lines(["--link-model", "--tiny"])
     fit = [r for r in rows if r["link_model"] == "fit"][0]
     assert fit["link_peak_gbs"] > 1 and "raw_rate_gbs_R" in fit and "header_bytes_H" in fit    # (no fit at this size)
+    assert len([r for r in rows if r["link_model"] == "span"]) == 2
     geo = {(r["row_bytes"], r["row_stride"]): r for r in rows if r["link_model"] is True}
     assert set(geo) == {(656, 656), (656, 768), (1152, 1152)}
     assert geo[(1152, 1152)]["sectors_per_row"] == 36 and geo[(1152, 1152)]["lines_per_row"] == 9
