@@ -75,11 +75,14 @@ extern "C" {
                                        resident while Stage One runs and starts on token
                                        g's misses, cut evenly over all SMs per token,
                                        while token g+1 is being placed.  Same results.
-                                       Calls with more than 8 tokens, or whose Stage One
-                                       blocks (tables x stage_one_cluster) would take
-                                       more than half of the SMs, run as
-                                       AVSG_XFER_SM_BALANCED: there the overlap costs
-                                       more than it hides                                */
+                                       A call whose Stage One, with a block per table,
+                                       would take more than half of the SMs is served in
+                                       rounds of 32 tables: Stage One stays on 32 SMs and
+                                       the transfer copies round r's misses while round
+                                       r + 1 is matched.  Calls with more than 8 tokens
+                                       or 1024 tables, and large calls with a thread-
+                                       block cluster per table or AVSG_INDEX_PAPER, run
+                                       as AVSG_XFER_SM_BALANCED                          */
 
 /* How Stage One finds the slot that holds an id (same results either way). */
 #define AVSG_INDEX_HASH   0u  /* open-addressing table in shared memory, rebuilt every step     */

@@ -26,7 +26,7 @@ struct avsg_ctx {
     int8_t* d_life = nullptr;
     uint8_t* d_buffer = nullptr;
     TableStats* d_stats = nullptr;
-    unsigned long long* d_ready = nullptr;         // overlapped Stage Two: per-token counters [OVERLAP_MAX_TOKENS],
+    unsigned long long* d_ready = nullptr;         // overlapped Stage Two: per-round, per-token counters [OVERLAP_MAX_COUNTERS],
                                                    //   one word counting the transfer blocks that are through,
                                                    //   one word with the sequence number of the last host-buffer call
     uint32_t* d_tcount = nullptr;                  //   and per-(table of the call, token) miss counts
@@ -219,10 +219,19 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         mode = AVSG_XFER_SM_BALANCED;                  // the overlapped kernel pairs with ONE Stage One launch
     // The overlapped transfer grid shares the GPU with the Stage One grid it waits for.  When Stage One's blocks
     // take more than half of the SMs, many transfer blocks only find room once Stage One is over and their fixed
-    // shares (Eq. 6) finish late: measured, a 96- or 128-table call is 3-6 % slower overlapped than not (64: 2 %
-    // faster).  Such calls run Stage Two after Stage One.
-    if (mode == AVSG_XFER_SM_OVERLAP && (uint64_t)n * c->s1_cluster > (uint64_t)c->sm_count / 2)
-        mode = AVSG_XFER_SM_BALANCED;
+    // shares (Eq. 6) finish late: measured, a 96- or 128-table call with one Stage One block per table is 3-6 %
+    // slower overlapped than not (64: 2 % faster).
+    // Such calls keep Stage One on S1_ROUND_BLOCKS SMs: its blocks serve the tables round by round and the transfer
+    // grid, resident on the other SMs, copies round r's misses while round r + 1 is matched (single-block hash /
+    // direct kernels; the cluster and paper-literal kernels run Stage Two after Stage One instead).
+    uint32_t round_size = n;
+    if (mode == AVSG_XFER_SM_OVERLAP && (uint64_t)n * c->s1_cluster > (uint64_t)c->sm_count / 2) {
+        const uint32_t rounds = (n + S1_ROUND_BLOCKS - 1u) / S1_ROUND_BLOCKS;
+        if (c->s1_cluster == 1 && c->cfg.index_mode != AVSG_INDEX_PAPER && rounds * n_q <= (uint32_t)OVERLAP_MAX_COUNTERS)
+            round_size = S1_ROUND_BLOCKS;
+        else
+            mode = AVSG_XFER_SM_BALANCED;
+    }
     // host buffers in the overlapped mode: no event between the two grids, the download waits for a sequence number
     const bool wait_on_sequence = host_io && mode == AVSG_XFER_SM_OVERLAP && c->wait_value64 != nullptr;
     // the position-level comparator reads the hit mask: use the library's own buffer if the caller wants none
@@ -254,6 +263,7 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         p.S = c->cfg.buffer_slots; p.logH = c->logH; p.row_bytes = c->cfg.row_bytes;
         p.K = K; p.n_q = n_q; p.L = (uint32_t)c->cfg.max_lifetime;
         p.first = first; p.list_stride = c->list_stride;
+        p.n_launch = cnt; p.round_size = round_size;
         p.where = c->d_where; p.max_context = c->cfg.max_context;
         p.qword = c->d_q; p.probe_retries = c->cfg.probe_retries; p.hash_a1 = c->cfg.hash_a1; p.hash_a2 = c->cfg.hash_a2;
         p.t_range = c->timing ? c->d_trange : nullptr;
@@ -262,8 +272,8 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         const bool overlap = mode == AVSG_XFER_SM_OVERLAP;
         p.ready = overlap ? c->d_ready : nullptr;
         p.tcount = overlap ? c->d_tcount : nullptr;
-        p.done_seq = wait_on_sequence ? c->d_ready + OVERLAP_MAX_TOKENS + 1 : nullptr;
-        p.done_ctr = reinterpret_cast<uint32_t*>(c->d_ready + OVERLAP_MAX_TOKENS + 2);
+        p.done_seq = wait_on_sequence ? c->d_ready + OVERLAP_MAX_COUNTERS + 1 : nullptr;
+        p.done_ctr = reinterpret_cast<uint32_t*>(c->d_ready + OVERLAP_MAX_COUNTERS + 2);
         p.host_seq = wait_on_sequence ? c->host_seq + 1 : 0;
         p.expect = n;
         for (uint32_t i = 0; i < cnt; ++i) {
@@ -274,7 +284,7 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
             p.kv_stride[i] = a->row_stride ? a->row_stride[first + i] : c->cfg.row_bytes;
         }
         if (c->s1_cluster > 1) CU(launch_stage_one_cluster(p, cnt, c->s1_cluster, stream));
-        else CU(launch_stage_one(p, cnt, stream));
+        else CU(launch_stage_one(p, cnt < round_size ? cnt : round_size, stream));
         return AVSG_OK;
     };
     for (uint32_t first = 0; first < n; first += chunk) {
@@ -330,22 +340,22 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         XferOverlapParams x;
         x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
         x.tcount = c->d_tcount; x.ready = c->d_ready;
-        x.done = reinterpret_cast<uint32_t*>(c->d_ready + OVERLAP_MAX_TOKENS);
+        x.done = reinterpret_cast<uint32_t*>(c->d_ready + OVERLAP_MAX_COUNTERS);
         x.n = n; x.n_q = n_q; x.list_stride = c->list_stride; x.row_bytes = c->cfg.row_bytes; x.S = c->cfg.buffer_slots;
-        x.expect = n;
+        x.round_size = round_size; x.expect_extra = 0;
         x.t_range = c->timing ? c->d_trange + 2 : nullptr;
         if (launch_transfer_overlap(x, c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count, c->xfer_threads, stream)
             != cudaSuccess) {
             // Stage One has run and raised the per-token counters, nothing will lower them: do it here, in
             // stream order, and remember that this call reserved slots whose rows were never copied
             cudaGetLastError();
-            cudaMemsetAsync(c->d_ready, 0, (OVERLAP_MAX_TOKENS + 1) * sizeof(unsigned long long), stream);
+            cudaMemsetAsync(c->d_ready, 0, (OVERLAP_MAX_COUNTERS + 1) * sizeof(unsigned long long), stream);
             c->host_status |= AVSG_STATUS_LAUNCH_FAILED;
             return AVSG_ECUDA;
         }
         if (wait_on_sequence) {
             c->host_seq += 1;
-            if (c->wait_value64(c->side, reinterpret_cast<CUdeviceptr>(c->d_ready + OVERLAP_MAX_TOKENS + 1), c->host_seq,
+            if (c->wait_value64(c->side, reinterpret_cast<CUdeviceptr>(c->d_ready + OVERLAP_MAX_COUNTERS + 1), c->host_seq,
                                 CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
                 return AVSG_ECUDA;
             if ((rc = download_outputs()) != AVSG_OK) return rc;
@@ -455,7 +465,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaMalloc(&c->d_buffer, T * S * cfg->row_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_stats, T * sizeof(TableStats)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_trange, 16 * sizeof(unsigned long long)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->d_ready, (OVERLAP_MAX_TOKENS + 3) * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_ready, (OVERLAP_MAX_COUNTERS + 3) * sizeof(unsigned long long)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_tcount, (size_t)OVERLAP_MAX_TABLES * OVERLAP_MAX_TOKENS * sizeof(uint32_t)) == cudaSuccess;
     c->big_args = new (std::nothrow) S1ParamsBig();
     ok = ok && c->big_args != nullptr;
@@ -502,7 +512,7 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
         const unsigned long long init[16] = {never, 0, never, 0, never, never, never, 0, never, 0, never, 0, never, never, never, 0};
         c->d_trange_init = c->d_trange + 8;
         if (cudaMemcpy(c->d_trange, init, sizeof(init), cudaMemcpyHostToDevice) != cudaSuccess ||
-            cudaMemset(c->d_ready, 0, (OVERLAP_MAX_TOKENS + 3) * sizeof(unsigned long long)) != cudaSuccess) {
+            cudaMemset(c->d_ready, 0, (OVERLAP_MAX_COUNTERS + 3) * sizeof(unsigned long long)) != cudaSuccess) {
             free_all(c); delete c; return AVSG_ECUDA;
         }
     }
@@ -647,8 +657,8 @@ int avsg_clear_status(avsg_ctx* c)
     CU(cudaDeviceSynchronize());
     CU(cudaMemset(c->d_status, 0, sizeof(uint32_t)));
     // a transfer kernel that gave up may have left the per-token counters of the overlapped mode raised
-    CU(cudaMemset(c->d_ready, 0, (OVERLAP_MAX_TOKENS + 1) * sizeof(unsigned long long)));    // not the sequence word
-    CU(cudaMemset(c->d_ready + OVERLAP_MAX_TOKENS + 2, 0, sizeof(unsigned long long)));      // arrivals after the last token
+    CU(cudaMemset(c->d_ready, 0, (OVERLAP_MAX_COUNTERS + 1) * sizeof(unsigned long long)));    // not the sequence word
+    CU(cudaMemset(c->d_ready + OVERLAP_MAX_COUNTERS + 2, 0, sizeof(unsigned long long)));      // arrivals after the last token
     c->host_status = 0;
     return AVSG_OK;
 }
@@ -661,9 +671,9 @@ int avsg_probe_wait_limit(avsg_ctx* c, void* cuda_stream)
     XferOverlapParams x;
     x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
     x.tcount = c->d_tcount; x.ready = c->d_ready;
-    x.done = reinterpret_cast<uint32_t*>(c->d_ready + OVERLAP_MAX_TOKENS);
+    x.done = reinterpret_cast<uint32_t*>(c->d_ready + OVERLAP_MAX_COUNTERS);
     x.n = 1; x.n_q = 1; x.list_stride = c->list_stride; x.row_bytes = c->cfg.row_bytes; x.S = c->cfg.buffer_slots;
-    x.expect = 1;                                       // one table's token that no Stage One will place
+    x.round_size = 1; x.expect_extra = 0;               // one table's token that no Stage One will place
     CU(launch_transfer_overlap(x, c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count, c->xfer_threads,
                                static_cast<cudaStream_t>(cuda_stream)));
     return AVSG_OK;

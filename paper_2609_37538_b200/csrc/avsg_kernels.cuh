@@ -90,14 +90,17 @@ struct S1ParamsT {
     int32_t*       miss_count;   // [n][n_q] or null
     uint32_t S, logH, row_bytes, K, n_q, L;
     uint32_t first;              // index within the call of this launch's first table
+    uint32_t n_launch;           // tables of this launch (the grid may have fewer blocks: a block then serves several)
+    uint32_t round_size;         // overlapped Stage Two: tables per publication round (= grid size of Stage One)
     uint32_t list_stride;        // entries per segment of miss_list
     uint32_t max_context;        // direct index: entries per table
     uint16_t* where;             // direct index [num_tables][max_context], or null for the hash index
     uint32_t* qword;             // paper-literal mode: packed metadata words [num_tables][S], else null
     uint32_t probe_retries, hash_a1, hash_a2;   // paper-literal mode: R, a1, a2
     unsigned long long* t_range = nullptr;      // timing on: [0] earliest block start, [1] latest block end (ns)
-    // overlapped Stage Two (null otherwise): ready[g] counts the tables of this call whose token g is placed (the
-    // transfer kernel zeroes it again); tcount[ti * n_q + g] = misses of token g of the ti-th table of the call
+    // overlapped Stage Two (null otherwise): ready[r * n_q + g] counts the tables of round r of this call whose token
+    // g is placed (the transfer kernel zeroes it again); round r = tables [r * round_size, (r + 1) * round_size) of
+    // the call; tcount[ti * n_q + g] = misses of token g of the ti-th table of the call
     unsigned long long* ready = nullptr;
     uint32_t*           tcount = nullptr;
     // calls with host buffers in that mode (null otherwise): the table that places the call's last token last
@@ -128,6 +131,8 @@ struct XferParams {
 };
 
 constexpr int OVERLAP_MAX_TOKENS = 8;
+constexpr int OVERLAP_MAX_COUNTERS = 512;            // rounds x tokens of one call
+constexpr uint32_t S1_ROUND_BLOCKS = 32;             // Stage One blocks of a call that is served in rounds
 constexpr int OVERLAP_MAX_TABLES = S1_BIG_TABLES;   // one Stage One launch
 constexpr uint32_t OVERLAP_SPIN_LIMIT = 1u << 18;   // polls before the wait gives up; a poll is an L2 round trip plus a 64 ns sleep, ~0.8 us measured: ~0.2 s
 
@@ -136,10 +141,11 @@ struct XferOverlapParams {       // Stage Two that starts on token g's misses wh
     const int2*    miss_list;
     uint32_t*      status;
     const uint32_t* tcount;      // [n][n_q]
-    unsigned long long* ready;   // [OVERLAP_MAX_TOKENS] tables that have placed token g; zero between calls
+    unsigned long long* ready;   // [rounds][n_q] tables of the round that have placed token g; zero between calls
     uint32_t*      done;         // blocks of this grid that are through; zero between calls
     uint32_t n, n_q, list_stride, row_bytes, S;
-    uint32_t expect;             // value ready[g] reaches: n, or more than that for the wait-limit diagnostic
+    uint32_t round_size;         // tables per round (n: one round)
+    uint32_t expect_extra;       // added to what a counter must reach: 0, or 1 for the wait-limit diagnostic
     unsigned long long* t_range = nullptr;
 };
 
@@ -181,8 +187,9 @@ size_t stage_one_smem_bytes(uint32_t S, uint32_t K, uint32_t L, bool direct = fa
 size_t stage_one_paper_smem_bytes(uint32_t S, uint32_t K, uint32_t L);
 uint32_t stage_one_threads(uint32_t S, uint32_t K);
 cudaError_t stage_one_prepare(size_t max_smem);
-cudaError_t launch_stage_one(const S1Params& p, uint32_t n_tables, cudaStream_t stream);
-cudaError_t launch_stage_one(const S1ParamsBig& p, uint32_t n_tables, cudaStream_t stream);   // hash / direct index only
+// n_blocks thread blocks serve the p.n_launch tables of the launch (one block per table unless the call runs in rounds)
+cudaError_t launch_stage_one(const S1Params& p, uint32_t n_blocks, cudaStream_t stream);
+cudaError_t launch_stage_one(const S1ParamsBig& p, uint32_t n_blocks, cudaStream_t stream);   // hash / direct index only
 // Stage One with one table per thread-block cluster of C blocks (C = 2, 4 or 8; hash / direct index only)
 uint32_t stage_one_cluster_threads(uint32_t S, uint32_t C);
 size_t stage_one_cluster_smem_bytes(uint32_t S, uint32_t K, uint32_t L, uint32_t C, bool direct);

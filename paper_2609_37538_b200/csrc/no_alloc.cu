@@ -93,6 +93,7 @@ extern "C" int avsg_step_noalloc(const avsg_noalloc_args* a, void* cuda_stream)
     p.indices = a->indices; p.slots = a->slots; p.hit = a->hit; p.miss_count = a->miss_count;
     p.S = a->buffer_slots; p.row_bytes = a->row_bytes; p.K = a->topk; p.n_q = a->n_tokens;
     p.L = (uint32_t)a->max_lifetime; p.first = 0; p.list_stride = list_stride;
+    p.n_launch = a->n; p.round_size = a->n;
     p.where = nullptr; p.max_context = 0;
     p.qword = nullptr; p.probe_retries = 0; p.hash_a1 = 0; p.hash_a2 = 0;
     p.logH = 1;

@@ -115,7 +115,7 @@ __device__ __forceinline__ void build_index(const Index& ix, const int32_t* s_to
     if ((threadIdx.x & 31u) == 0 && live) atomicAdd(s_fill, live);
 }
 
-template <bool DIRECT, int CAP>
+template <bool DIRECT, int CAP, bool ROUNDS>
 __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_constant__ S1ParamsT<CAP> p)
 {
     extern __shared__ __align__(16) unsigned char smem[];
@@ -137,20 +137,6 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
     const uint32_t priv_stride = nt + 4u;                 // +4: rows start in different banks
     uint8_t*  s_priv     = L <= PRIV_HIST_MAX_L ? reinterpret_cast<uint8_t*>(s_fill + 8) : nullptr;
 
-    const uint32_t ti = p.first + blockIdx.x;            // table index within the call
-    const uint32_t table = p.table_id[blockIdx.x];
-    int32_t* g_tok = p.tok + (size_t)table * S;
-    int8_t*  g_life = p.life + (size_t)table * S;
-
-    const uint32_t spt = S >= nt ? S / nt : 1u;           // slots per thread, power of two <= 8
-    const uint32_t j0 = tid * spt;
-    const bool own = j0 < S;
-    const uint32_t ipt = (K + nt - 1) / nt;               // ids per thread, <= 8
-    const uint32_t i0 = tid * ipt;
-
-    Index ix{s_key, s_val, s_tok, H - 1u, p.logH};
-    uint16_t* where = DIRECT ? p.where + (size_t)table * p.max_context : nullptr;
-
     // Programmatic dependent launch: this grid may have been started while the previous kernel of the stream
     // was still running; nothing is read before that kernel has completed.  The next kernel (Stage Two) is
     // allowed to start its own prologue right away - it waits the same way before it reads the miss list.
@@ -158,229 +144,258 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (p.t_range && threadIdx.x == 0) atomicMin(p.t_range, global_ns());
 
-    // ---- issue every global load first: table state and the first token's ids ----
-    int4 t4[MAX_SPT / 4];
-    int32_t t1[3];
-    uint32_t lw0, lw1;
-    if (own) {
-        if ((spt & 3u) == 0) {
-#pragma unroll
-            for (uint32_t q = 0; q < (uint32_t)MAX_SPT / 4; ++q)
-                if (q < spt / 4) t4[q] = __ldg(reinterpret_cast<const int4*>(g_tok + j0) + q);
-        } else {
-#pragma unroll
-            for (uint32_t k = 0; k < 3; ++k)
-                if (k < spt) t1[k] = __ldg(g_tok + j0 + k);
-        }
-    }
-    life_load(g_life, j0, spt, own, lw0, lw1);
-    int32_t xs[MAX_IPT];
-    load_ids(p.indices + (size_t)ti * p.n_q * K, i0, ipt, K, xs);
-    const uint32_t id_limit = p.id_limit[blockIdx.x];
+    // The grid usually has one block per table (ROUNDS = false: one pass, bt = blockIdx.x).  A call with many tables
+    // and an overlapped Stage Two is launched with fewer blocks than tables (ROUNDS = true): a block then serves the
+    // tables bt = blockIdx.x, blockIdx.x + gridDim.x, ... one after the other, so that Stage One stays on a few SMs
+    // and publishes its tables round by round while the transfer grid, resident on the other SMs, already copies
+    // the earlier rounds' misses.
+    auto one_table = [&](const uint32_t bt) {
+        const uint32_t ti = p.first + bt;            // table index within the call
+        const uint32_t table = p.table_id[bt];
+        int32_t* g_tok = p.tok + (size_t)table * S;
+        int8_t*  g_life = p.life + (size_t)table * S;
 
-    if constexpr (!DIRECT) {
-        for (uint32_t i = tid; i < H / 4; i += nt)
-            reinterpret_cast<int4*>(s_key)[i] = make_int4(EMPTY, EMPTY, EMPTY, EMPTY);
-    }
-    if (s_priv)
-        for (uint32_t i = tid; i < ((uint32_t)(L + 2) * priv_stride + 15u) / 16u; i += nt)
-            reinterpret_cast<int4*>(s_priv)[i] = make_int4(0, 0, 0, 0);
-    if (tid == 0) *s_fill = 0;
-    if (own) {
-        if ((spt & 3u) == 0) {
-#pragma unroll
-            for (uint32_t q = 0; q < (uint32_t)MAX_SPT / 4; ++q)
-                if (q < spt / 4) reinterpret_cast<int4*>(s_tok + j0)[q] = t4[q];
-        } else {
-#pragma unroll
-            for (uint32_t k = 0; k < 3; ++k)
-                if (k < spt) s_tok[j0 + k] = t1[k];
-        }
-    }
-    // global pre-decay of the iteration's first token (Alg. 1 Pass 1)
-    life_store(s_life, j0, spt, own, decay4(lw0, 1), decay4(lw1, 1));
-    __syncthreads();
-    uint32_t fill_bound = 0;                              // hash index: non-empty buckets (upper bound)
-    if (!DIRECT) {
-        build_index(ix, s_tok, j0, spt, own, s_fill, p.status);
-        __syncthreads();
-        fill_bound = *s_fill;
-    }
+        const uint32_t spt = S >= nt ? S / nt : 1u;           // slots per thread, power of two <= 8
+        const uint32_t j0 = tid * spt;
+        const bool own = j0 < S;
+        const uint32_t ipt = (K + nt - 1) / nt;               // ids per thread, <= 8
+        const uint32_t i0 = tid * ipt;
 
-    uint32_t list_off = 0, sum_valid = 0, sum_miss = 0, sum_decay = 0;
-    int2* list = p.miss_list + (size_t)ti * p.list_stride;
+        Index ix{s_key, s_val, s_tok, H - 1u, p.logH};
+        uint16_t* where = DIRECT ? p.where + (size_t)table * p.max_context : nullptr;
 
-
-    for (uint32_t g = 0; g < p.n_q; ++g) {
-        const size_t row = ((size_t)ti * p.n_q + g) * K;
-        int32_t* O = p.slots + row;
-        uint8_t* Hm = p.hit ? p.hit + row : nullptr;
-        if (tid < 128) s_hist[tid] = 0;
-
-        // ---- Probe, refresh hits to L, emit hit slots (Pass 1 + Pass 2) ----
-        uint32_t missmask = 0, nmiss = 0, nvalid = 0;
-        uint32_t cand[MAX_IPT];                             // direct index: candidate slot per id
-        check_ids(xs, i0, ipt, K, id_limit, p.status);      // out-of-range ids become padding (id_limit <= max_context)
-        if (DIRECT) {
-#pragma unroll
-            for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {   // all loads are issued before any is used
-                cand[k] = 0xFFFFFFFFu;
-                if (k < ipt && i0 + k < K && xs[k] >= 0) cand[k] = __ldcg(where + xs[k]) & (S - 1u);
-            }
-        }
-#pragma unroll
-        for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {
-            const uint32_t i = i0 + k;
-            if (k < ipt && i < K) {
-                const int32_t x = xs[k];
-                if (x >= 0 && (!DIRECT || cand[k] != 0xFFFFFFFFu)) {
-                    ++nvalid;
-                    int32_t j;
-                    if (DIRECT) j = s_tok[cand[k]] == x ? (int32_t)cand[k] : -1;
-                    else j = index_find(ix, x, p.status);
-                    if (j >= 0) {
-                        s_life[j] = (int8_t)L;
-                        O[i] = j;
-                        if (Hm) Hm[i] = 1;
-                    } else {
-                        missmask |= 1u << k;
-                        ++nmiss;
-                    }
-                } else {
-                    O[i] = -1;
-                    if (Hm) Hm[i] = 0;
-                }
-            }
-        }
-        // order-preserving compaction of the misses: t = x[not m]
-        uint32_t total;
-        uint32_t off = block_excl_scan(nmiss | (nvalid << 16), s_scan_a, total) & 0xFFFFu;
-        const uint32_t n_g = total & 0xFFFFu;
-        sum_valid += total >> 16;
-        sum_miss += n_g;
-#pragma unroll
-        for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {
-            if (missmask & (1u << k)) {
-                s_miss_x[off] = xs[k];
-                s_miss_pos[off] = (uint16_t)(i0 + k);
-                ++off;
-            }
-        }
-        // the next token's ids travel while this token's misses are placed
-        if (g + 1 < p.n_q) load_ids(p.indices + row + K, i0, ipt, K, xs);
-        if (tid == 0 && p.miss_count) p.miss_count[(size_t)ti * p.n_q + g] = (int32_t)n_g;
-        if (n_g == 0) { __syncthreads(); publish_token(p, ti, table, g, 0, blockIdx.x); continue; }
-        __syncthreads();
-
-        // ---- Pass 3: CollectDead; if fewer than n_g slots are dead, decay until enough are ----
-        uint32_t w0, w1;
-        life_load(s_life, j0, spt, own, w0, w1);
-        uint32_t sg0 = w0 & 0x80808080u, sg1 = w1 & 0x80808080u;       // sign bits = dead slots
-        uint32_t dtotal, d = 0;
-        uint32_t doff = block_excl_scan(__popc(sg0) + __popc(sg1), s_scan_b, dtotal);
-        if (dtotal < n_g) {
-            // the while-loop of Alg. 1 in closed form: d = fewest unit decays after which n_g slots are dead,
-            // read off the histogram of the lifetimes (only needed on this, the rarer, path)
-            count_lifetimes(w0, w1, spt, own, L, s_priv, priv_stride, s_hist);
-            __syncthreads();
-            uint32_t cum = 0;
-            bool found = false;
-            d = (uint32_t)L + 1u;
-            for (uint32_t b = 0; b <= (uint32_t)L + 1u; ++b) {   // bin b counts lifetime b-1; dead after b decays
-                cum += s_hist[b];
-                if (cum >= n_g) { d = b; found = true; break; }
-            }
-            if (!found && tid == 0) atomicOr(p.status, ST_NO_DEAD_SLOTS);
-            w0 = decay4(w0, d);
-            w1 = decay4(w1, d);
-            life_store(s_life, j0, spt, own, w0, w1);
-            sg0 = w0 & 0x80808080u; sg1 = w1 & 0x80808080u;
-            doff = block_excl_scan(__popc(sg0) + __popc(sg1), s_scan_b, dtotal);
-        }
-        // dead slots in increasing order; the first n_g are handed out
-#pragma unroll
-        for (uint32_t k = 0; k < (uint32_t)MAX_SPT; ++k) {
-            const uint32_t bit = k < 4 ? (sg0 >> (8 * k + 7)) & 1u : (sg1 >> (8 * (k - 4) + 7)) & 1u;
-            if (bit) {
-                if (doff < n_g) s_dead[doff] = (uint16_t)(j0 + k);
-                ++doff;
-            }
-        }
-        __syncthreads();
-
-        // ---- install the misses: k-th miss takes the k-th dead slot ----
-        const bool rebuild = !DIRECT && fill_bound + n_g > (H / 4u) * 3u;
-        const uint32_t n_take = n_g < dtotal ? n_g : dtotal;
-        for (uint32_t k = tid; k < n_take; k += nt) {
-            const uint32_t j = s_dead[k];
-            const int32_t x = s_miss_x[k];
-            const uint32_t i = s_miss_pos[k];
-            if (j < S && i < K) {
-                s_tok[j] = x;
-                s_life[j] = (int8_t)L;
-                O[i] = (int32_t)j;
-                if (Hm) Hm[i] = 0;
-                list[list_off + k] = make_int2(x, (int32_t)j);
-                if (DIRECT) __stcg(where + x, (uint16_t)j);
-                else if (!rebuild) index_insert(ix, x, j, p.status);
+        // ---- issue every global load first: table state and the first token's ids ----
+        int4 t4[MAX_SPT / 4];
+        int32_t t1[3];
+        uint32_t lw0, lw1;
+        if (own) {
+            if ((spt & 3u) == 0) {
+    #pragma unroll
+                for (uint32_t q = 0; q < (uint32_t)MAX_SPT / 4; ++q)
+                    if (q < spt / 4) t4[q] = __ldg(reinterpret_cast<const int4*>(g_tok + j0) + q);
             } else {
-                list[list_off + k] = make_int2(-1, -1);          // Stage Two skips it
-                atomicOr(p.status, ST_BAD_SLOT);
+    #pragma unroll
+                for (uint32_t k = 0; k < 3; ++k)
+                    if (k < spt) t1[k] = __ldg(g_tok + j0 + k);
             }
         }
-        list_off += n_take;
-        sum_decay += d;
-        if (!rebuild) {
-            fill_bound += n_g;
-            __syncthreads();
-        } else if constexpr (!DIRECT) {
-            __syncthreads();
+        life_load(g_life, j0, spt, own, lw0, lw1);
+        int32_t xs[MAX_IPT];
+        load_ids(p.indices + (size_t)ti * p.n_q * K, i0, ipt, K, xs);
+        const uint32_t id_limit = p.id_limit[bt];
+
+        if constexpr (!DIRECT) {
             for (uint32_t i = tid; i < H / 4; i += nt)
                 reinterpret_cast<int4*>(s_key)[i] = make_int4(EMPTY, EMPTY, EMPTY, EMPTY);
-            if (tid == 0) *s_fill = 0;
-            __syncthreads();
+        }
+        if (s_priv)
+            for (uint32_t i = tid; i < ((uint32_t)(L + 2) * priv_stride + 15u) / 16u; i += nt)
+                reinterpret_cast<int4*>(s_priv)[i] = make_int4(0, 0, 0, 0);
+        if (tid == 0) *s_fill = 0;
+        if (own) {
+            if ((spt & 3u) == 0) {
+    #pragma unroll
+                for (uint32_t q = 0; q < (uint32_t)MAX_SPT / 4; ++q)
+                    if (q < spt / 4) reinterpret_cast<int4*>(s_tok + j0)[q] = t4[q];
+            } else {
+    #pragma unroll
+                for (uint32_t k = 0; k < 3; ++k)
+                    if (k < spt) s_tok[j0 + k] = t1[k];
+            }
+        }
+        // global pre-decay of the iteration's first token (Alg. 1 Pass 1)
+        life_store(s_life, j0, spt, own, decay4(lw0, 1), decay4(lw1, 1));
+        __syncthreads();
+        uint32_t fill_bound = 0;                              // hash index: non-empty buckets (upper bound)
+        if (!DIRECT) {
             build_index(ix, s_tok, j0, spt, own, s_fill, p.status);
             __syncthreads();
             fill_bound = *s_fill;
         }
-        publish_token(p, ti, table, g, n_take, blockIdx.x);
-    }
 
-    // ---- write the table back; speculative entries (id >= N) become empty (Alg. 4) ----
-    const int32_t N = p.verified_len_dev ? __ldg(p.verified_len_dev + ti) : p.verified_len[blockIdx.x];
-    if (own) {
-        if ((spt & 3u) == 0) {
-            for (uint32_t q = 0; q < spt / 4; ++q) {
-                int4 v = reinterpret_cast<const int4*>(s_tok + j0)[q];
-                v.x = v.x >= N ? -1 : v.x; v.y = v.y >= N ? -1 : v.y;
-                v.z = v.z >= N ? -1 : v.z; v.w = v.w >= N ? -1 : v.w;
-                reinterpret_cast<int4*>(g_tok + j0)[q] = v;
+        uint32_t list_off = 0, sum_valid = 0, sum_miss = 0, sum_decay = 0;
+        int2* list = p.miss_list + (size_t)ti * p.list_stride;
+
+
+        for (uint32_t g = 0; g < p.n_q; ++g) {
+            const size_t row = ((size_t)ti * p.n_q + g) * K;
+            int32_t* O = p.slots + row;
+            uint8_t* Hm = p.hit ? p.hit + row : nullptr;
+            if (tid < 128) s_hist[tid] = 0;
+
+            // ---- Probe, refresh hits to L, emit hit slots (Pass 1 + Pass 2) ----
+            uint32_t missmask = 0, nmiss = 0, nvalid = 0;
+            uint32_t cand[MAX_IPT];                             // direct index: candidate slot per id
+            check_ids(xs, i0, ipt, K, id_limit, p.status);      // out-of-range ids become padding (id_limit <= max_context)
+            if (DIRECT) {
+    #pragma unroll
+                for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {   // all loads are issued before any is used
+                    cand[k] = 0xFFFFFFFFu;
+                    if (k < ipt && i0 + k < K && xs[k] >= 0) cand[k] = __ldcg(where + xs[k]) & (S - 1u);
+                }
             }
-        } else {
-            for (uint32_t k = 0; k < spt; ++k) {
-                const int32_t v = s_tok[j0 + k];
-                g_tok[j0 + k] = v >= N ? -1 : v;
+    #pragma unroll
+            for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {
+                const uint32_t i = i0 + k;
+                if (k < ipt && i < K) {
+                    const int32_t x = xs[k];
+                    if (x >= 0 && (!DIRECT || cand[k] != 0xFFFFFFFFu)) {
+                        ++nvalid;
+                        int32_t j;
+                        if (DIRECT) j = s_tok[cand[k]] == x ? (int32_t)cand[k] : -1;
+                        else j = index_find(ix, x, p.status);
+                        if (j >= 0) {
+                            s_life[j] = (int8_t)L;
+                            O[i] = j;
+                            if (Hm) Hm[i] = 1;
+                        } else {
+                            missmask |= 1u << k;
+                            ++nmiss;
+                        }
+                    } else {
+                        O[i] = -1;
+                        if (Hm) Hm[i] = 0;
+                    }
+                }
             }
+            // order-preserving compaction of the misses: t = x[not m]
+            uint32_t total;
+            uint32_t off = block_excl_scan(nmiss | (nvalid << 16), s_scan_a, total) & 0xFFFFu;
+            const uint32_t n_g = total & 0xFFFFu;
+            sum_valid += total >> 16;
+            sum_miss += n_g;
+    #pragma unroll
+            for (uint32_t k = 0; k < (uint32_t)MAX_IPT; ++k) {
+                if (missmask & (1u << k)) {
+                    s_miss_x[off] = xs[k];
+                    s_miss_pos[off] = (uint16_t)(i0 + k);
+                    ++off;
+                }
+            }
+            // the next token's ids travel while this token's misses are placed
+            if (g + 1 < p.n_q) load_ids(p.indices + row + K, i0, ipt, K, xs);
+            if (tid == 0 && p.miss_count) p.miss_count[(size_t)ti * p.n_q + g] = (int32_t)n_g;
+            if (n_g == 0) { __syncthreads(); publish_token(p, ti, table, g, 0, bt); continue; }
+            __syncthreads();
+
+            // ---- Pass 3: CollectDead; if fewer than n_g slots are dead, decay until enough are ----
+            uint32_t w0, w1;
+            life_load(s_life, j0, spt, own, w0, w1);
+            uint32_t sg0 = w0 & 0x80808080u, sg1 = w1 & 0x80808080u;       // sign bits = dead slots
+            uint32_t dtotal, d = 0;
+            uint32_t doff = block_excl_scan(__popc(sg0) + __popc(sg1), s_scan_b, dtotal);
+            if (dtotal < n_g) {
+                // the while-loop of Alg. 1 in closed form: d = fewest unit decays after which n_g slots are dead,
+                // read off the histogram of the lifetimes (only needed on this, the rarer, path)
+                count_lifetimes(w0, w1, spt, own, L, s_priv, priv_stride, s_hist);
+                __syncthreads();
+                uint32_t cum = 0;
+                bool found = false;
+                d = (uint32_t)L + 1u;
+                for (uint32_t b = 0; b <= (uint32_t)L + 1u; ++b) {   // bin b counts lifetime b-1; dead after b decays
+                    cum += s_hist[b];
+                    if (cum >= n_g) { d = b; found = true; break; }
+                }
+                if (!found && tid == 0) atomicOr(p.status, ST_NO_DEAD_SLOTS);
+                w0 = decay4(w0, d);
+                w1 = decay4(w1, d);
+                life_store(s_life, j0, spt, own, w0, w1);
+                sg0 = w0 & 0x80808080u; sg1 = w1 & 0x80808080u;
+                doff = block_excl_scan(__popc(sg0) + __popc(sg1), s_scan_b, dtotal);
+            }
+            // dead slots in increasing order; the first n_g are handed out
+    #pragma unroll
+            for (uint32_t k = 0; k < (uint32_t)MAX_SPT; ++k) {
+                const uint32_t bit = k < 4 ? (sg0 >> (8 * k + 7)) & 1u : (sg1 >> (8 * (k - 4) + 7)) & 1u;
+                if (bit) {
+                    if (doff < n_g) s_dead[doff] = (uint16_t)(j0 + k);
+                    ++doff;
+                }
+            }
+            __syncthreads();
+
+            // ---- install the misses: k-th miss takes the k-th dead slot ----
+            const bool rebuild = !DIRECT && fill_bound + n_g > (H / 4u) * 3u;
+            const uint32_t n_take = n_g < dtotal ? n_g : dtotal;
+            for (uint32_t k = tid; k < n_take; k += nt) {
+                const uint32_t j = s_dead[k];
+                const int32_t x = s_miss_x[k];
+                const uint32_t i = s_miss_pos[k];
+                if (j < S && i < K) {
+                    s_tok[j] = x;
+                    s_life[j] = (int8_t)L;
+                    O[i] = (int32_t)j;
+                    if (Hm) Hm[i] = 0;
+                    list[list_off + k] = make_int2(x, (int32_t)j);
+                    if (DIRECT) __stcg(where + x, (uint16_t)j);
+                    else if (!rebuild) index_insert(ix, x, j, p.status);
+                } else {
+                    list[list_off + k] = make_int2(-1, -1);          // Stage Two skips it
+                    atomicOr(p.status, ST_BAD_SLOT);
+                }
+            }
+            list_off += n_take;
+            sum_decay += d;
+            if (!rebuild) {
+                fill_bound += n_g;
+                __syncthreads();
+            } else if constexpr (!DIRECT) {
+                __syncthreads();
+                for (uint32_t i = tid; i < H / 4; i += nt)
+                    reinterpret_cast<int4*>(s_key)[i] = make_int4(EMPTY, EMPTY, EMPTY, EMPTY);
+                if (tid == 0) *s_fill = 0;
+                __syncthreads();
+                build_index(ix, s_tok, j0, spt, own, s_fill, p.status);
+                __syncthreads();
+                fill_bound = *s_fill;
+            }
+            publish_token(p, ti, table, g, n_take, bt);
         }
-        uint32_t w0, w1;
-        life_load(s_life, j0, spt, own, w0, w1);
-        life_store(g_life, j0, spt, own, w0, w1);
-    }
-    if (tid == 0) {
-        SegDesc sd;
-        sd.src_base = p.kv_base[blockIdx.x];
-        sd.src_stride = p.kv_stride[blockIdx.x];
-        sd.dst_base = reinterpret_cast<uint64_t>(p.buffer + (size_t)table * S * p.row_bytes);
-        sd.count = list_off;
-        sd.pad = 0;
-        p.seg[ti] = sd;
-        TableStats* st = p.stats + table;
-        st->steps += 1;
-        st->tokens += p.n_q;
-        st->hits += sum_valid - sum_miss;
-        st->misses += sum_miss;
-        st->rows += list_off;
-        st->extra_decays += sum_decay;
+
+        // ---- write the table back; speculative entries (id >= N) become empty (Alg. 4) ----
+        const int32_t N = p.verified_len_dev ? __ldg(p.verified_len_dev + ti) : p.verified_len[bt];
+        if (own) {
+            if ((spt & 3u) == 0) {
+                for (uint32_t q = 0; q < spt / 4; ++q) {
+                    int4 v = reinterpret_cast<const int4*>(s_tok + j0)[q];
+                    v.x = v.x >= N ? -1 : v.x; v.y = v.y >= N ? -1 : v.y;
+                    v.z = v.z >= N ? -1 : v.z; v.w = v.w >= N ? -1 : v.w;
+                    reinterpret_cast<int4*>(g_tok + j0)[q] = v;
+                }
+            } else {
+                for (uint32_t k = 0; k < spt; ++k) {
+                    const int32_t v = s_tok[j0 + k];
+                    g_tok[j0 + k] = v >= N ? -1 : v;
+                }
+            }
+            uint32_t w0, w1;
+            life_load(s_life, j0, spt, own, w0, w1);
+            life_store(g_life, j0, spt, own, w0, w1);
+        }
+        if (tid == 0) {
+            SegDesc sd;
+            sd.src_base = p.kv_base[bt];
+            sd.src_stride = p.kv_stride[bt];
+            sd.dst_base = reinterpret_cast<uint64_t>(p.buffer + (size_t)table * S * p.row_bytes);
+            sd.count = list_off;
+            sd.pad = 0;
+            p.seg[ti] = sd;
+            TableStats* st = p.stats + table;
+            st->steps += 1;
+            st->tokens += p.n_q;
+            st->hits += sum_valid - sum_miss;
+            st->misses += sum_miss;
+            st->rows += list_off;
+            st->extra_decays += sum_decay;
+        }
+    };
+    if constexpr (ROUNDS) {
+        for (uint32_t bt = blockIdx.x; bt < p.n_launch; bt += gridDim.x) {
+            if (bt != blockIdx.x) __syncthreads();        // the previous table's last reads of shared memory are over
+            one_table(bt);
+        }
+    } else {
+        one_table(blockIdx.x);
     }
     if (p.t_range) {
         __syncthreads();
@@ -754,10 +769,14 @@ uint32_t stage_one_threads(uint32_t S, uint32_t K)
 cudaError_t stage_one_prepare(size_t max_smem)
 {
     const void* kernels[] = {
-        reinterpret_cast<const void*>(avsg_stage_one_kernel<false, S1_MAX_TABLES>),
-        reinterpret_cast<const void*>(avsg_stage_one_kernel<true, S1_MAX_TABLES>),
-        reinterpret_cast<const void*>(avsg_stage_one_kernel<false, S1_BIG_TABLES>),
-        reinterpret_cast<const void*>(avsg_stage_one_kernel<true, S1_BIG_TABLES>),
+        reinterpret_cast<const void*>(avsg_stage_one_kernel<false, S1_MAX_TABLES, false>),
+        reinterpret_cast<const void*>(avsg_stage_one_kernel<true, S1_MAX_TABLES, false>),
+        reinterpret_cast<const void*>(avsg_stage_one_kernel<false, S1_BIG_TABLES, false>),
+        reinterpret_cast<const void*>(avsg_stage_one_kernel<true, S1_BIG_TABLES, false>),
+        reinterpret_cast<const void*>(avsg_stage_one_kernel<false, S1_MAX_TABLES, true>),
+        reinterpret_cast<const void*>(avsg_stage_one_kernel<true, S1_MAX_TABLES, true>),
+        reinterpret_cast<const void*>(avsg_stage_one_kernel<false, S1_BIG_TABLES, true>),
+        reinterpret_cast<const void*>(avsg_stage_one_kernel<true, S1_BIG_TABLES, true>),
         reinterpret_cast<const void*>(avsg_stage_one_paper_kernel)};
     for (const void* k : kernels) {
         cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
@@ -781,8 +800,11 @@ cudaError_t launch_stage_one_t(const S1ParamsT<CAP>& p, uint32_t n_tables, cudaS
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return direct ? cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel<true, CAP>, p)
-                  : cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel<false, CAP>, p);
+    if (n_tables < p.n_launch)              // fewer blocks than tables: the blocks serve the tables in rounds
+        return direct ? cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel<true, CAP, true>, p)
+                      : cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel<false, CAP, true>, p);
+    return direct ? cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel<true, CAP, false>, p)
+                  : cudaLaunchKernelEx(&cfg, avsg_stage_one_kernel<false, CAP, false>, p);
 }
 }  // namespace
 

@@ -142,7 +142,7 @@ __device__ __forceinline__ void publish_token(const P& p, uint32_t ti, uint32_t 
     __syncthreads();
     if (tid == 0) {
         __threadfence();
-        atomicAdd(p.ready + g, 1ull);
+        atomicAdd(p.ready + (size_t)(ti / p.round_size) * p.n_q + g, 1ull);
         // calls with host buffers: the table that arrives last after the call's last token announces that every
         // table of the call has written its slot table, hit mask and miss counts.  The arrivals are counted in a
         // word of their own that wraps to zero by itself (atomicInc), whatever state the transfer kernel leaves

@@ -148,7 +148,8 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_kernel(const __grid_con
 __device__ __forceinline__ void retire_block(const XferOverlapParams& p)
 {
     if (atomicAdd(p.done, 1u) == gridDim.x - 1u) {
-        for (uint32_t k = 0; k < p.n_q; ++k) p.ready[k] = 0ull;
+        const uint32_t rounds = (p.n + p.round_size - 1u) / p.round_size;
+        for (uint32_t k = 0; k < rounds * p.n_q; ++k) p.ready[k] = 0ull;
         *p.done = 0u;
         __threadfence();
     }
@@ -156,13 +157,16 @@ __device__ __forceinline__ void retire_block(const XferOverlapParams& p)
 
 // Stage Two that overlaps Stage One (the latency-hiding direction of App. G).  The grid is launched with
 // programmatic stream serialization and does NOT wait for Stage One to complete: its blocks become resident
-// once every Stage One block has started, then wait - with a bound - until all tables of the call have
-// placed token g (Stage One raises ready[g] per table, after making that token's miss-list entries
-// visible), cut token g's misses evenly over the blocks (Eq. 6 per token) and copy them while Stage One
-// places token g+1.  Every Stage One block is resident before this grid starts, so it always makes progress
-// without this grid's help; if a wait still runs out the block sets ST_WAIT_TIMEOUT and stops copying.
-// Before leaving, every block waits for the completion of the Stage One grid, so that the completion of
-// this grid implies it.  All reads of data written by the running Stage One go to L2 (ld.cg / acquire).
+// once every Stage One block has started, then wait - with a bound - until all tables of a round have
+// placed token g (Stage One raises ready[round][g] per table, after making that token's miss-list entries
+// visible), cut that token's misses evenly over the blocks (Eq. 6 per round and token) and copy them while
+// Stage One places the next token or the next round of tables.  A call is one round unless it has so many
+// tables that Stage One, with a block per table, would take most of the SMs: then Stage One runs with
+// round_size blocks that serve the tables round by round, and this grid follows them.  Every Stage One block
+// is resident before this grid starts and never waits for it, so it always makes progress; if a wait still
+// runs out the block sets ST_WAIT_TIMEOUT and stops copying.  Before leaving, every block waits for the
+// completion of the Stage One grid, so that the completion of this grid implies it.  All reads of data written
+// by the running Stage One go to L2 (ld.cg / acquire).
 __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __grid_constant__ XferOverlapParams p)
 {
     __shared__ uint32_t s_pref[OVERLAP_MAX_TABLES + 1];
@@ -172,7 +176,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __
     __shared__ uint32_t s_ok;
 
     const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31u;
-    const uint32_t n = p.n;
+    const uint32_t n = p.n, rounds = (n + p.round_size - 1u) / p.round_size;
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (p.t_range && tid == 0) atomicMin(p.t_range, global_ns());
@@ -180,77 +184,82 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __
     __syncthreads();
 
     const uint32_t cpr = p.row_bytes >> 4;
-    bool first_row = p.t_range != nullptr, copied = false;
-    for (uint32_t g = 0; g < p.n_q; ++g) {
-        if (tid == 0) {
-            uint32_t ok = 0;
-            for (uint32_t spin = 0; spin < OVERLAP_SPIN_LIMIT; ++spin) {
-                unsigned long long v;
-                asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p.ready + g) : "memory");
-                if (v >= p.expect) { ok = 1; break; }
-                __nanosleep(64);
+    bool first_row = p.t_range != nullptr, copied = false, gave_up = false;
+    for (uint32_t r = 0; r < rounds && !gave_up; ++r) {
+        const uint32_t base = r * p.round_size;                        // tables [base, base + nr) of the call
+        const uint32_t nr = n - base < p.round_size ? n - base : p.round_size;
+        for (uint32_t g = 0; g < p.n_q; ++g) {
+            if (tid == 0) {
+                uint32_t ok = 0;
+                for (uint32_t spin = 0; spin < OVERLAP_SPIN_LIMIT; ++spin) {
+                    unsigned long long v;
+                    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p.ready + (size_t)r * p.n_q + g) : "memory");
+                    if (v >= nr + p.expect_extra) { ok = 1; break; }
+                    __nanosleep(64);
+                }
+                if (!ok) atomicOr(p.status, ST_WAIT_TIMEOUT);
+                s_ok = ok;
+                if (!ok) retire_block(p);
             }
-            if (!ok) atomicOr(p.status, ST_WAIT_TIMEOUT);
-            s_ok = ok;
-            if (!ok) retire_block(p);
-        }
-        __syncthreads();
-        if (!s_ok) break;                                          // same decision in every thread
-        if (g + 1 == p.n_q && tid == nt - 1) retire_block(p);      // beside the copy, not in front of it
-        if (g == 0)                                                // the bases are published with token 0
-            for (uint32_t i = tid; i < n; i += nt) {
-                s_src[i] = __ldcg(&p.seg[i].src_base);
-                s_stride[i] = __ldcg(&p.seg[i].src_stride);
-                s_dst[i] = __ldcg(&p.seg[i].dst_base);
-            }
+            __syncthreads();
+            if (!s_ok) { gave_up = true; break; }                      // same decision in every thread
+            if (r + 1 == rounds && g + 1 == p.n_q && tid == nt - 1) retire_block(p);    // beside the copy, not in front of it
+            if (g == 0)                                                // a table's bases are published with its token 0
+                for (uint32_t i = base + tid; i < base + nr; i += nt) {
+                    s_src[i] = __ldcg(&p.seg[i].src_base);
+                    s_stride[i] = __ldcg(&p.seg[i].src_stride);
+                    s_dst[i] = __ldcg(&p.seg[i].dst_base);
+                }
 
-        // prefix sum of token g's miss counts over the tables of the call (n <= OVERLAP_MAX_TABLES)
-        uint32_t running = 0;
-        for (uint32_t base = 0; base < n; base += nt) {
-            const uint32_t i = base + tid;
-            const uint32_t c = i < n ? __ldcg(p.tcount + (size_t)i * p.n_q + g) : 0u;
-            uint32_t total;
-            const uint32_t excl = block_excl_scan(c, s_w, total);
-            if (i < n) s_pref[i] = running + excl;
-            running += total;
+            // prefix sum of token g's miss counts over the tables of the round
+            uint32_t running = 0;
+            for (uint32_t b0 = 0; b0 < nr; b0 += nt) {
+                const uint32_t i = b0 + tid;
+                const uint32_t c = i < nr ? __ldcg(p.tcount + (size_t)(base + i) * p.n_q + g) : 0u;
+                uint32_t total;
+                const uint32_t excl = block_excl_scan(c, s_w, total);
+                if (i < nr) s_pref[i] = running + excl;
+                running += total;
+                __syncthreads();
+            }
+            if (tid == 0) s_pref[nr] = running;
+            __syncthreads();
+
+            const uint32_t C = gridDim.x, cb = blockIdx.x, q = running / C, rem = running % C;
+            const uint32_t m0 = cb * q + (cb < rem ? cb : rem);
+            const uint32_t m1 = m0 + q + (cb < rem ? 1u : 0u);
+            if (first_row && tid == 0 && m1 > m0) atomicMin(p.t_range + 2, global_ns());
+            copied = copied || m1 > m0;
+            for (uint32_t m = m0 + (tid >> 5); m < m1; m += nt >> 5) {
+                uint32_t lo = 0, hi = nr;                              // largest lo with s_pref[lo] <= m
+                while (hi - lo > 1) {
+                    const uint32_t mid = (lo + hi) >> 1;
+                    if (s_pref[mid] <= m) lo = mid; else hi = mid;
+                }
+                const uint32_t t = base + lo;                          // the table, within the call
+                const uint32_t local = s_off[t] + (m - s_pref[lo]);    // entry of the table's miss list
+                if (local >= p.list_stride) {
+                    if (lane == 0) atomicOr(p.status, ST_BAD_SEGMENT);
+                    continue;
+                }
+                const int2 e = __ldcg(p.miss_list + (size_t)t * p.list_stride + local);
+                if (e.x < 0) continue;
+                if (e.y < 0 || (uint32_t)e.y >= p.S) {
+                    if (lane == 0) atomicOr(p.status, ST_BAD_SLOT);
+                    continue;
+                }
+                const uint64_t src = s_src[t] + (uint64_t)(uint32_t)e.x * s_stride[t];
+                const uint64_t dst = s_dst[t] + (uint64_t)(uint32_t)e.y * p.row_bytes;
+                copy_row(src, dst, cpr, lane);
+                if (first_row) {
+                    if (tid == 0) atomicMin(p.t_range + 3, global_ns());
+                    first_row = false;
+                }
+            }
+            __syncthreads();
+            for (uint32_t i = tid; i < nr; i += nt) s_off[base + i] += s_pref[i + 1] - s_pref[i];
             __syncthreads();
         }
-        if (tid == 0) s_pref[n] = running;
-        __syncthreads();
-
-        const uint32_t C = gridDim.x, cb = blockIdx.x, q = running / C, r = running % C;
-        const uint32_t m0 = cb * q + (cb < r ? cb : r);
-        const uint32_t m1 = m0 + q + (cb < r ? 1u : 0u);
-        if (first_row && tid == 0 && m1 > m0) atomicMin(p.t_range + 2, global_ns());
-        copied = copied || m1 > m0;
-        for (uint32_t m = m0 + (tid >> 5); m < m1; m += nt >> 5) {
-            uint32_t lo = 0, hi = n;                               // largest lo with s_pref[lo] <= m
-            while (hi - lo > 1) {
-                const uint32_t mid = (lo + hi) >> 1;
-                if (s_pref[mid] <= m) lo = mid; else hi = mid;
-            }
-            const uint32_t local = s_off[lo] + (m - s_pref[lo]);   // entry of the table's miss list
-            if (local >= p.list_stride) {
-                if (lane == 0) atomicOr(p.status, ST_BAD_SEGMENT);
-                continue;
-            }
-            const int2 e = __ldcg(p.miss_list + (size_t)lo * p.list_stride + local);
-            if (e.x < 0) continue;
-            if (e.y < 0 || (uint32_t)e.y >= p.S) {
-                if (lane == 0) atomicOr(p.status, ST_BAD_SLOT);
-                continue;
-            }
-            const uint64_t src = s_src[lo] + (uint64_t)(uint32_t)e.x * s_stride[lo];
-            const uint64_t dst = s_dst[lo] + (uint64_t)(uint32_t)e.y * p.row_bytes;
-            copy_row(src, dst, cpr, lane);
-            if (first_row) {
-                if (tid == 0) atomicMin(p.t_range + 3, global_ns());
-                first_row = false;
-            }
-        }
-        __syncthreads();
-        for (uint32_t i = tid; i < n; i += nt) s_off[i] += s_pref[i + 1] - s_pref[i];
-        __syncthreads();
     }
     unsigned long long t_copied = 0;
     if (p.t_range) {

@@ -32,6 +32,7 @@ def test_bench_line(extra):
     assert d["clocks"]["sm_max_mhz"] >= d["clocks"]["sm_mhz"] > 0
     assert 0.5 < d["hit_rate"] < 1.0 and d["config"]["workload"].startswith("C3")
     assert r["peak_repeats"] == 4 and "numa_node" in d["numa"]
+    assert d["one_call_per_step"]["tables_per_call"] == 8 and d["one_call_per_step"]["gbs"] > 0
     t = d["target"]
     assert 8 * 2048 <= t["cold_step"]["rows"] <= 8 * 4096 and 0 < t["cold_step"]["frac"] < 1.2   # token 0 misses everything
     assert set(t["met"]) == {"cold_step", "steady_call_stage_two_events", "steady_call_stage_two_in_kernel"}

@@ -259,7 +259,9 @@ def test_overlap_mode_four_tokens_and_mode_switches(avsg):
 
 
 @pytest.mark.parametrize("n,n_q,K,S", [(74, 2, 64, 256),       # Stage One on half of a B200's SMs: still overlapped
-                                        (75, 2, 64, 256),       # one more table: runs as the balanced mode
+                                        (75, 2, 64, 256),       # one more table: Stage One serves the tables in rounds of 32
+                                        (100, 4, 32, 256),      # four rounds (the last of 4 tables) x four tokens
+                                        (600, 1, 16, 64),       # 19 rounds, the large argument block
                                         (128, 2, 64, 256),      # as many tables as the small argument block takes
                                         (5, 8, 96, 1024),       # as many tokens as the overlapped kernel takes
                                         (3, 9, 100, 1024),      # one more: runs as the balanced mode
