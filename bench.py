@@ -353,6 +353,7 @@ def run_cuda(args):
         slots_all = torch.empty_like(X_all[0])
         ctx.restore_state()
         torch.cuda.synchronize()
+        rows_before = ctx.stats()["rows_copied"]
         ev4 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
         for k in range(K):
             flush.fill_(k & 0xFF)
@@ -361,7 +362,7 @@ def run_cuda(args):
             ev4[k][1].record()
         torch.cuda.synchronize()
         one_ms = sum(a.elapsed_time(b) for a, b in ev4)
-        assert ctx.stats()["rows_copied"] - st1["rows_copied"] == rows_timed        # the same misses as the timed steps
+        assert ctx.stats()["rows_copied"] - rows_before == rows_timed               # the same misses as the timed steps
         del X_all, slots_all
 
     # ---- end to end: ids from pinned host memory, slot table back to pinned host memory ----
