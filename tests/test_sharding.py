@@ -63,6 +63,32 @@ def test_numa_helpers_against_a_fake_sysfs_tree(tmp_path):
         os.sched_setaffinity(0, before)
 
 
+def test_strong_scaling_splits_the_single_gpu_workload_by_request():
+    """bench.py --scaling strong: the ranks' tables partition the tables of the single-GPU run (same seed, same
+    per-table recipes), every rank keeps all layers of its requests, one call per layer."""
+    import importlib.util
+    import types
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    spec = importlib.util.spec_from_file_location("bench_module", os.path.join(root, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    args = types.SimpleNamespace(requests=6, layers=3, scaling="strong", buffer_slots=0, n_tokens=0)
+    single = bench._workload(0, 8, args, world=1)
+    assert single.num_tables == 18 and len(single.calls) == 3
+    world = 4
+    parts = [bench._workload(r, 8, args, world=world) for r in range(world)]
+    seen = []
+    for w in parts:
+        assert len(w.calls) == 3 and all(len(c) == len(w.calls[0]) for c in w.calls)       # every layer, same requests
+        assert sorted(t for c in w.calls for t in c) == list(range(w.num_tables))          # local ids, each table once
+        seen += [(t.seed, t.table) for t in w.tables]
+    assert sorted(seen) == sorted((t.seed, t.table) for t in single.tables)                # a partition of the job
+    assert [len(w.calls[0]) for w in parts] == [2, 2, 1, 1]                                # 6 requests over 4 ranks
+    weak = [bench._workload(r, 8, types.SimpleNamespace(requests=6, layers=3, scaling="weak", buffer_slots=0,
+                                                        n_tokens=0), world=world) for r in range(2)]
+    assert weak[0].num_tables == weak[1].num_tables == 18 and weak[0].tables[0].seed != weak[1].tables[0].seed
+
+
 def _free_port():
     s = socket.socket()
     s.bind(("127.0.0.1", 0))
