@@ -463,8 +463,9 @@ def run_cuda(args):
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms_j / K, "ms_per_step_without_l2_flush": tmax["warm_ms"] / K, "higher_is_better": True,
         "scaling": args.scaling if world > 1 else "weak", "vs_baseline": None,
-        "dtype": "int32/u8", "data": "synthetic", "config": dict(_config(w), host_row_stride=stride, stage_one_index=args.index, stage_two=args.stage_two,
-                                                       stage_one_cluster=args.cluster),
+        "dtype": "int32/u8", "data": "synthetic", "config": _config(w),
+        "variant": {"host_row_stride": stride, "stage_one_index": args.index, "stage_two": args.stage_two,
+                    "stage_one_cluster": args.cluster},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "GB/s",
                 "h2d_bytes_per_step": int(ids_bytes + rows_timed * rb / K), "d2h_bytes_per_step": int(ids_bytes + mc_bytes),

@@ -55,7 +55,11 @@ extern "C" {
 #define AVSG_STATUS_BAD_SEGMENT     0x08u /* Stage Two could not resolve a miss-list entry      */
 #define AVSG_STATUS_BAD_ID          0x10u /* an id >= kv_rows of its table, or >= max_context
                                              with the direct index (taken as padding)          */
-#define AVSG_STATUS_WAIT_TIMEOUT    0x20u /* overlapped Stage Two gave up waiting for Stage One */
+#define AVSG_STATUS_WAIT_TIMEOUT    0x20u /* overlapped Stage Two gave up waiting for Stage One:
+                                             rows of that call were not copied, and the counters
+                                             of the overlapped mode may be left raised - call
+                                             avsg_clear_status() before the context's next step,
+                                             whose results are undefined otherwise              */
 #define AVSG_STATUS_LAUNCH_FAILED   0x40u /* a Stage Two launch failed after Stage One had run:
                                              slots were reserved whose rows were never copied  */
 
