@@ -760,7 +760,7 @@ def test_paper_literal_mode_unsorted_ids(avsg):
 
 
 # ---- randomly drawn shapes: tables, S, K, tokens, L, row size, index and transfer mode -------------------------------
-@pytest.mark.parametrize("seed", range(12))
+@pytest.mark.parametrize("seed", range(24))
 def test_random_shapes(avsg, seed):
     rng = np.random.default_rng(1000 + seed)
     S = int(2 ** rng.integers(5, 14))                                  # 32 .. 8192
@@ -769,7 +769,7 @@ def test_random_shapes(avsg, seed):
     K = int(rng.integers(1, k_max + 1)) if rng.random() < 0.3 else int(min(k_max, 2 ** rng.integers(0, 12)))
     L = int(rng.choice([1, 2, 8, 16, 30, 31, 64]))
     rb = int(rng.choice([16, 48, 656, 1152]))
-    requests = int(rng.choice([1, 2, 5, 9]))
+    requests = int(rng.choice([1, 2, 5, 9])) if seed < 12 else int(rng.choice([3, 9, 40, 80, 100]))   # 80, 100: rounds
     ctxlen = int(max(2 * K * n_q, rng.integers(K * n_q + 8, 40 * K * n_q + 64)))
     base = rng.choice(["C2", "C4", "C5"])
     kw = dict(topk=K, buffer_slots=S, n_iters=int(rng.integers(3, 14)), max_lifetime=L, row_bytes=rb)
@@ -789,6 +789,17 @@ def test_random_shapes(avsg, seed):
     mode = getattr(avsg, str(rng.choice(["XFER_SM_BALANCED", "XFER_REQUEST_LEVEL", "XFER_POSITION_LEVEL",
                                          "XFER_SM_OVERLAP"])))
     index_mode = int(rng.choice([avsg.INDEX_HASH, avsg.INDEX_DIRECT]))
+    cluster = 0
+    if seed >= 12:                                                       # the later seeds also force cluster sizes
+        cluster = int(rng.choice([0, 0, 2, 4, 8]))
+        if cluster and w.buffer_slots // cluster < 32:
+            cluster = 0
+        if w.num_tables > 20:                                            # keep the big batches small per table
+            w = tr.workload("C5", requests=w.num_tables, ctx_lo=max(4, min(K, 64) // 2), ctx_hi=max(256, 8 * min(K, 64)),
+                            topk=min(K, 64), buffer_slots=max(64, min(S, 512)), n_iters=kw["n_iters"], max_lifetime=L,
+                            row_bytes=rb)
+            if cluster and w.buffer_slots // cluster < 32:
+                cluster = 0
     _parity(w, mode=mode, index_mode=index_mode, host_io=bool(rng.random() < 0.3),
             xfer_geometry=(int(rng.choice([1, 37, 148, 300])), int(rng.choice([32, 128, 256, 1024]))),
-            permute_seed=seed if seed % 2 else None)
+            permute_seed=seed if seed % 2 else None, cluster=cluster)
