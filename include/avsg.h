@@ -56,10 +56,9 @@ extern "C" {
 #define AVSG_STATUS_BAD_ID          0x10u /* an id >= kv_rows of its table, or >= max_context
                                              with the direct index (taken as padding)          */
 #define AVSG_STATUS_WAIT_TIMEOUT    0x20u /* overlapped Stage Two gave up waiting for Stage One:
-                                             rows of that call were not copied, and the counters
-                                             of the overlapped mode may be left raised - call
-                                             avsg_clear_status() before the context's next step,
-                                             whose results are undefined otherwise              */
+                                             rows of THAT call were not copied.  Later calls are
+                                             not affected (the hand-over flags carry the number
+                                             of their call)                                     */
 #define AVSG_STATUS_LAUNCH_FAILED   0x40u /* a Stage Two launch failed after Stage One had run:
                                              slots were reserved whose rows were never copied  */
 
@@ -244,9 +243,7 @@ int avsg_table_stats(avsg_ctx *ctx, uint32_t table_id, avsg_stats_t *out);
  * in *status_word when not NULL. */
 int avsg_sync_status(avsg_ctx *ctx, uint32_t *status_word);
 
-/* No passage of the paper: waits for the device, zeroes the status word and
- * the counters of the overlapped mode (which a call that reported AVSG_STATUS_WAIT_TIMEOUT may have
- * left raised). */
+/* No passage of the paper: waits for the device and zeroes the status word. */
 int avsg_clear_status(avsg_ctx *ctx);
 
 /* Diagnostic for AVSG_XFER_SM_OVERLAP: launches the overlapped transfer kernel

@@ -26,10 +26,11 @@ struct avsg_ctx {
     int8_t* d_life = nullptr;
     uint8_t* d_buffer = nullptr;
     TableStats* d_stats = nullptr;
-    unsigned long long* d_ready = nullptr;         // overlapped Stage Two: per-round, per-token counters [OVERLAP_MAX_COUNTERS],
-                                                   //   one word counting the transfer blocks that are through,
-                                                   //   one word with the sequence number of the last host-buffer call
-    uint32_t* d_tcount = nullptr;                  //   and per-(table of the call, token) miss counts
+    unsigned long long* d_flags = nullptr;         // overlapped Stage Two: per-(table of the call, token) flags
+                                                   //   (call number << 32 | miss count) [OVERLAP_MAX_TABLES x TOKENS]
+    unsigned long long* d_sync = nullptr;          //   [0] the call number, [1] transfer blocks that are through,
+                                                   //   [2] sequence number of the last host-buffer call,
+                                                   //   [3] arrivals after a host-buffer call's last token
     S1ParamsBig* big_args = nullptr;               // host: the large Stage One argument block, built in place per call
     unsigned long long* d_trange = nullptr;        // [8] time marks of the last timed call, then [8] their initial values
     unsigned long long* d_trange_init = nullptr;
@@ -88,7 +89,7 @@ uint32_t ilog2(uint32_t v) { uint32_t l = 0; while ((1u << l) < v) ++l; return l
 void free_all(avsg_ctx* c)
 {
     cudaFree(c->d_tok); cudaFree(c->d_life); cudaFree(c->d_buffer); cudaFree(c->d_stats); cudaFree(c->d_trange);
-    cudaFree(c->d_ready); cudaFree(c->d_tcount);
+    cudaFree(c->d_flags); cudaFree(c->d_sync);
     delete c->big_args;
     cudaFree(c->d_list); cudaFree(c->d_seg); cudaFree(c->d_status); cudaFree(c->d_where); cudaFree(c->d_q); cudaFree(c->d_q_snap);
     cudaFree(c->d_tok_snap); cudaFree(c->d_life_snap);
@@ -226,8 +227,7 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
     // direct kernels; the cluster and paper-literal kernels run Stage Two after Stage One instead).
     uint32_t round_size = n;
     if (mode == AVSG_XFER_SM_OVERLAP && (uint64_t)n * c->s1_cluster > (uint64_t)c->sm_count / 2) {
-        const uint32_t rounds = (n + S1_ROUND_BLOCKS - 1u) / S1_ROUND_BLOCKS;
-        if (c->s1_cluster == 1 && c->cfg.index_mode != AVSG_INDEX_PAPER && rounds * n_q <= (uint32_t)OVERLAP_MAX_COUNTERS)
+        if (c->s1_cluster == 1 && c->cfg.index_mode != AVSG_INDEX_PAPER)
             round_size = S1_ROUND_BLOCKS;
         else
             mode = AVSG_XFER_SM_BALANCED;
@@ -270,10 +270,10 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         p.verified_len_dev = a->verified_len_dev;
         // (every field is assigned: the large block is re-used from call to call)
         const bool overlap = mode == AVSG_XFER_SM_OVERLAP;
-        p.ready = overlap ? c->d_ready : nullptr;
-        p.tcount = overlap ? c->d_tcount : nullptr;
-        p.done_seq = wait_on_sequence ? c->d_ready + OVERLAP_MAX_COUNTERS + 1 : nullptr;
-        p.done_ctr = reinterpret_cast<uint32_t*>(c->d_ready + OVERLAP_MAX_COUNTERS + 2);
+        p.flags = overlap ? c->d_flags : nullptr;
+        p.epoch = reinterpret_cast<const uint32_t*>(c->d_sync);
+        p.done_seq = wait_on_sequence ? c->d_sync + 2 : nullptr;
+        p.done_ctr = reinterpret_cast<uint32_t*>(c->d_sync + 3);
         p.host_seq = wait_on_sequence ? c->host_seq + 1 : 0;
         p.expect = n;
         for (uint32_t i = 0; i < cnt; ++i) {
@@ -339,23 +339,23 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
     } else if (mode == AVSG_XFER_SM_OVERLAP) {
         XferOverlapParams x;
         x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
-        x.tcount = c->d_tcount; x.ready = c->d_ready;
-        x.done = reinterpret_cast<uint32_t*>(c->d_ready + OVERLAP_MAX_COUNTERS);
+        x.flags = c->d_flags; x.epoch = reinterpret_cast<uint32_t*>(c->d_sync);
+        x.done = reinterpret_cast<uint32_t*>(c->d_sync + 1);
         x.n = n; x.n_q = n_q; x.list_stride = c->list_stride; x.row_bytes = c->cfg.row_bytes; x.S = c->cfg.buffer_slots;
         x.round_size = round_size; x.expect_extra = 0;
         x.t_range = c->timing ? c->d_trange + 2 : nullptr;
         if (launch_transfer_overlap(x, c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count, c->xfer_threads, stream)
             != cudaSuccess) {
-            // Stage One has run and raised the per-token counters, nothing will lower them: do it here, in
-            // stream order, and remember that this call reserved slots whose rows were never copied
+            // Stage One has run and written flags with the current call number, which nothing will advance: wipe
+            // them here, in stream order, and remember that this call reserved slots whose rows were never copied
             cudaGetLastError();
-            cudaMemsetAsync(c->d_ready, 0, (OVERLAP_MAX_COUNTERS + 1) * sizeof(unsigned long long), stream);
+            cudaMemsetAsync(c->d_flags, 0, (size_t)OVERLAP_MAX_TABLES * OVERLAP_MAX_TOKENS * sizeof(unsigned long long), stream);
             c->host_status |= AVSG_STATUS_LAUNCH_FAILED;
             return AVSG_ECUDA;
         }
         if (wait_on_sequence) {
             c->host_seq += 1;
-            if (c->wait_value64(c->side, reinterpret_cast<CUdeviceptr>(c->d_ready + OVERLAP_MAX_COUNTERS + 1), c->host_seq,
+            if (c->wait_value64(c->side, reinterpret_cast<CUdeviceptr>(c->d_sync + 2), c->host_seq,
                                 CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
                 return AVSG_ECUDA;
             if ((rc = download_outputs()) != AVSG_OK) return rc;
@@ -465,8 +465,8 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     ok = ok && cudaMalloc(&c->d_buffer, T * S * cfg->row_bytes) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_stats, T * sizeof(TableStats)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->d_trange, 16 * sizeof(unsigned long long)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->d_ready, (OVERLAP_MAX_COUNTERS + 3) * sizeof(unsigned long long)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->d_tcount, (size_t)OVERLAP_MAX_TABLES * OVERLAP_MAX_TOKENS * sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_flags, (size_t)OVERLAP_MAX_TABLES * OVERLAP_MAX_TOKENS * sizeof(unsigned long long)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->d_sync, 8 * sizeof(unsigned long long)) == cudaSuccess;
     c->big_args = new (std::nothrow) S1ParamsBig();
     ok = ok && c->big_args != nullptr;
     ok = ok && cudaMalloc(&c->d_list, n_ids * sizeof(int2)) == cudaSuccess;
@@ -508,11 +508,13 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     {
         // [0] Stage One first start, [1] its last end; Stage Two: [2] first start, [3] last end, [4] first copy loop,
         // [5] first row in, [6] first block done; minima start at "never", maxima at 0
-        const unsigned long long never = ~0ull;
+        const unsigned long long never = ~0ull, first_epoch = 1;      // call numbers start at 1: a zeroed flag is never valid
         const unsigned long long init[16] = {never, 0, never, 0, never, never, never, 0, never, 0, never, 0, never, never, never, 0};
         c->d_trange_init = c->d_trange + 8;
         if (cudaMemcpy(c->d_trange, init, sizeof(init), cudaMemcpyHostToDevice) != cudaSuccess ||
-            cudaMemset(c->d_ready, 0, (OVERLAP_MAX_COUNTERS + 3) * sizeof(unsigned long long)) != cudaSuccess) {
+            cudaMemset(c->d_flags, 0, (size_t)OVERLAP_MAX_TABLES * OVERLAP_MAX_TOKENS * sizeof(unsigned long long)) != cudaSuccess ||
+            cudaMemset(c->d_sync, 0, 8 * sizeof(unsigned long long)) != cudaSuccess ||
+            cudaMemcpy(c->d_sync, &first_epoch, sizeof(first_epoch), cudaMemcpyHostToDevice) != cudaSuccess) {
             free_all(c); delete c; return AVSG_ECUDA;
         }
     }
@@ -657,8 +659,10 @@ int avsg_clear_status(avsg_ctx* c)
     CU(cudaDeviceSynchronize());
     CU(cudaMemset(c->d_status, 0, sizeof(uint32_t)));
     // a transfer kernel that gave up may have left the per-token counters of the overlapped mode raised
-    CU(cudaMemset(c->d_ready, 0, (OVERLAP_MAX_COUNTERS + 1) * sizeof(unsigned long long)));    // not the sequence word
-    CU(cudaMemset(c->d_ready + OVERLAP_MAX_COUNTERS + 2, 0, sizeof(unsigned long long)));      // arrivals after the last token
+    // (the flags of the overlapped mode carry their call's number and need no clearing; the two arrival counters
+    // wrap to zero by themselves unless a grid was lost half way)
+    CU(cudaMemset(c->d_sync + 1, 0, sizeof(unsigned long long)));
+    CU(cudaMemset(c->d_sync + 3, 0, sizeof(unsigned long long)));
     c->host_status = 0;
     return AVSG_OK;
 }
@@ -670,10 +674,10 @@ int avsg_probe_wait_limit(avsg_ctx* c, void* cuda_stream)
     if (!guard.ok) return AVSG_ECUDA;
     XferOverlapParams x;
     x.seg = c->d_seg; x.miss_list = c->d_list; x.status = c->d_status;
-    x.tcount = c->d_tcount; x.ready = c->d_ready;
-    x.done = reinterpret_cast<uint32_t*>(c->d_ready + OVERLAP_MAX_COUNTERS);
+    x.flags = c->d_flags; x.epoch = reinterpret_cast<uint32_t*>(c->d_sync);
+    x.done = reinterpret_cast<uint32_t*>(c->d_sync + 1);
     x.n = 1; x.n_q = 1; x.list_stride = c->list_stride; x.row_bytes = c->cfg.row_bytes; x.S = c->cfg.buffer_slots;
-    x.round_size = 1; x.expect_extra = 0;               // one table's token that no Stage One will place
+    x.round_size = 1; x.expect_extra = 0x40000000u;     // a call number no Stage One will ever write: the wait must run out
     CU(launch_transfer_overlap(x, c->xfer_blocks ? c->xfer_blocks : (uint32_t)c->sm_count, c->xfer_threads,
                                static_cast<cudaStream_t>(cuda_stream)));
     return AVSG_OK;

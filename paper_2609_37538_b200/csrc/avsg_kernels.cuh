@@ -98,11 +98,11 @@ struct S1ParamsT {
     uint32_t* qword;             // paper-literal mode: packed metadata words [num_tables][S], else null
     uint32_t probe_retries, hash_a1, hash_a2;   // paper-literal mode: R, a1, a2
     unsigned long long* t_range = nullptr;      // timing on: [0] earliest block start, [1] latest block end (ns)
-    // overlapped Stage Two (null otherwise): ready[r * n_q + g] counts the tables of round r of this call whose token
-    // g is placed (the transfer kernel zeroes it again); round r = tables [r * round_size, (r + 1) * round_size) of
-    // the call; tcount[ti * n_q + g] = misses of token g of the ti-th table of the call
-    unsigned long long* ready = nullptr;
-    uint32_t*           tcount = nullptr;
+    // overlapped Stage Two (null otherwise): flags[ti * n_q + g] = (epoch << 32) | misses of token g of the ti-th
+    // table of the call, written when that token is placed; *epoch is the number of the current overlapped call
+    // (the transfer grid advances it when it is through), so flags of earlier calls never look valid
+    unsigned long long* flags = nullptr;
+    const uint32_t*     epoch = nullptr;
     // calls with host buffers in that mode (null otherwise): the table that places the call's last token last
     // writes the call's sequence number to *done_seq, which the output download waits for
     unsigned long long* done_seq = nullptr;
@@ -131,7 +131,6 @@ struct XferParams {
 };
 
 constexpr int OVERLAP_MAX_TOKENS = 8;
-constexpr int OVERLAP_MAX_COUNTERS = 512;            // rounds x tokens of one call
 constexpr uint32_t S1_ROUND_BLOCKS = 32;             // Stage One blocks of a call that is served in rounds
 constexpr int OVERLAP_MAX_TABLES = S1_BIG_TABLES;   // one Stage One launch
 constexpr uint32_t OVERLAP_SPIN_LIMIT = 1u << 18;   // polls before the wait gives up; a poll is an L2 round trip plus a 64 ns sleep, ~0.8 us measured: ~0.2 s
@@ -140,9 +139,9 @@ struct XferOverlapParams {       // Stage Two that starts on token g's misses wh
     const SegDesc* seg;          // bases written by Stage One before it publishes token 0
     const int2*    miss_list;
     uint32_t*      status;
-    const uint32_t* tcount;      // [n][n_q]
-    unsigned long long* ready;   // [rounds][n_q] tables of the round that have placed token g; zero between calls
-    uint32_t*      done;         // blocks of this grid that are through; zero between calls
+    const unsigned long long* flags;   // [n][n_q] (epoch << 32) | miss count, written by Stage One per placed token
+    uint32_t*      epoch;        // number of the current overlapped call; advanced by the last block of this grid
+    uint32_t*      done;         // blocks of this grid that are through; wraps to zero by itself
     uint32_t n, n_q, list_stride, row_bytes, S;
     uint32_t round_size;         // tables per round (n: one round)
     uint32_t expect_extra;       // added to what a counter must reach: 0, or 1 for the wait-limit diagnostic

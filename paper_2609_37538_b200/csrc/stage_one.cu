@@ -143,6 +143,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (p.t_range && threadIdx.x == 0) atomicMin(p.t_range, global_ns());
+    const uint32_t epoch = p.flags ? __ldcg(p.epoch) : 0u;      // the number of this overlapped call
 
     // The grid usually has one block per table (ROUNDS = false: one pass, bt = blockIdx.x).  A call with many tables
     // and an overlapped Stage Two is launched with fewer blocks than tables (ROUNDS = true): a block then serves the
@@ -275,7 +276,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
             // the next token's ids travel while this token's misses are placed
             if (g + 1 < p.n_q) load_ids(p.indices + row + K, i0, ipt, K, xs);
             if (tid == 0 && p.miss_count) p.miss_count[(size_t)ti * p.n_q + g] = (int32_t)n_g;
-            if (n_g == 0) { __syncthreads(); publish_token(p, ti, table, g, 0, bt); continue; }
+            if (n_g == 0) { __syncthreads(); publish_token(p, ti, table, g, 0, bt, epoch); continue; }
             __syncthreads();
 
             // ---- Pass 3: CollectDead; if fewer than n_g slots are dead, decay until enough are ----
@@ -349,7 +350,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_kernel(const __grid_co
                 __syncthreads();
                 fill_bound = *s_fill;
             }
-            publish_token(p, ti, table, g, n_take, bt);
+            publish_token(p, ti, table, g, n_take, bt, epoch);
         }
 
         // ---- write the table back; speculative entries (id >= N) become empty (Alg. 4) ----
@@ -500,6 +501,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_paper_kernel(const __g
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (p.t_range && threadIdx.x == 0) atomicMin(p.t_range, global_ns());
+    const uint32_t epoch = p.flags ? __ldcg(p.epoch) : 0u;
 
     // ---- load the table; global pre-decay ----
     if (own)
@@ -577,7 +579,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_paper_kernel(const __g
         }
         if (g + 1 < p.n_q) load_ids(p.indices + row + K, i0, ipt, K, xs);
         if (tid == 0 && p.miss_count) p.miss_count[(size_t)ti * p.n_q + g] = (int32_t)n_g;
-        if (n_g == 0) { __syncthreads(); publish_token(p, ti, table, g, 0, blockIdx.x); continue; }
+        if (n_g == 0) { __syncthreads(); publish_token(p, ti, table, g, 0, blockIdx.x, epoch); continue; }
         __syncthreads();
 
         // ---- CollectDead / decay until n_g slots are dead ----
@@ -659,7 +661,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_paper_kernel(const __g
         list_off += n_take;
         sum_decay += d;
         __syncthreads();
-        publish_token(p, ti, table, g, n_take, blockIdx.x);
+        publish_token(p, ti, table, g, n_take, blockIdx.x, epoch);
     }
 
     // ---- write back; speculative entries (id >= N) become empty ----

@@ -222,6 +222,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_cluster_kernel(const _
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (p.t_range && tid == 0) atomicMin(p.t_range, global_ns());
+    const uint32_t epoch = p.flags ? __ldcg(p.epoch) : 0u;      // the number of this overlapped call
 
     // ---- issue every global load first: this block's part of the table state and of the first token's ids ----
     int4 t4[MAX_SPT / 4];
@@ -329,7 +330,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_cluster_kernel(const _
         sum_miss += n_g;
         if (rank == 0 && tid == 0 && p.miss_count) p.miss_count[(size_t)ti * p.n_q + g] = (int32_t)n_g;
         if (n_g == 0) {                                   // the same decision in every block of the cluster
-            if (rank == 0) publish_token(p, ti, table, g, 0, bt);
+            if (rank == 0) publish_token(p, ti, table, g, 0, bt, epoch);
             continue;
         }
 
@@ -414,7 +415,7 @@ __global__ void __launch_bounds__(1024, 1) avsg_stage_one_cluster_kernel(const _
         } else if constexpr (!DIRECT) {
             fill_bound = build();
         }
-        if (rank == 0) publish_token(p, ti, table, g, n_take, bt);
+        if (rank == 0) publish_token(p, ti, table, g, n_take, bt, epoch);
     }
 
     // ---- write this block's slots back; speculative entries (id >= N) become empty (Alg. 4) ----

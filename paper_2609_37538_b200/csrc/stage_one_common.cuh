@@ -117,18 +117,19 @@ __device__ __forceinline__ void count_lifetimes(uint32_t w0, uint32_t w1, uint32
     }
 }
 
-// Overlapped Stage Two only (p.ready set): tells the transfer kernel, which is already resident, that token g of
+// Overlapped Stage Two only (p.flags set): tells the transfer kernel, which is already resident, that token g of
 // this table is placed - `count` more entries of the table's miss list are final.  Called by every thread of the
 // block: the block meets after its list writes; one thread then fences (the barrier makes the fence cover the whole
-// block's earlier writes, as in a grid-wide barrier) and raises the counter of token g.
+// block's earlier writes, as in a grid-wide barrier) and writes the table's flag of token g: the call's number
+// (read once when the kernel starts) in the upper half, the count in the lower.
 template <typename P>
 __device__ __forceinline__ void publish_token(const P& p, uint32_t ti, uint32_t table, uint32_t g, uint32_t count,
-                                              uint32_t bt)      // bt: the table's index within this launch
+                                              uint32_t bt,      // bt: the table's index within this launch
+                                              uint32_t epoch)
 {
-    if (!p.ready) return;
+    if (!p.flags) return;
     const uint32_t tid = threadIdx.x;
     if (tid == 0) {
-        p.tcount[(size_t)ti * p.n_q + g] = count;
         if (g == 0) {
             SegDesc sd;
             sd.src_base = p.kv_base[bt];
@@ -142,7 +143,8 @@ __device__ __forceinline__ void publish_token(const P& p, uint32_t ti, uint32_t 
     __syncthreads();
     if (tid == 0) {
         __threadfence();
-        atomicAdd(p.ready + (size_t)(ti / p.round_size) * p.n_q + g, 1ull);
+        *reinterpret_cast<volatile unsigned long long*>(p.flags + (size_t)ti * p.n_q + g) =
+            ((unsigned long long)epoch << 32) | count;
         // calls with host buffers: the table that arrives last after the call's last token announces that every
         // table of the call has written its slot table, hit mask and miss counts.  The arrivals are counted in a
         // word of their own that wraps to zero by itself (atomicInc), whatever state the transfer kernel leaves

@@ -141,45 +141,38 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_kernel(const __grid_con
     }
 }
 
-// Called once per block after its last look at the per-token counters (or when it gave up).  The last block to
-// call it zeroes the counters for the next call - Stage One raised them for the last time before the last token's
-// wait could end - early and off the critical path.  The kernel arguments hold nothing that changes from call to
-// call, so a captured call can be replayed.
-__device__ __forceinline__ void retire_block(const XferOverlapParams& p)
-{
-    if (atomicAdd(p.done, 1u) == gridDim.x - 1u) {
-        const uint32_t rounds = (p.n + p.round_size - 1u) / p.round_size;
-        for (uint32_t k = 0; k < rounds * p.n_q; ++k) p.ready[k] = 0ull;
-        *p.done = 0u;
-        __threadfence();
-    }
-}
-
 // Stage Two that overlaps Stage One (the latency-hiding direction of App. G).  The grid is launched with
 // programmatic stream serialization and does NOT wait for Stage One to complete: its blocks become resident
 // once every Stage One block has started, then wait - with a bound - until all tables of a round have
-// placed token g (Stage One raises ready[round][g] per table, after making that token's miss-list entries
-// visible), cut that token's misses evenly over the blocks (Eq. 6 per round and token) and copy them while
+// placed token g (Stage One writes a flag per table and token, carrying the number of the call and the
+// token's miss count, after making that token's miss-list entries visible; every thread polls one table's
+// flag), cut that token's misses evenly over the blocks (Eq. 6 per round and token) and copy them while
 // Stage One places the next token or the next round of tables.  A call is one round unless it has so many
 // tables that Stage One, with a block per table, would take most of the SMs: then Stage One runs with
 // round_size blocks that serve the tables round by round, and this grid follows them.  Every Stage One block
 // is resident before this grid starts and never waits for it, so it always makes progress; if a wait still
 // runs out the block sets ST_WAIT_TIMEOUT and stops copying.  Before leaving, every block waits for the
-// completion of the Stage One grid, so that the completion of this grid implies it.  All reads of data written
-// by the running Stage One go to L2 (ld.cg / acquire).
+// completion of the Stage One grid, so that the completion of this grid implies it; the last block to leave
+// then advances the call number, so that no flag of this call can be taken for one of the next - nothing has
+// to be zeroed between calls, and the kernel arguments hold nothing that changes from call to call (a
+// captured call can be replayed).  All reads of data written by the running Stage One go to L2 (ld.cg /
+// acquire).
 __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __grid_constant__ XferOverlapParams p)
 {
     __shared__ uint32_t s_pref[OVERLAP_MAX_TABLES + 1];
     __shared__ uint32_t s_off[OVERLAP_MAX_TABLES];
     __shared__ uint64_t s_src[OVERLAP_MAX_TABLES], s_stride[OVERLAP_MAX_TABLES], s_dst[OVERLAP_MAX_TABLES];
     __shared__ uint32_t s_w[40];
-    __shared__ uint32_t s_ok;
 
     const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31u;
     const uint32_t n = p.n, rounds = (n + p.round_size - 1u) / p.round_size;
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (p.t_range && tid == 0) atomicMin(p.t_range, global_ns());
+    // the number of this call: the previous overlapped call's grid advanced it before this call's Stage One,
+    // which this grid was launched behind, could start
+    uint32_t epoch;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(epoch) : "l"(p.epoch) : "memory");
     for (uint32_t i = tid; i < n; i += nt) s_off[i] = 0;
     __syncthreads();
 
@@ -189,21 +182,21 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __
         const uint32_t base = r * p.round_size;                        // tables [base, base + nr) of the call
         const uint32_t nr = n - base < p.round_size ? n - base : p.round_size;
         for (uint32_t g = 0; g < p.n_q; ++g) {
-            if (tid == 0) {
-                uint32_t ok = 0;
-                for (uint32_t spin = 0; spin < OVERLAP_SPIN_LIMIT; ++spin) {
-                    unsigned long long v;
-                    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p.ready + (size_t)r * p.n_q + g) : "memory");
-                    if (v >= nr + p.expect_extra) { ok = 1; break; }
+            // every thread waits for the flag of one table of the round (of several, if the block is small)
+            int ok = 1;
+            for (uint32_t i = tid; i < nr; i += nt) {
+                const unsigned long long* f = p.flags + (size_t)(base + i) * p.n_q + g;
+                unsigned long long v = 0;
+                uint32_t spin = 0;
+                for (; spin < OVERLAP_SPIN_LIMIT; ++spin) {
+                    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(f) : "memory");
+                    if ((uint32_t)(v >> 32) == epoch + p.expect_extra) break;
                     __nanosleep(64);
                 }
-                if (!ok) atomicOr(p.status, ST_WAIT_TIMEOUT);
-                s_ok = ok;
-                if (!ok) retire_block(p);
+                if (spin == OVERLAP_SPIN_LIMIT) { ok = 0; atomicOr(p.status, ST_WAIT_TIMEOUT); break; }
+                s_pref[i] = (uint32_t)v;                               // the table's miss count of this token
             }
-            __syncthreads();
-            if (!s_ok) { gave_up = true; break; }                      // same decision in every thread
-            if (r + 1 == rounds && g + 1 == p.n_q && tid == nt - 1) retire_block(p);    // beside the copy, not in front of it
+            if (!__syncthreads_and(ok)) { gave_up = true; break; }     // same decision in every thread
             if (g == 0)                                                // a table's bases are published with its token 0
                 for (uint32_t i = base + tid; i < base + nr; i += nt) {
                     s_src[i] = __ldcg(&p.seg[i].src_base);
@@ -211,11 +204,11 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __
                     s_dst[i] = __ldcg(&p.seg[i].dst_base);
                 }
 
-            // prefix sum of token g's miss counts over the tables of the round
+            // prefix sum of token g's miss counts over the tables of the round (the counts came with the flags)
             uint32_t running = 0;
             for (uint32_t b0 = 0; b0 < nr; b0 += nt) {
                 const uint32_t i = b0 + tid;
-                const uint32_t c = i < nr ? __ldcg(p.tcount + (size_t)(base + i) * p.n_q + g) : 0u;
+                const uint32_t c = i < nr ? s_pref[i] : 0u;
                 uint32_t total;
                 const uint32_t excl = block_excl_scan(c, s_w, total);
                 if (i < nr) s_pref[i] = running + excl;
@@ -270,6 +263,13 @@ __global__ void __launch_bounds__(1024, 1) avsg_transfer_overlap_kernel(const __
     if (p.t_range && tid == 0) {
         atomicMax(p.t_range + 1, global_ns());                     // the block's end, the wait for Stage One included
         if (copied) atomicMin(p.t_range + 4, t_copied);
+    }
+    // Stage One is complete (the wait above), so no flag of this call will be written any more: the last block to
+    // arrive here advances the call number (0 is never used: the flags start out as zero)
+    __syncthreads();
+    if (tid == 0 && atomicInc(p.done, gridDim.x - 1u) == gridDim.x - 1u) {
+        const uint32_t next = epoch + 1u ? epoch + 1u : 1u;
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" :: "l"(p.epoch), "r"(next) : "memory");
     }
 }
 

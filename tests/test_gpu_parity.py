@@ -419,9 +419,16 @@ def test_overlap_wait_gives_up_and_the_context_stays_usable(avsg):
     assert time.time() - t0 < 10.0
     assert word == avsg.STATUS_WAIT_TIMEOUT, word
     assert (ctx.buffer(0).cpu().numpy() == before).all()
+    # the flags of the overlapped mode carry the number of their call, which the kernel that gave up advanced all
+    # the same: the next calls run correctly even BEFORE the status word is cleared (it stays set: it is sticky)
+    for t in range(4, 6):
+        step(t)
+    assert ctx.sync_status() == avsg.STATUS_WAIT_TIMEOUT
+    ctx.probe_wait_limit()                       # and a second lost Stage One changes nothing about that
+    assert ctx.sync_status() == avsg.STATUS_WAIT_TIMEOUT
     ctx.clear_status()
     assert ctx.sync_status() == 0
-    for t in range(4, 8):
+    for t in range(6, 8):
         step(t)
     assert ctx.sync_status() == 0
 
