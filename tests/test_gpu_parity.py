@@ -433,6 +433,57 @@ def test_overlap_wait_gives_up_and_the_context_stays_usable(avsg):
     assert ctx.sync_status() == 0
 
 
+@pytest.mark.parametrize("index,cluster", [("INDEX_HASH", 0), ("INDEX_DIRECT", 0), ("INDEX_DIRECT", 2)])
+def test_soak_random_subsets_modes_and_token_counts(avsg, index, cluster):
+    """300 calls on one context: every call takes a random subset of the tables in a random order, a random number
+    of tokens, a random Stage Two mode and either device or host buffers; every table is compared with its own
+    oracle after every call it took part in.  Exercises the hand-over flags of the overlapped mode across calls of
+    different shapes (a table's flag of an earlier call must never be taken for a current one)."""
+    import torch
+    rng = np.random.default_rng(77)
+    n, S, K, n_q_max, rb, ctxlen, L = 7, 512, 48, 4, 48, 4000, 5
+    kv = []
+    for i in range(n):
+        b = avsg.pinned_empty(ctxlen * rb)
+        tr.fill_kv(b.data_ptr(), 31, i, ctxlen, rb)
+        kv.append(b)
+    ctx = avsg.Context(n, S, rb, K, n_q_max, L, index_mode=getattr(avsg, index), max_context=ctxlen,
+                       stage_one_cluster=cluster)
+    orc = [OracleTable(S, rb, L) for _ in range(n)]
+    prev = [rng.choice(ctxlen, K, replace=False) for _ in range(n)]
+    modes = [avsg.XFER_SM_OVERLAP, avsg.XFER_SM_OVERLAP, avsg.XFER_SM_BALANCED, avsg.XFER_REQUEST_LEVEL,
+             avsg.XFER_POSITION_LEVEL]
+    for call in range(300):
+        tabs = [int(t) for t in rng.permutation(n)[: int(rng.integers(1, n + 1))]]
+        n_q = int(rng.integers(1, n_q_max + 1))
+        ctx.set_transfer_mode(int(rng.choice(modes)))
+        X = np.empty((len(tabs), n_q, K), np.int32)
+        for a, t in enumerate(tabs):
+            for g in range(n_q):                                     # ~85 % overlap with the table's last selection
+                keep = rng.choice(prev[t], int(0.85 * K), replace=False)
+                pool = np.setdiff1d(np.arange(ctxlen), keep)
+                sel = rng.permutation(np.concatenate([keep, rng.choice(pool, K - len(keep), replace=False)]))
+                X[a, g] = sel
+                prev[t] = sel
+        vlen = [ctxlen] * len(tabs)
+        if call % 3 == 2:
+            out = ctx.step_host(tabs, torch.from_numpy(X).pin_memory(), [kv[t] for t in tabs], vlen)
+        else:
+            out = ctx.step(tabs, torch.from_numpy(X).cuda(), [kv[t] for t in tabs], vlen)
+        torch.cuda.synchronize()
+        slots, hit, mc = out.slots.cpu().numpy(), out.hit.cpu().numpy(), out.miss_count.cpu().numpy()
+        for a, t in enumerate(tabs):
+            r = orc[t].step(X[a], ctxlen, kv[t].numpy(), rb)
+            assert (slots[a] == r.O).all() and (hit[a] == r.M).all() and (mc[a] == r.n).all(), (call, t)
+            if call % 10 == 9:
+                assert (ctx.buffer(t).cpu().numpy() == orc[t].rows()).all(), (call, t)
+    for t in range(n):
+        tok, life = ctx.export_state(t)
+        c, l = orc[t].export_state()
+        assert (tok == c).all() and (life == l).all() and (ctx.buffer(t).cpu().numpy() == orc[t].rows()).all(), t
+    assert ctx.sync_status() == 0
+
+
 # ---- behaviours ---------------------------------------------------------------------------------------------
 def test_regenerated_speculative_row_is_fetched_again(avsg):
     import torch
