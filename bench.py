@@ -245,7 +245,7 @@ def run_cuda(args):
     kv = []
     stride = args.row_stride or w.row_bytes
     for ti, cfg in enumerate(w.tables):
-        buf = avsg.pinned_empty(cfg.context * stride)
+        buf = avsg.pinned_empty(cfg.context * stride, huge_pages=args.host_kv == "huge")
         tr.fill_kv(buf.data_ptr(), w.seed, ti, cfg.context, w.row_bytes, row_stride=stride)
         kv.append(buf)
 
@@ -465,7 +465,7 @@ def run_cuda(args):
         "scaling": args.scaling if world > 1 else "weak", "vs_baseline": None,
         "dtype": "int32/u8", "data": "synthetic", "config": _config(w),
         "variant": {"host_row_stride": stride, "stage_one_index": args.index, "stage_two": args.stage_two,
-                    "stage_one_cluster": args.cluster},
+                    "stage_one_cluster": args.cluster, "host_kv": args.host_kv},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "GB/s",
                 "h2d_bytes_per_step": int(ids_bytes + rows_timed * rb / K), "d2h_bytes_per_step": int(ids_bytes + mc_bytes),
@@ -558,13 +558,13 @@ def run_cuda(args):
 # --suite: the five configurations, hit rates, per-call times and the Stage Two comparators (extra report;
 # the default run prints only the one line above)
 # ------------------------------------------------------------------------------------------------------------
-def _suite_one(avsg, torch, tr, name, mode, mode_name, link_peak, needed_rows=None, **kw):
+def _suite_one(avsg, torch, tr, name, mode, mode_name, link_peak, needed_rows=None, huge_pages=False, **kw):
     w = tr.workload(name, **kw)
     cores = os.cpu_count() or 1
     traces = _gen_traces(w, cores)
     kv = []
     for ti, cfg in enumerate(w.tables):
-        buf = avsg.pinned_empty(cfg.context * w.row_bytes)
+        buf = avsg.pinned_empty(cfg.context * w.row_bytes, huge_pages=huge_pages)
         tr.fill_kv(buf.data_ptr(), w.seed, ti, cfg.context, w.row_bytes)
         kv.append(buf)
     ctx = avsg.Context(num_tables=w.num_tables, buffer_slots=w.buffer_slots, row_bytes=w.row_bytes,
@@ -607,6 +607,11 @@ def _suite_one(avsg, torch, tr, name, mode, mode_name, link_peak, needed_rows=No
         "rows_per_iter_list": [r for _, _, r in per_iter],
     }
     ctx.close()
+    if huge_pages:
+        out["host_kv_pages"] = {"requested": "2 MiB transparent huge pages",
+                                "huge_fraction": sum(b.huge_bytes for b in kv) / max(1, sum(b.mapped_bytes for b in kv))}
+        for b in kv:
+            b.free()
     return out
 
 
@@ -720,6 +725,11 @@ def run_suite(args):
                 r2 = _suite_one(avsg, torch, tr, name, mode, mn, best, needed_rows=need, **kw)
                 r2.pop("rows_per_iter_list")
                 print(json.dumps(r2), flush=True)
+        if name == "C4":      # the widest spread of rows over host memory: the same run with the host KV in huge pages
+            r2 = _suite_one(avsg, torch, tr, name, M.XFER_SM_BALANCED, "sm_balanced, host KV from avsg_host_kv_alloc",
+                            best, huge_pages=True, **kw)
+            r2.pop("rows_per_iter_list")
+            print(json.dumps(r2), flush=True)
         if name == "C3":      # copy-engine comparator on a few iterations (one async copy per run of rows)
             kw2 = dict(kw, n_iters=6)
             r2 = _suite_one(avsg, torch, tr, name, M.XFER_COPY_ENGINE, "copy_engine", best, needed_rows=need[:6], **kw2)
@@ -1178,6 +1188,8 @@ def main():
     ap.add_argument("--numa-bind", default="auto", choices=["auto", "on", "off"],
                     help="bind the rank to the CPUs of its GPU's NUMA node before the host KV is allocated "
                          "(auto = when there are several ranks)")
+    ap.add_argument("--host-kv", default="pinned", choices=["pinned", "huge"],
+                    help="host KV from torch's pinned allocator (default) or from avsg_host_kv_alloc with huge pages")
     ap.add_argument("--tiny", action="store_true",
                     help="with --suite / --table3 / --sweeps: shrunk shapes that finish in seconds (what the tests run)")
     ap.add_argument("--no-comparators", action="store_true",

@@ -33,6 +33,7 @@
 #ifndef AVSG_H
 #define AVSG_H
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -344,6 +345,36 @@ typedef struct {
 } avsg_noalloc_args;
 
 int avsg_step_noalloc(const avsg_noalloc_args *args, void *cuda_stream);
+
+/*
+ * App. G (the host KV pool is an mmap of huge pages): page-locked,
+ * device-mapped HOST memory for a table's host KV, for callers that do not
+ * bring their own pool.  Any pinned, device-mapped memory serves as kv_base;
+ * this is one way to get it.
+ *
+ * The range is an anonymous private mapping aligned to 2 MiB, touched page by
+ * page by the CALLING thread (so it lands on that thread's NUMA node: bind the
+ * thread first) and registered with the CUDA runtime for the current device's
+ * context (portable, mapped).  With AVSG_HOST_KV_HUGE_PAGES the kernel is
+ * asked, before the first touch, to back it with transparent 2 MiB pages; the
+ * request is advisory, the memory is valid either way.  Contents start as
+ * zeros.
+ *   bytes        > 0; rounded up to 2 MiB internally
+ *   out          HOST: receives the base address (host pointer; usable as
+ *                kv_base as it is)
+ *   huge_bytes   HOST or NULL: receives how many bytes of the range the kernel
+ *                reports as backed by huge pages right after the touch
+ *                (0 when it cannot be read)
+ * AVSG_EINVAL for bad arguments, AVSG_ENOMEM when the mapping fails,
+ * AVSG_ECUDA when registration fails (the mapping is released again).
+ *
+ * avsg_host_kv_free: unregisters and unmaps a range avsg_host_kv_alloc
+ * returned; no call that reads it may be in flight.  AVSG_EINVAL for a pointer
+ * that did not come from avsg_host_kv_alloc (or was freed already).
+ */
+#define AVSG_HOST_KV_HUGE_PAGES 1u
+int avsg_host_kv_alloc(size_t bytes, uint32_t flags, void **out, uint64_t *huge_bytes);
+int avsg_host_kv_free(void *base);
 
 /* No passage of the paper: a static string naming an AVSG_E* code. */
 const char *avsg_strerror(int code);

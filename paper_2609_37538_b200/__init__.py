@@ -4,6 +4,6 @@ from .binding import (  # noqa: F401
     XFER_ALL_K, XFER_COPY_ENGINE, XFER_POSITION_LEVEL, XFER_REQUEST_LEVEL, XFER_SM_BALANCED, XFER_SM_OVERLAP,
     STATUS_BAD_ID, STATUS_BAD_SEGMENT, STATUS_BAD_SLOT, STATUS_NO_DEAD_SLOTS, STATUS_PROBE_EXHAUSTED, STATUS_WAIT_TIMEOUT,
     AvsgConfig, AvsgError, AvsgStats, AvsgStepArgs, Context, PreparedCall, StepOutput,
-    load_library, pinned_empty,
+    load_library, pinned_empty, HostKV, HOST_KV_HUGE_PAGES,
     AvsgNoAllocArgs, NOALLOC_MAX_IDS, NOALLOC_MAX_TABLES, step_noalloc,
 )

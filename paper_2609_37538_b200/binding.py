@@ -27,7 +27,7 @@ EXPORTS = (
     "avsg_sync_status", "avsg_export_state", "avsg_import_state", "avsg_save_state", "avsg_restore_state",
     "avsg_set_transfer_mode", "avsg_set_timing", "avsg_set_transfer_geometry", "avsg_strerror",
     "avsg_step_noalloc", "avsg_export_hash_state", "avsg_import_hash_state", "avsg_clear_status",
-    "avsg_probe_wait_limit",
+    "avsg_probe_wait_limit", "avsg_host_kv_alloc", "avsg_host_kv_free",
 )
 
 
@@ -112,6 +112,9 @@ def load_library():
     lib.avsg_step_noalloc.argtypes, lib.avsg_step_noalloc.restype = [ctypes.POINTER(AvsgNoAllocArgs), vp], i32
     lib.avsg_export_hash_state.argtypes, lib.avsg_export_hash_state.restype = [vp, u32, vp, vp], i32
     lib.avsg_import_hash_state.argtypes, lib.avsg_import_hash_state.restype = [vp, u32, vp, vp], i32
+    lib.avsg_host_kv_alloc.argtypes = [ctypes.c_size_t, u32, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_uint64)]
+    lib.avsg_host_kv_alloc.restype = i32
+    lib.avsg_host_kv_free.argtypes, lib.avsg_host_kv_free.restype = [vp], i32
     _lib = lib
     return lib
 
@@ -121,8 +124,43 @@ def _check(rc: int, what: str) -> None:
         raise AvsgError(rc, "%s: %s" % (what, load_library().avsg_strerror(rc).decode()))
 
 
-def pinned_empty(nbytes: int):
-    """Pinned (page-locked, device-mapped) host bytes for a table's host KV."""
+HOST_KV_HUGE_PAGES = 1
+
+
+class HostKV:
+    """A range from avsg_host_kv_alloc: pinned, device-mapped host bytes, zero-filled, touched by the calling thread."""
+
+    def __init__(self, nbytes: int, huge_pages: bool = True):
+        ptr, huge = ctypes.c_void_p(), ctypes.c_uint64()
+        _check(load_library().avsg_host_kv_alloc(int(nbytes), HOST_KV_HUGE_PAGES if huge_pages else 0,
+                                                 ctypes.byref(ptr), ctypes.byref(huge)), "avsg_host_kv_alloc")
+        self.ptr, self.nbytes, self.huge_bytes = int(ptr.value), int(nbytes), int(huge.value)
+        self.mapped_bytes = -(-int(nbytes) // (2 << 20)) * (2 << 20)           # what the library registered
+
+    def data_ptr(self) -> int:
+        return self.ptr
+
+    def numpy(self):
+        """The bytes as a numpy view (no copy); dead after free()."""
+        return np.ctypeslib.as_array((ctypes.c_uint8 * self.nbytes).from_address(self.ptr))
+
+    def free(self) -> None:
+        if self.ptr:
+            ptr, self.ptr = self.ptr, 0
+            _check(load_library().avsg_host_kv_free(ptr), "avsg_host_kv_free")
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def pinned_empty(nbytes: int, huge_pages: bool = False):
+    """Pinned (page-locked, device-mapped) host bytes for a table's host KV: a torch tensor, or with huge_pages a
+    HostKV range backed by transparent 2 MiB pages where the kernel grants them (App. G)."""
+    if huge_pages:
+        return HostKV(nbytes, True)
     import torch
     return torch.empty(int(nbytes), dtype=torch.uint8, pin_memory=True)
 

@@ -14,15 +14,16 @@ from oracle import OracleTable
 class HostKV:
     """Pinned host KV of a set of tables, filled by the seeded generator."""
 
-    def __init__(self, w: tr.Workload, tables: Sequence[int], row_stride: Optional[int] = None):
+    def __init__(self, w: tr.Workload, tables: Sequence[int], row_stride: Optional[int] = None,
+                 huge_pages: bool = False):
         import paper_2609_37538_b200 as avsg
         self.stride = w.row_bytes if row_stride is None else row_stride
         self.t, self.np = {}, {}
         for ti in tables:
             cfg = w.tables[ti]
-            buf = avsg.pinned_empty(cfg.context * self.stride)
+            buf = avsg.pinned_empty(cfg.context * self.stride, huge_pages=huge_pages)
             if self.stride != w.row_bytes:
-                buf.fill_(0xEE)
+                buf.numpy()[:] = 0xEE
             tr.fill_kv(buf.data_ptr(), w.seed, ti, cfg.context, w.row_bytes, row_stride=self.stride)
             self.t[ti] = buf
             self.np[ti] = buf.numpy()
@@ -31,7 +32,8 @@ class HostKV:
 def run_parity(w: tr.Workload, *, tables: Optional[Sequence[int]] = None, mode: int = 0, host_io: bool = False,
                row_stride: Optional[int] = None, buffer_every: int = 1, oracle_tables: Optional[Sequence[int]] = None,
                n_iters: Optional[int] = None, threads: Optional[int] = None, xfer_geometry=None,
-               index_mode: int = 0, permute_seed: Optional[int] = None, cluster: int = 0) -> Dict:
+               index_mode: int = 0, permute_seed: Optional[int] = None, cluster: int = 0,
+               huge_pages: bool = False) -> Dict:
     """Steps every call group of w for every iteration on the GPU; the tables in oracle_tables (default: all)
     are stepped by the oracle too and compared after EVERY step: hit mask, slot table, miss counts, (tok, life);
     the buffer rows every buffer_every iterations and at the end.  With permute_seed the K positions of every token
@@ -52,7 +54,7 @@ def run_parity(w: tr.Workload, *, tables: Optional[Sequence[int]] = None, mode: 
             rng = np.random.default_rng([permute_seed, ti])
             order = np.argsort(rng.random(X.shape), axis=-1)
             traces[ti] = (np.ascontiguousarray(np.take_along_axis(X, order, axis=-1)), N)
-    kv = HostKV(w, ids, row_stride)
+    kv = HostKV(w, ids, row_stride, huge_pages)
     T = w.n_iters if n_iters is None else min(n_iters, w.n_iters)
     local = {ti: k for k, ti in enumerate(ids)}                  # context table id of a workload table
     ctx = avsg.Context(num_tables=len(ids), buffer_slots=w.buffer_slots, row_bytes=w.row_bytes, max_topk=w.topk,

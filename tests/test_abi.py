@@ -64,6 +64,13 @@ def test_error_strings_and_argument_errors_need_no_gpu():
                  lambda: lib.avsg_save_state(None, None), lambda: lib.avsg_restore_state(None, None),
                  lambda: lib.avsg_reset(None, None, 0), lambda: lib.avsg_step_host(None, None, None)):
         assert call() == avsg.EINVAL
+    p = ctypes.c_void_p()
+    assert lib.avsg_host_kv_alloc(0, 0, ctypes.byref(p), None) == avsg.EINVAL          # no bytes
+    assert lib.avsg_host_kv_alloc(4096, 2, ctypes.byref(p), None) == avsg.EINVAL       # unknown flag
+    assert lib.avsg_host_kv_alloc(4096, 0, None, None) == avsg.EINVAL                  # nowhere to put the address
+    assert lib.avsg_host_kv_alloc(1 << 60, 0, ctypes.byref(p), None) == avsg.EINVAL    # beyond any address space
+    assert lib.avsg_host_kv_free(None) == avsg.EINVAL
+    assert lib.avsg_host_kv_free(ctypes.c_void_p(4096)) == avsg.EINVAL                 # not from the allocator
 
 
 def test_product_sources_do_not_touch_the_oracle():

@@ -10,7 +10,7 @@ pytestmark = pytest.mark.gpu
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-@pytest.mark.parametrize("extra", [[], ["--stage-two", "balanced", "--index", "hash"]])
+@pytest.mark.parametrize("extra", [[], ["--stage-two", "balanced", "--index", "hash", "--host-kv", "huge"]])
 def test_bench_line(extra):
     cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--requests", "4", "--layers", "2", "--steps", "4", "--warmup", "3",
            "--replays", "20", "--tiny"] + extra
@@ -59,6 +59,9 @@ def test_suite_report_tiny():
     assert by[("C5", "request_level")]["steady"]["rows_per_iter"] == by[("C5", "sm_balanced")]["steady"]["rows_per_iter"]
     assert by[("C5", "transfer_all_k")]["steady"]["rows_per_iter"] > by[("C5", "sm_balanced")]["steady"]["rows_per_iter"]
     assert ("C3", "copy_engine") in by
+    huge = by[("C4", "sm_balanced, host KV from avsg_host_kv_alloc")]
+    assert huge["steady"]["rows_per_iter"] == by[("C4", "sm_balanced")]["steady"]["rows_per_iter"]
+    assert 0 <= huge["host_kv_pages"]["huge_fraction"] <= 1
     modes = [r for r in rows if r["suite"] == "stage_two_modes"]
     assert len(modes) == 5 and all(set(m["us_per_iteration"]) == {"direct/balanced", "direct/overlap", "hash/balanced",
                                                                    "hash/overlap"} for m in modes)

@@ -111,6 +111,26 @@ def test_strided_host_rows_and_host_io(avsg):
     _parity(w, host_io=True)
 
 
+def test_host_kv_from_the_library_allocator(avsg):
+    """App. G: host KV in ranges from avsg_host_kv_alloc (2 MiB-aligned, huge pages requested, registered)."""
+    import ctypes
+    w = tr.workload("C4", topk=256, buffer_slots=1024, n_iters=10, context=1 << 15, requests=3, hot_size=64,
+                    hot_range=1024)
+    _parity(w, huge_pages=True)
+    _parity(w, huge_pages=True, row_stride=1024, mode=avsg.XFER_SM_OVERLAP)
+    kv = avsg.HostKV(5 << 20, huge_pages=True)
+    assert kv.ptr % (2 << 20) == 0 and 0 <= kv.huge_bytes <= 6 << 20
+    assert not kv.numpy().any()                                  # starts as zeros
+    plain = avsg.HostKV(4096, huge_pages=False)
+    assert plain.ptr % (2 << 20) == 0
+    lib = avsg.load_library()
+    ptr = kv.ptr
+    kv.free()
+    assert lib.avsg_host_kv_free(ptr) == avsg.EINVAL             # freed already
+    kv.free()                                                    # the wrapper's second free is a no-op
+    plain.free()
+
+
 def test_other_row_sizes(avsg):
     for rb in (16, 1152, 4096):
         _parity(tr.workload("C2", topk=128, buffer_slots=512, n_iters=10, context=8192, row_bytes=rb))
