@@ -154,6 +154,22 @@ typedef struct {
                                       AVSG_STATUS_BAD_ID.  Without it ids are not checked
                                       against the host allocation (the direct index still
                                       bounds them by max_context)                        */
+    uint64_t       *stage_one_done; /* DEVICE or NULL (latency hiding, App. G / Sec. 6): when
+                                      given, the library stores stage_one_done_value there
+                                      (8-byte aligned; device-scope release) as soon as
+                                      Stage One has finished every table of the call, i.e.
+                                      slots, hit and miss_count are final and the rows of
+                                      all HIT positions can be read, while Stage Two is
+                                      still copying the missed rows.  A consumer on another
+                                      stream waits for the value (a stream wait-value
+                                      operation, or a kernel that polls) and starts on the
+                                      hits; it still has to wait for the call's stream
+                                      before it reads a missed row.  avsg_step only:
+                                      avsg_step_host (which returns its outputs that early
+                                      by itself) and AVSG_XFER_ALL_K (no hits) refuse it
+                                      with AVSG_EINVAL                                   */
+    uint64_t        stage_one_done_value; /* what is stored; the caller chooses values that
+                                      let it tell calls apart (e.g. a running count)     */
 } avsg_step_args;
 
 typedef struct {

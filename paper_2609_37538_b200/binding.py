@@ -44,7 +44,8 @@ class AvsgStepArgs(ctypes.Structure):
                 ("topk", ctypes.c_uint32), ("indices", ctypes.c_void_p), ("kv_base", ctypes.c_void_p),
                 ("row_stride", ctypes.c_void_p), ("verified_len", ctypes.c_void_p), ("slots", ctypes.c_void_p),
                 ("hit", ctypes.c_void_p), ("miss_count", ctypes.c_void_p), ("verified_len_dev", ctypes.c_void_p),
-                ("kv_rows", ctypes.c_void_p)]
+                ("kv_rows", ctypes.c_void_p), ("stage_one_done", ctypes.c_void_p),
+                ("stage_one_done_value", ctypes.c_uint64)]
 
 
 class AvsgStats(ctypes.Structure):
@@ -225,11 +226,17 @@ class PreparedCall:
         self.args = a
 
     def run(self, indices, verified_len: Sequence[int], slots, hit=None, miss_count=None, stream=None,
-            host: bool = False) -> None:
+            host: bool = False, stage_one_done=None) -> None:
         """indices / slots / hit / miss_count: tensors (device, or pinned host when host=True) or addresses.
         verified_len: a sequence of n ints, or an int32 CUDA tensor [n] that the kernel reads when it runs
-        (what a call captured in a CUDA graph needs when the sequences grow between replays)."""
+        (what a call captured in a CUDA graph needs when the sequences grow between replays).
+        stage_one_done: None or (device int64 tensor or address, value): the word receives the value once the
+        slot table, hit mask and miss counts of the whole call are final, while the missed rows still travel."""
         a = self.args
+        if stage_one_done is not None:
+            a.stage_one_done, a.stage_one_done_value = _addr(stage_one_done[0]), int(stage_one_done[1])
+        else:
+            a.stage_one_done, a.stage_one_done_value = None, 0
         if hasattr(verified_len, "data_ptr"):
             a.verified_len_dev = verified_len.data_ptr()
         else:
@@ -274,7 +281,7 @@ class Context:
         return PreparedCall(self, table_ids, kv, n_tokens, topk, row_stride, kv_rows)
 
     def step(self, table_ids, indices, kv, verified_len, row_stride=None, want_hit: bool = True,
-             want_miss_count: bool = True, stream=None, kv_rows=None) -> StepOutput:
+             want_miss_count: bool = True, stream=None, kv_rows=None, stage_one_done=None) -> StepOutput:
         """One decode iteration. indices: int32 CUDA tensor [n, n_tokens, topk]. Returns device tensors."""
         import torch
         assert indices.is_cuda and indices.dtype == torch.int32 and indices.is_contiguous() and indices.dim() == 3
@@ -283,7 +290,7 @@ class Context:
         slots = torch.empty_like(indices)
         hit = torch.empty(indices.shape, dtype=torch.uint8, device=indices.device) if want_hit else None
         mc = torch.empty((n, n_q), dtype=torch.int32, device=indices.device) if want_miss_count else None
-        call.run(indices, verified_len, slots, hit, mc, stream)
+        call.run(indices, verified_len, slots, hit, mc, stream, stage_one_done=stage_one_done)
         return StepOutput(slots, hit, mc)
 
     def step_host(self, table_ids, indices, kv, verified_len, row_stride=None, want_hit: bool = True,

@@ -190,6 +190,9 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
 {
     int rc = check_args(c, a);
     if (rc != AVSG_OK) return rc;
+    if (a->stage_one_done && (host_io || c->cfg.transfer_mode == AVSG_XFER_ALL_K ||
+                              (reinterpret_cast<uint64_t>(a->stage_one_done) & 7u)))
+        return AVSG_EINVAL;
     DeviceGuard guard(c->cfg.device);
     if (!guard.ok) return AVSG_ECUDA;
 
@@ -272,9 +275,9 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         const bool overlap = mode == AVSG_XFER_SM_OVERLAP;
         p.flags = overlap ? c->d_flags : nullptr;
         p.epoch = reinterpret_cast<const uint32_t*>(c->d_sync);
-        p.done_seq = wait_on_sequence ? c->d_sync + 2 : nullptr;
+        p.done_seq = wait_on_sequence ? c->d_sync + 2 : reinterpret_cast<unsigned long long*>(a->stage_one_done);
         p.done_ctr = reinterpret_cast<uint32_t*>(c->d_sync + 3);
-        p.host_seq = wait_on_sequence ? c->host_seq + 1 : 0;
+        p.host_seq = wait_on_sequence ? c->host_seq + 1 : a->stage_one_done_value;
         p.expect = n;
         for (uint32_t i = 0; i < cnt; ++i) {
             p.table_id[i] = a->table_ids[first + i];

@@ -127,9 +127,10 @@ __device__ __forceinline__ void publish_token(const P& p, uint32_t ti, uint32_t 
                                               uint32_t bt,      // bt: the table's index within this launch
                                               uint32_t epoch)
 {
-    if (!p.flags) return;
+    const bool announce = p.done_seq && g + 1 == p.n_q;
+    if (!p.flags && !announce) return;
     const uint32_t tid = threadIdx.x;
-    if (tid == 0) {
+    if (tid == 0 && p.flags) {
         if (g == 0) {
             SegDesc sd;
             sd.src_base = p.kv_base[bt];
@@ -143,13 +144,14 @@ __device__ __forceinline__ void publish_token(const P& p, uint32_t ti, uint32_t 
     __syncthreads();
     if (tid == 0) {
         __threadfence();
-        *reinterpret_cast<volatile unsigned long long*>(p.flags + (size_t)ti * p.n_q + g) =
-            ((unsigned long long)epoch << 32) | count;
-        // calls with host buffers: the table that arrives last after the call's last token announces that every
-        // table of the call has written its slot table, hit mask and miss counts.  The arrivals are counted in a
-        // word of their own that wraps to zero by itself (atomicInc), whatever state the transfer kernel leaves
-        // the per-token counters in.
-        if (p.done_seq && g + 1 == p.n_q && atomicInc(p.done_ctr, p.expect - 1u) == p.expect - 1u) {
+        if (p.flags)
+            *reinterpret_cast<volatile unsigned long long*>(p.flags + (size_t)ti * p.n_q + g) =
+                ((unsigned long long)epoch << 32) | count;
+        // calls that asked for it (host buffers in the overlapped mode, or a caller's own signal word): the table
+        // that arrives last after the call's last token announces that every table of the call has written its
+        // slot table, hit mask and miss counts.  The arrivals are counted in a word of their own that wraps to
+        // zero by itself (atomicInc), whatever state the transfer kernel leaves the per-token counters in.
+        if (announce && atomicInc(p.done_ctr, p.expect - 1u) == p.expect - 1u) {
             __threadfence();
             *reinterpret_cast<volatile unsigned long long*>(p.done_seq) = p.host_seq;
         }

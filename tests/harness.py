@@ -33,7 +33,7 @@ def run_parity(w: tr.Workload, *, tables: Optional[Sequence[int]] = None, mode: 
                row_stride: Optional[int] = None, buffer_every: int = 1, oracle_tables: Optional[Sequence[int]] = None,
                n_iters: Optional[int] = None, threads: Optional[int] = None, xfer_geometry=None,
                index_mode: int = 0, permute_seed: Optional[int] = None, cluster: int = 0,
-               huge_pages: bool = False) -> Dict:
+               huge_pages: bool = False, signal: bool = False) -> Dict:
     """Steps every call group of w for every iteration on the GPU; the tables in oracle_tables (default: all)
     are stepped by the oracle too and compared after EVERY step: hit mask, slot table, miss counts, (tok, life);
     the buffer rows every buffer_every iterations and at the end.  With permute_seed the K positions of every token
@@ -75,6 +75,8 @@ def run_parity(w: tr.Workload, *, tables: Optional[Sequence[int]] = None, mode: 
             return orc[ti].step_all_k(X[t], kv.np[ti], kv.stride)
         return orc[ti].step(X[t], int(N[t]), kv.np[ti], kv.stride)
 
+    n_signalled = 0
+    signal_word = torch.zeros(1, dtype=torch.int64, device="cuda") if signal else None
     try:
         for t in range(T):
             for grp in calls:
@@ -89,8 +91,15 @@ def run_parity(w: tr.Workload, *, tables: Optional[Sequence[int]] = None, mode: 
                     torch.cuda.synchronize()
                     slots, hit, mc = out.slots.numpy(), out.hit.numpy(), out.miss_count.numpy()
                 else:
-                    out = ctx.step(tids, torch.from_numpy(Xh).cuda(), kvs, vlen, strides)
+                    if signal:                       # the call announces the end of its Stage One in a word of ours
+                        n_signalled += 1
+                        out = ctx.step(tids, torch.from_numpy(Xh).cuda(), kvs, vlen, strides,
+                                       stage_one_done=(signal_word, n_signalled))
+                    else:
+                        out = ctx.step(tids, torch.from_numpy(Xh).cuda(), kvs, vlen, strides)
                     torch.cuda.synchronize()
+                    if signal:
+                        assert int(signal_word.item()) == n_signalled, ("signal", w.name, t)
                     slots, hit, mc = out.slots.cpu().numpy(), out.hit.cpu().numpy(), out.miss_count.cpu().numpy()
                 for k, ti in enumerate(grp):
                     if ti not in check:

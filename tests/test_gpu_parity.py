@@ -298,14 +298,16 @@ def test_overlap_mode_limits(avsg, n, n_q, K, S):
     ctx = avsg.Context(n, S, rb, K, n_q, 16, transfer_mode=avsg.XFER_SM_OVERLAP, index_mode=avsg.INDEX_DIRECT,
                        max_context=ctxlen + n_q)
     orc = [OracleTable(S, rb, 16) for _ in range(n)]
+    word = torch.zeros(1, dtype=torch.int64, device="cuda")
     for t in range(T):
         X = np.stack([traces[i][0][t] for i in range(n)])
         N = [int(traces[i][1][t]) for i in range(n)]
         if t % 2:                                        # every other iteration through the host-buffer entry point
             out = ctx.step_host(list(range(n)), torch.from_numpy(X).pin_memory(), [kv] * n, N)
-        else:
-            out = ctx.step(list(range(n)), torch.from_numpy(X).cuda(), [kv] * n, N)
+        else:                                            # ... and these announce the end of their Stage One
+            out = ctx.step(list(range(n)), torch.from_numpy(X).cuda(), [kv] * n, N, stage_one_done=(word, 1000 + t))
         torch.cuda.synchronize()
+        assert int(word.item()) == 1000 + t - (t % 2), t
         slots, mc = out.slots.cpu().numpy(), out.miss_count.cpu().numpy()
         for i in range(n):
             r = orc[i].step(X[i], N[i], kv.numpy(), rb)
@@ -313,6 +315,82 @@ def test_overlap_mode_limits(avsg, n, n_q, K, S):
     for i in range(0, n, max(1, n // 7)):
         assert (ctx.buffer(i).cpu().numpy() == orc[i].rows()).all(), i
     assert ctx.sync_status() == 0
+
+
+def test_stage_one_done_signal(avsg):
+    """Latency hiding (App. G / Sec. 6): a call announces, in a device word of the caller, that its slot table, hit
+    mask and miss counts are final.  Every kind of Stage One kernel writes it, in both Stage Two modes; a second
+    stream that waits for the value reads the final outputs while nothing orders it after Stage Two."""
+    import torch
+    from cuda.bindings import driver as drv
+    w = tr.workload("C3", topk=256, buffer_slots=1024, n_iters=8, context=8192, requests=3, layers=1, recent_window=512)
+    for kw in (dict(), dict(mode=avsg.XFER_SM_OVERLAP), dict(index_mode=avsg.INDEX_DIRECT, mode=avsg.XFER_SM_OVERLAP),
+               dict(cluster=2), dict(cluster=4, mode=avsg.XFER_SM_OVERLAP),
+               dict(mode=avsg.XFER_REQUEST_LEVEL), dict(mode=avsg.XFER_POSITION_LEVEL)):
+        _parity(w, signal=True, **kw)
+
+    n, n_q, K, S, rb, ctxlen, T = 6, 2, 512, 2048, 656, 30000, 6
+    cfgs = [tr.TraceConfig(seed=41, table=i, topk=K, n_q=n_q, n_iters=T, context=ctxlen, ctx_growth=True,
+                           beta=(6, 2), p_recent=0.5, recent_window=2048) for i in range(n)]
+    traces = [tr.generate(c) for c in cfgs]
+    kv = []
+    for i in range(n):
+        b = avsg.pinned_empty(ctxlen * rb)
+        tr.fill_kv(b.data_ptr(), 41, i, ctxlen, rb)
+        kv.append(b)
+    side = torch.cuda.Stream()
+    word = torch.zeros(1, dtype=torch.int64, device="cuda")
+    ctx = avsg.Context(n, S, rb, K, n_q, 16, index_mode=avsg.INDEX_PAPER)       # the paper-literal kernel writes it too
+    for t in range(3):
+        X = torch.from_numpy(np.stack([traces[i][0][t] for i in range(n)])).cuda()
+        ctx.step(list(range(n)), X, kv, [int(traces[i][1][t]) for i in range(n)], stage_one_done=(word, 7 + t))
+        torch.cuda.synchronize()
+        assert int(word.item()) == 7 + t
+    assert ctx.sync_status() == 0
+    ctx.close()
+    for mode in (avsg.XFER_SM_BALANCED, avsg.XFER_SM_OVERLAP):
+        ctx = avsg.Context(n, S, rb, K, n_q, 16, transfer_mode=mode, index_mode=avsg.INDEX_DIRECT, max_context=ctxlen + n_q)
+        orc = [OracleTable(S, rb, 16) for _ in range(n)]
+        call = ctx.prepare(list(range(n)), kv, n_q, K)
+        early_slots = torch.empty((n, n_q, K), dtype=torch.int32, pin_memory=True)
+        early_hit = torch.empty((n, n_q, K), dtype=torch.uint8, pin_memory=True)
+        for t in range(T):
+            X = np.stack([traces[i][0][t] for i in range(n)])
+            N = [int(traces[i][1][t]) for i in range(n)]
+            Xd = torch.from_numpy(X).cuda()
+            slots = torch.empty_like(Xd)
+            hit = torch.empty(Xd.shape, dtype=torch.uint8, device="cuda")
+            torch.cuda.synchronize()
+            value = (mode + 1) * 100 + t
+            call.run(Xd, N, slots, hit, None, torch.cuda.current_stream(), stage_one_done=(word, value))
+            # the consumer: waits for the word, not for the call's stream
+            err, = drv.cuStreamWaitValue64(side.cuda_stream, word.data_ptr(), value,
+                                           drv.CUstreamWaitValue_flags.CU_STREAM_WAIT_VALUE_EQ)
+            assert err == drv.CUresult.CUDA_SUCCESS
+            with torch.cuda.stream(side):
+                early_slots.copy_(slots, non_blocking=True)
+                early_hit.copy_(hit, non_blocking=True)
+            side.synchronize()
+            torch.cuda.synchronize()
+            for i in range(n):
+                r = orc[i].step(X[i], N[i], kv[i].numpy(), rb)
+                assert (early_slots[i].numpy() == r.O).all() and (early_hit[i].numpy() == r.M).all(), (mode, t, i)
+        assert ctx.sync_status() == 0
+        # refusals: the host-buffer entry point, a misaligned word
+        Xh = torch.from_numpy(X).pin_memory()
+        sh = torch.empty(Xh.shape, dtype=torch.int32, pin_memory=True)
+        with pytest.raises(avsg.AvsgError) as e:
+            call.run(Xh, N, sh, None, None, None, host=True, stage_one_done=(word, 1))
+        assert e.value.code == avsg.EINVAL
+        with pytest.raises(avsg.AvsgError) as e:
+            call.run(Xd, N, slots, None, None, None, stage_one_done=(word.data_ptr() + 4, 1))
+        assert e.value.code == avsg.EINVAL
+        ctx.close()
+    ctx = avsg.Context(n, S, rb, K, n_q, 16, transfer_mode=avsg.XFER_ALL_K)
+    with pytest.raises(avsg.AvsgError) as e:
+        ctx.step(list(range(n)), Xd, kv, N, stage_one_done=(word, 1))
+    assert e.value.code == avsg.EINVAL
+    ctx.close()
 
 
 @pytest.mark.parametrize("cluster", [0, 2])
