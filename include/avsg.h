@@ -169,7 +169,11 @@ typedef struct {
                                       by itself) and AVSG_XFER_ALL_K (no hits) refuse it
                                       with AVSG_EINVAL                                   */
     uint64_t        stage_one_done_value; /* what is stored; the caller chooses values that
-                                      let it tell calls apart (e.g. a running count)     */
+                                      let it tell calls apart (e.g. a running count).  A
+                                      call captured in a CUDA graph stores the value it was
+                                      captured with on every replay: reset the word between
+                                      replays, or wait for it with a comparison that the
+                                      consumer re-arms                                   */
 } avsg_step_args;
 
 typedef struct {
