@@ -22,6 +22,8 @@
  *     of caller memory.  The context owns all state, the KV buffers and the
  *     scratch it needs; everything is allocated in avsg_create().
  *   - Calls on one context must not overlap in time (one stream at a time).
+ *     Different contexts share nothing: their calls may run on different
+ *     streams, or be issued by different host threads, at the same time.
  *   - Kernel-side problems (a bounded loop that ran out, a slot or segment
  *     index out of range, an id beyond kv_rows or the direct index) never
  *     fault: the kernel records a code in a status word that avsg_stats(),

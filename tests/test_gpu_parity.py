@@ -582,6 +582,51 @@ def test_soak_random_subsets_modes_and_token_counts(avsg, index, cluster):
     assert ctx.sync_status() == 0
 
 
+@pytest.mark.parametrize("n,mode_name", [(6, "XFER_SM_OVERLAP"), (90, "XFER_SM_OVERLAP"), (40, "XFER_SM_BALANCED")])
+def test_two_contexts_on_two_streams_at_once(avsg, n, mode_name):
+    """Two contexts, each on a stream of its own, issue their calls without waiting for one another: the kernels of
+    both share the GPU.  In the overlapped mode the waiting transfer grid of one context must never keep the other's
+    Stage One off the SMs (a transfer grid only starts once every block of its own Stage One has started; 90 tables
+    take the round-by-round path).  Both are compared with their oracles after every iteration."""
+    import torch
+    S, K, n_q, rb, ctxlen, T = 512, 64, 2, 656, 5000, 8
+    kv = avsg.pinned_empty(ctxlen * rb)
+    tr.fill_kv(kv.data_ptr(), 17, 0, ctxlen, rb)
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    ctxs, orcs, traces = [], [], []
+    for c in range(2):
+        ctxs.append(avsg.Context(n, S, rb, K, n_q, 16, transfer_mode=getattr(avsg, mode_name),
+                                 index_mode=avsg.INDEX_DIRECT if c == 0 else avsg.INDEX_HASH, max_context=ctxlen + n_q))
+        orcs.append([OracleTable(S, rb, 16) for _ in range(n)])
+        traces.append([tr.generate(tr.TraceConfig(seed=60 + c, table=i, topk=K, n_q=n_q, n_iters=T, context=ctxlen,
+                                                  ctx_growth=True, beta=(9, 1), p_recent=0.5, recent_window=512))
+                       for i in range(n)])
+    for t in range(T):
+        outs, Xs, Ns = [], [], []
+        for c in range(2):
+            X = np.stack([traces[c][i][0][t] for i in range(n)])
+            N = [int(traces[c][i][1][t]) for i in range(n)]
+            Xd = torch.from_numpy(X).cuda()
+            Xs.append(X); Ns.append(N)
+            outs.append((Xd, None))
+        torch.cuda.synchronize()
+        for c in range(2):                                # issued back to back, nothing waits in between
+            with torch.cuda.stream(streams[c]):
+                outs[c] = (outs[c][0], ctxs[c].step(list(range(n)), outs[c][0], [kv] * n, Ns[c], stream=streams[c]))
+        torch.cuda.synchronize()
+        for c in range(2):
+            out = outs[c][1]
+            slots, hit, mc = out.slots.cpu().numpy(), out.hit.cpu().numpy(), out.miss_count.cpu().numpy()
+            for i in range(n):
+                r = orcs[c][i].step(Xs[c][i], Ns[c][i], kv.numpy(), rb)
+                assert (slots[i] == r.O).all() and (hit[i] == r.M).all() and (mc[i] == r.n).all(), (t, c, i)
+    for c in range(2):
+        for i in range(0, n, max(1, n // 5)):
+            assert (ctxs[c].buffer(i).cpu().numpy() == orcs[c][i].rows()).all(), (c, i)
+        assert ctxs[c].sync_status() == 0
+        ctxs[c].close()
+
+
 # ---- behaviours ---------------------------------------------------------------------------------------------
 def test_regenerated_speculative_row_is_fetched_again(avsg):
     import torch
