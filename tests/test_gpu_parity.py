@@ -627,6 +627,45 @@ def test_two_contexts_on_two_streams_at_once(avsg, n, mode_name):
         ctxs[c].close()
 
 
+def test_two_host_threads_each_with_a_context(avsg):
+    """Two host threads, each driving a context and a stream of its own for the whole trace, nothing shared but the
+    library and the GPU: both stay bit-exact."""
+    import torch
+    from concurrent.futures import ThreadPoolExecutor
+    n, S, K, n_q, rb, ctxlen, T = 12, 512, 64, 2, 656, 5000, 10
+    kv = avsg.pinned_empty(ctxlen * rb)
+    tr.fill_kv(kv.data_ptr(), 18, 0, ctxlen, rb)
+
+    def drive(c):
+        torch.cuda.set_device(0)
+        stream = torch.cuda.Stream()
+        ctx = avsg.Context(n, S, rb, K, n_q, 16, transfer_mode=avsg.XFER_SM_OVERLAP,
+                           index_mode=avsg.INDEX_DIRECT if c else avsg.INDEX_HASH, max_context=ctxlen + n_q)
+        orc = [OracleTable(S, rb, 16) for _ in range(n)]
+        traces = [tr.generate(tr.TraceConfig(seed=70 + c, table=i, topk=K, n_q=n_q, n_iters=T, context=ctxlen,
+                                             ctx_growth=True, beta=(9, 1), p_recent=0.5, recent_window=512))
+                  for i in range(n)]
+        with torch.cuda.stream(stream):
+            for t in range(T):
+                X = np.stack([traces[i][0][t] for i in range(n)])
+                N = [int(traces[i][1][t]) for i in range(n)]
+                out = ctx.step(list(range(n)), torch.from_numpy(X).cuda(), [kv] * n, N, stream=stream)
+                stream.synchronize()
+                slots, mc = out.slots.cpu().numpy(), out.miss_count.cpu().numpy()
+                for i in range(n):
+                    r = orc[i].step(X[i], N[i], kv.numpy(), rb)
+                    assert (slots[i] == r.O).all() and (mc[i] == r.n).all(), (c, t, i)
+            stream.synchronize()
+            for i in range(0, n, 3):
+                assert (ctx.buffer(i).cpu().numpy() == orc[i].rows()).all(), (c, i)
+        assert ctx.sync_status() == 0
+        ctx.close()
+        return True
+
+    with ThreadPoolExecutor(max_workers=2) as ex:
+        assert all(ex.map(drive, range(2)))
+
+
 # ---- behaviours ---------------------------------------------------------------------------------------------
 def test_regenerated_speculative_row_is_fetched_again(avsg):
     import torch
