@@ -940,6 +940,33 @@ def run_breakdown(args):
                     for k in marks:
                         marks[k].append(st[k])
             ctx.close()
+            # pass 3: when are the hits usable?  A second stream waits for the word the call writes at the end of
+            # its Stage One (avsg_step_args.stage_one_done), not for the call's stream, and records an event
+            hits_at = []
+            try:
+                from cuda.bindings import driver as drv
+            except ImportError:
+                drv = None
+            if drv is not None:
+                ctx = avsg.Context(num_tables=w.num_tables, buffer_slots=w.buffer_slots, row_bytes=w.row_bytes,
+                                   max_topk=w.topk, max_tokens=w.n_q, max_lifetime=w.max_lifetime, transfer_mode=mode,
+                                   index_mode=avsg.INDEX_DIRECT, max_context=max(c.context for c in w.tables) + w.n_q)
+                call = ctx.prepare(grp, [kv[t] for t in grp], w.n_q, w.topk)
+                side = torch.cuda.Stream()
+                word = torch.zeros(1, dtype=torch.int64, device="cuda")
+                for t in range(w.n_iters):
+                    flush.fill_(t & 0xFF)
+                    torch.cuda.synchronize()
+                    e0, es = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    err, = drv.cuStreamWaitValue64(side.cuda_stream, word.data_ptr(), t + 1,
+                                                   drv.CUstreamWaitValue_flags.CU_STREAM_WAIT_VALUE_EQ)
+                    assert err == drv.CUresult.CUDA_SUCCESS
+                    es.record(side)
+                    e0.record(); call.run(X[t], V[t], slots, None, None, stream, stage_one_done=(word, t + 1))
+                    torch.cuda.synchronize()
+                    if t >= w.n_iters // 4:
+                        hits_at.append(e0.elapsed_time(es) * 1e3)
+                ctx.close()
             mean = lambda v: sum(v) / max(1, len(v))
             rows = mean(rows_per)
             ev, copy_start, first_row = mean(untimed), mean(marks["last_copy_start_us"]), mean(marks["last_first_row_us"])
@@ -951,7 +978,8 @@ def run_breakdown(args):
                 "split_us": {"launch_and_event_gap": ev - call_k, "stage_one_exposed": copy_start,
                              "first_row": first_row - copy_start, "copy": first_done - first_row,
                              "tail": call_k - first_done},
-                "stage_one_kernel_us": mean(marks["last_stage_one_kernel_us"]), "call_kernel_us": call_k}), flush=True)
+                "stage_one_kernel_us": mean(marks["last_stage_one_kernel_us"]), "call_kernel_us": call_k,
+                "hits_usable_us": mean(hits_at) if hits_at else None}), flush=True)
         del kv
 
 

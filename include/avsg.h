@@ -163,10 +163,16 @@ typedef struct {
                                       slots, hit and miss_count are final and the rows of
                                       all HIT positions can be read, while Stage Two is
                                       still copying the missed rows.  A consumer on another
-                                      stream waits for the value (a stream wait-value
-                                      operation, or a kernel that polls) and starts on the
-                                      hits; it still has to wait for the call's stream
-                                      before it reads a missed row.  avsg_step only:
+                                      stream waits for the value with a stream wait-value
+                                      operation and starts on the hits; it still has to
+                                      wait for the call's stream before it reads a missed
+                                      row.  Quicker: a consumer kernel launched right behind
+                                      avsg_step on the SAME stream with programmatic stream
+                                      serialization (the operator's kernels release their
+                                      dependents as soon as they run, and all their blocks
+                                      are resident by then): it polls the word, works on
+                                      the hits, and executes griddepcontrol.wait before it
+                                      touches a missed row.  avsg_step only:
                                       avsg_step_host (which returns its outputs that early
                                       by itself) and AVSG_XFER_ALL_K (no hits) refuse it
                                       with AVSG_EINVAL                                   */

@@ -1,5 +1,6 @@
 """Bit-exact parity of the CUDA path (through the C ABI) with the CPU oracle, on a B200."""
 import ctypes
+import os
 
 import numpy as np
 import pytest
@@ -8,6 +9,7 @@ import avsg_traces as tr
 from oracle import OracleTable
 
 pytestmark = pytest.mark.gpu
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 @pytest.fixture(scope="module")
@@ -390,6 +392,91 @@ def test_stage_one_done_signal(avsg):
     with pytest.raises(avsg.AvsgError) as e:
         ctx.step(list(range(n)), Xd, kv, N, stage_one_done=(word, 1))
     assert e.value.code == avsg.EINVAL
+    ctx.close()
+
+
+@pytest.fixture(scope="module")
+def early_consumer(tmp_path_factory):
+    """tests/cuda/early_consumer.cu built into a shared object: a stand-in for an attention kernel."""
+    import ctypes
+    import subprocess
+    from paper_2609_37538_b200 import build as pkg_build
+    so = tmp_path_factory.mktemp("consumer") / "early_consumer.so"
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    flags = [f for f in pkg_build.NVCC_FLAGS if f != "--use_fast_math"]
+    subprocess.check_call([nvcc] + flags + ["-o", str(so), os.path.join(ROOT, "tests", "cuda", "early_consumer.cu")])
+    lib = ctypes.CDLL(str(so))
+    vp, u32, u64 = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64
+    lib.launch_early_consumer.argtypes = [vp, u64, vp, vp, vp, u32, u32, vp, u32, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.launch_early_consumer.restype = ctypes.c_int
+    return lib
+
+
+@pytest.mark.parametrize("mode_name", ["XFER_SM_OVERLAP", "XFER_SM_BALANCED"])
+def test_a_kernel_on_the_same_stream_starts_on_the_hits(avsg, early_consumer, mode_name):
+    """Latency hiding (Sec. 6): a consumer kernel launched right behind avsg_step on the same stream, with
+    programmatic stream serialization, runs while Stage Two still copies.  It waits for the call's stage_one_done
+    word, then holds the final slot table and hit mask and reads a HIT row; only then does it wait for the stream's
+    earlier work (griddepcontrol.wait) and read a MISSED row.  All four are compared with the oracle / the host KV,
+    and the hits were usable before the misses had arrived."""
+    import torch
+    n, n_q, K, S, rb, ctxlen, T = 16, 2, 2048, 8192, 656, 60000, 6
+    cfgs = [tr.TraceConfig(seed=51, table=i, topk=K, n_q=n_q, n_iters=T, context=ctxlen, ctx_growth=True,
+                           beta=(18, 2), p_recent=0.5, recent_window=4096) for i in range(n)]
+    traces = [tr.generate(c) for c in cfgs]
+    kv = []
+    for i in range(n):
+        b = avsg.pinned_empty(ctxlen * rb)
+        tr.fill_kv(b.data_ptr(), 51, i, ctxlen, rb)
+        kv.append(b)
+    ctx = avsg.Context(n, S, rb, K, n_q, 16, transfer_mode=getattr(avsg, mode_name), index_mode=avsg.INDEX_DIRECT,
+                       max_context=ctxlen + n_q)
+    orc = [OracleTable(S, rb, 16) for _ in range(n)]
+    call = ctx.prepare(list(range(n)), kv, n_q, K)
+    dev = dict(device="cuda")
+    word = torch.zeros(1, dtype=torch.int64, **dev)
+    slots = torch.empty((n, n_q, K), dtype=torch.int32, **dev)
+    hit = torch.empty((n, n_q, K), dtype=torch.uint8, **dev)
+    slots_early, hit_early = torch.empty_like(slots), torch.empty_like(hit)
+    hit_row, miss_row = torch.zeros(rb, dtype=torch.uint8, **dev), torch.zeros(rb, dtype=torch.uint8, **dev)
+    picked = torch.empty(2, dtype=torch.int32, **dev)
+    marks = torch.zeros(4, dtype=torch.int64, **dev)
+    status = torch.zeros(1, dtype=torch.int32, **dev)
+    stream = torch.cuda.current_stream()
+    buf0 = ctx.buffer(0)
+    lead = []
+    for t in range(T):
+        X = np.stack([traces[i][0][t] for i in range(n)])
+        N = [int(traces[i][1][t]) for i in range(n)]
+        Xd = torch.from_numpy(X).cuda()
+        slots_early.fill_(-7); hit_early.fill_(9)
+        torch.cuda.synchronize()
+        call.run(Xd, N, slots, hit, None, stream, stage_one_done=(word, t + 1))
+        rc = early_consumer.launch_early_consumer(word.data_ptr(), t + 1, Xd.data_ptr(), slots.data_ptr(), hit.data_ptr(),
+                                                  n * n_q * K, n_q * K, buf0.data_ptr(), rb, slots_early.data_ptr(),
+                                                  hit_early.data_ptr(), hit_row.data_ptr(), miss_row.data_ptr(),
+                                                  picked.data_ptr(), marks.data_ptr(), status.data_ptr(),
+                                                  stream.cuda_stream or None)
+        assert rc == 0
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0                              # the consumer's wait did not run out
+        for i in range(n):
+            r = orc[i].step(X[i], N[i], kv[i].numpy(), rb)
+            assert (slots_early[i].cpu().numpy() == r.O).all() and (hit_early[i].cpu().numpy() == r.M).all(), (t, i)
+        hit_id, miss_id = (int(v) for v in picked.cpu())
+        host0 = kv[0].numpy().reshape(ctxlen, rb)
+        if t > 0:
+            assert hit_id >= 0
+        if hit_id >= 0:
+            assert (hit_row.cpu().numpy() == host0[hit_id]).all(), t         # read BEFORE Stage Two was waited for
+        assert miss_id >= 0 and (miss_row.cpu().numpy() == host0[miss_id]).all(), t
+        t0, t1, t2, t3 = (int(v) for v in marks.cpu())
+        assert t0 <= t1 <= t2 <= t3
+        lead.append((t3 - t2) / 1e3)
+    # steady calls move ~2000 rows (tens of microseconds): the consumer had finished with the hits and still had to
+    # wait for the missed rows, i.e. its first phase ran while Stage Two was copying
+    assert max(lead[1:]) > 5.0, lead
+    assert ctx.sync_status() == 0
     ctx.close()
 
 
