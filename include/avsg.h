@@ -160,9 +160,14 @@ typedef struct {
                                       given, the library stores stage_one_done_value there
                                       (8-byte aligned; device-scope release) as soon as
                                       Stage One has finished every table of the call, i.e.
-                                      slots, hit and miss_count are final and the rows of
-                                      all HIT positions can be read, while Stage Two is
-                                      still copying the missed rows.  A consumer on another
+                                      slots, hit and miss_count are final and every row
+                                      that was resident BEFORE the call can be read, while
+                                      Stage Two is still copying the missed rows.  Those are
+                                      all hits of the first token; a hit of a later token
+                                      may be on a slot that an earlier token of the same
+                                      call has just reserved (Sec. 3.6) - that slot is also
+                                      the slot of a missed position of an earlier token of
+                                      the table - and its row is still on its way.  A consumer on another
                                       stream waits for the value with a stream wait-value
                                       operation and starts on the hits; it still has to
                                       wait for the call's stream before it reads a missed

@@ -7,7 +7,8 @@
 // and Stage Two are still at work - and only then: every block of both is resident by the time it begins, so its
 // wait below is for kernels that are running, never for one that has yet to be scheduled.
 //   phase 1  wait (bounded) for the word the call writes at the end of its Stage One (avsg_step_args.stage_one_done);
-//            the slot table and the hit mask are final: copy them out, and read the row of one HIT position
+//            the slot table and the hit mask are final: copy them out, and read the row of one position of the FIRST
+//            token that hit (a hit of a later token may be on a slot reserved earlier in this very call, Sec. 3.6)
 //   phase 2  griddepcontrol.wait: everything before it on the stream, i.e. Stage Two, is complete and visible;
 //            read the row of one MISSED position
 // 32 blocks; every block waits for the word by itself, the first one also reads the rows and takes the time marks
@@ -39,6 +40,9 @@ struct ConsumerArgs {
     const uint8_t* hit;          // [n_pos] written by the call
     uint32_t n_pos;              // positions of the whole call
     uint32_t n_pos_table0;       // positions of table 0 (rows are read from table 0's buffer only)
+    uint32_t topk;               // positions of table 0's FIRST token: only there is every hit a row that was resident
+                                 // before the call (a later token may hit a slot an earlier token of this call has
+                                 // just reserved, whose row is still on its way)
     const uint8_t* buffer0;      // table 0's rows
     uint32_t row_bytes;
     int32_t* slots_early;        // [n_pos] out
@@ -73,9 +77,10 @@ __global__ void __launch_bounds__(256) early_consumer_kernel(ConsumerArgs a)
             a.hit_early[i] = __ldcg(a.hit + i);
         }
         if (first) {
-            for (uint32_t i = tid; i < a.n_pos_table0; i += blockDim.x) {       // first hit and first miss of table 0
-                if (__ldcg(a.slots + i) < 0) continue;
-                atomicMin(__ldcg(a.hit + i) ? &s_hit_pos : &s_miss_pos, (int)i);
+            for (uint32_t i = tid; i < a.n_pos_table0; i += blockDim.x) {       // table 0: first hit of its first token,
+                if (__ldcg(a.slots + i) < 0) continue;                           // first miss of any token
+                if (!__ldcg(a.hit + i)) atomicMin(&s_miss_pos, (int)i);
+                else if (i < a.topk) atomicMin(&s_hit_pos, (int)i);
             }
             __syncthreads();
             if (tid == 0) {
@@ -101,14 +106,14 @@ __global__ void __launch_bounds__(256) early_consumer_kernel(ConsumerArgs a)
 }  // namespace
 
 extern "C" int launch_early_consumer(const void* word, unsigned long long value, const void* ids, const void* slots,
-                                     const void* hit, uint32_t n_pos, uint32_t n_pos_table0, const void* buffer0,
+                                     const void* hit, uint32_t n_pos, uint32_t n_pos_table0, uint32_t topk, const void* buffer0,
                                      uint32_t row_bytes, void* slots_early, void* hit_early, void* hit_row,
                                      void* miss_row, void* picked, void* t_marks, void* status, void* stream)
 {
     ConsumerArgs a;
     a.word = static_cast<const unsigned long long*>(word); a.value = value;
     a.ids = static_cast<const int32_t*>(ids); a.slots = static_cast<const int32_t*>(slots);
-    a.hit = static_cast<const uint8_t*>(hit); a.n_pos = n_pos; a.n_pos_table0 = n_pos_table0;
+    a.hit = static_cast<const uint8_t*>(hit); a.n_pos = n_pos; a.n_pos_table0 = n_pos_table0; a.topk = topk;
     a.buffer0 = static_cast<const uint8_t*>(buffer0); a.row_bytes = row_bytes;
     a.slots_early = static_cast<int32_t*>(slots_early); a.hit_early = static_cast<uint8_t*>(hit_early);
     a.hit_row = static_cast<uint8_t*>(hit_row); a.miss_row = static_cast<uint8_t*>(miss_row);
