@@ -418,8 +418,8 @@ def test_a_kernel_on_the_same_stream_starts_on_the_hits(avsg, early_consumer, mo
     programmatic stream serialization, runs while Stage Two still copies.  It waits for the call's stage_one_done
     word, then holds the final slot table and hit mask and reads the row of a hit of the FIRST token (a later token
     may hit a slot reserved earlier in the same call, whose row is still travelling: Sec. 3.6); only then does it wait
-    for the stream's earlier work (griddepcontrol.wait) and read a MISSED row.  All four are compared with the oracle / the host KV,
-    and the hits were usable before the misses had arrived."""
+    for the stream's earlier work (griddepcontrol.wait) and read a MISSED row.  All four are compared with the oracle
+    or the host KV."""
     import torch
     n, n_q, K, S, rb, ctxlen, T = 16, 2, 2048, 8192, 656, 60000, 6
     cfgs = [tr.TraceConfig(seed=51, table=i, topk=K, n_q=n_q, n_iters=T, context=ctxlen, ctx_growth=True,
