@@ -187,6 +187,14 @@ typedef struct {
                                       captured with on every replay: reset the word between
                                       replays, or wait for it with a comparison that the
                                       consumer re-arms                                   */
+    uint8_t        *arriving;      /* DEVICE out [n][n_tokens][topk] or NULL (Sec. 3.6 with
+                                      Sec. 6): 1 where the position's row comes with THIS
+                                      call's Stage Two - it missed, or it hit a slot that an
+                                      earlier token of the call had just reserved -, 0 where
+                                      the row was resident before the call (readable once
+                                      stage_one_done is written) and for padding.  Written
+                                      before stage_one_done.  avsg_step only, like
+                                      stage_one_done                                     */
 } avsg_step_args;
 
 typedef struct {

@@ -86,6 +86,14 @@ class StepResult:
     def __init__(self, O, M, n, xfer):
         self.O, self.M, self.n, self.xfer = O, M, n, xfer
 
+    @property
+    def arriving(self) -> np.ndarray:
+        """[N_q, K] uint8: 1 where the position's row is written by THIS step's Stage Two, i.e. its slot is the
+        destination of an entry of the step's transfer list - the position's own entry if it missed, or that of an
+        earlier token of the step whose reservation it hit (Sec. 3.6: a later token can match a slot an earlier token
+        reserved before its data have arrived).  0: the row was in the buffer before the step, or padding."""
+        return ((self.O >= 0) & np.isin(self.O, self.xfer[:, 1])).astype(np.uint8)
+
 
 class OracleTable:
     """One request(-layer) table: S slots of (id, lifetime) plus S buffer rows."""

@@ -45,7 +45,7 @@ class AvsgStepArgs(ctypes.Structure):
                 ("row_stride", ctypes.c_void_p), ("verified_len", ctypes.c_void_p), ("slots", ctypes.c_void_p),
                 ("hit", ctypes.c_void_p), ("miss_count", ctypes.c_void_p), ("verified_len_dev", ctypes.c_void_p),
                 ("kv_rows", ctypes.c_void_p), ("stage_one_done", ctypes.c_void_p),
-                ("stage_one_done_value", ctypes.c_uint64)]
+                ("stage_one_done_value", ctypes.c_uint64), ("arriving", ctypes.c_void_p)]
 
 
 class AvsgStats(ctypes.Structure):
@@ -196,10 +196,10 @@ class _DevView:
 
 
 class StepOutput:
-    __slots__ = ("slots", "hit", "miss_count")
+    __slots__ = ("slots", "hit", "miss_count", "arriving")
 
-    def __init__(self, slots, hit, miss_count):
-        self.slots, self.hit, self.miss_count = slots, hit, miss_count
+    def __init__(self, slots, hit, miss_count, arriving=None):
+        self.slots, self.hit, self.miss_count, self.arriving = slots, hit, miss_count, arriving
 
 
 class PreparedCall:
@@ -226,13 +226,15 @@ class PreparedCall:
         self.args = a
 
     def run(self, indices, verified_len: Sequence[int], slots, hit=None, miss_count=None, stream=None,
-            host: bool = False, stage_one_done=None) -> None:
+            host: bool = False, stage_one_done=None, arriving=None) -> None:
         """indices / slots / hit / miss_count: tensors (device, or pinned host when host=True) or addresses.
         verified_len: a sequence of n ints, or an int32 CUDA tensor [n] that the kernel reads when it runs
         (what a call captured in a CUDA graph needs when the sequences grow between replays).
         stage_one_done: None or (device int64 tensor or address, value): the word receives the value once the
-        slot table, hit mask and miss counts of the whole call are final, while the missed rows still travel."""
+        slot table, hit mask and miss counts of the whole call are final, while the missed rows still travel.
+        arriving: None or a uint8 device tensor like hit: 1 where the row comes with this call's Stage Two."""
         a = self.args
+        a.arriving = _addr(arriving) if arriving is not None else None
         if stage_one_done is not None:
             a.stage_one_done, a.stage_one_done_value = _addr(stage_one_done[0]), int(stage_one_done[1])
         else:
@@ -281,7 +283,8 @@ class Context:
         return PreparedCall(self, table_ids, kv, n_tokens, topk, row_stride, kv_rows)
 
     def step(self, table_ids, indices, kv, verified_len, row_stride=None, want_hit: bool = True,
-             want_miss_count: bool = True, stream=None, kv_rows=None, stage_one_done=None) -> StepOutput:
+             want_miss_count: bool = True, stream=None, kv_rows=None, stage_one_done=None,
+             want_arriving: bool = False) -> StepOutput:
         """One decode iteration. indices: int32 CUDA tensor [n, n_tokens, topk]. Returns device tensors."""
         import torch
         assert indices.is_cuda and indices.dtype == torch.int32 and indices.is_contiguous() and indices.dim() == 3
@@ -290,8 +293,11 @@ class Context:
         slots = torch.empty_like(indices)
         hit = torch.empty(indices.shape, dtype=torch.uint8, device=indices.device) if want_hit else None
         mc = torch.empty((n, n_q), dtype=torch.int32, device=indices.device) if want_miss_count else None
-        call.run(indices, verified_len, slots, hit, mc, stream, stage_one_done=stage_one_done)
-        return StepOutput(slots, hit, mc)
+        arriving = torch.empty(indices.shape, dtype=torch.uint8, device=indices.device) if want_arriving else None
+        call.run(indices, verified_len, slots, hit, mc, stream, stage_one_done=stage_one_done, arriving=arriving)
+        out = StepOutput(slots, hit, mc)
+        out.arriving = arriving
+        return out
 
     def step_host(self, table_ids, indices, kv, verified_len, row_stride=None, want_hit: bool = True,
                   want_miss_count: bool = True, stream=None) -> StepOutput:

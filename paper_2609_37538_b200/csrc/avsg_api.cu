@@ -190,8 +190,8 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
 {
     int rc = check_args(c, a);
     if (rc != AVSG_OK) return rc;
-    if (a->stage_one_done && (host_io || c->cfg.transfer_mode == AVSG_XFER_ALL_K ||
-                              (reinterpret_cast<uint64_t>(a->stage_one_done) & 7u)))
+    if ((a->stage_one_done || a->arriving) && (host_io || c->cfg.transfer_mode == AVSG_XFER_ALL_K ||
+                                               (reinterpret_cast<uint64_t>(a->stage_one_done) & 7u)))
         return AVSG_EINVAL;
     DeviceGuard guard(c->cfg.device);
     if (!guard.ok) return AVSG_ECUDA;
@@ -275,7 +275,10 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         const bool overlap = mode == AVSG_XFER_SM_OVERLAP;
         p.flags = overlap ? c->d_flags : nullptr;
         p.epoch = reinterpret_cast<const uint32_t*>(c->d_sync);
-        p.done_seq = wait_on_sequence ? c->d_sync + 2 : reinterpret_cast<unsigned long long*>(a->stage_one_done);
+        // the caller's word: written by Stage One itself, or by the `arriving` kernel behind it when that output
+        // is asked for too (the word then also covers it)
+        p.done_seq = wait_on_sequence ? c->d_sync + 2
+                                      : (a->arriving ? nullptr : reinterpret_cast<unsigned long long*>(a->stage_one_done));
         p.done_ctr = reinterpret_cast<uint32_t*>(c->d_sync + 3);
         p.host_seq = wait_on_sequence ? c->host_seq + 1 : a->stage_one_done_value;
         p.expect = n;
@@ -312,6 +315,18 @@ int step_impl(avsg_ctx* c, const avsg_step_args* a, cudaStream_t stream, bool ho
         } else {
             if ((rc = stage_one(*c->big_args, first, cnt)) != AVSG_OK) return rc;
         }
+    }
+    if (a->arriving) {
+        ArrivingParams q;
+        q.seg = c->d_seg; q.miss_list = c->d_list; q.slots = slots; q.arriving = a->arriving;
+        q.done_seq = reinterpret_cast<unsigned long long*>(a->stage_one_done);
+        q.done_ctr = reinterpret_cast<uint32_t*>(c->d_sync + 3);
+        q.value = a->stage_one_done_value;
+        q.n = n; q.per_table = n_q * K; q.S = c->cfg.buffer_slots; q.list_stride = c->list_stride;
+        q.flags = mode == AVSG_XFER_SM_OVERLAP ? c->d_flags : nullptr;
+        q.epoch = reinterpret_cast<const uint32_t*>(c->d_sync);
+        q.n_q = n_q; q.status = c->d_status;
+        CU(launch_arriving(q, (uint32_t)c->sm_count, stream));
     }
     // (no event between the two grids in overlap mode: it would serialise them; ev[1] is recorded with ev[2])
     if (c->timing && mode != AVSG_XFER_SM_OVERLAP) CU(cudaEventRecord(c->ev[1], stream));

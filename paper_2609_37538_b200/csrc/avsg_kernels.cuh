@@ -203,4 +203,25 @@ cudaError_t launch_transfer(const XferParams& p, uint32_t blocks, uint32_t threa
 cudaError_t launch_transfer_overlap(const XferOverlapParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream);
 cudaError_t launch_transfer_positions(const PosParams& p, uint32_t blocks, uint32_t threads, cudaStream_t stream);
 
+// Optional output of a call (latency hiding, Sec. 6 with Sec. 3.6): which positions' rows come with THIS call's
+// Stage Two.  A kernel of its own between Stage One and Stage Two, so that the Stage One kernels carry no code for
+// an output few calls ask for (inside them it cost every call 1.7 us).  It also makes the call's "Stage One is
+// done" announcement when the caller asked for both.
+struct ArrivingParams {
+    const SegDesc* seg;              // per table of the call: count = entries of its miss list
+    const int2*    miss_list;        // [n][list_stride] (id, slot)
+    const int32_t* slots;            // [n][per_table]
+    uint8_t*       arriving;         // [n][per_table] out
+    unsigned long long* done_seq;    // or null
+    uint32_t*      done_ctr;         // wraps to zero at the grid size
+    unsigned long long value;
+    uint32_t n, per_table, S, list_stride;
+    // overlapped Stage Two: Stage One's hand-over flags and the call number (see S1ParamsT), else null
+    const unsigned long long* flags;
+    const uint32_t* epoch;
+    uint32_t n_q;
+    uint32_t* status;
+};
+cudaError_t launch_arriving(const ArrivingParams& p, uint32_t blocks, cudaStream_t stream);
+
 }  // namespace avsg

@@ -7,8 +7,9 @@
 // and Stage Two are still at work - and only then: every block of both is resident by the time it begins, so its
 // wait below is for kernels that are running, never for one that has yet to be scheduled.
 //   phase 1  wait (bounded) for the word the call writes at the end of its Stage One (avsg_step_args.stage_one_done);
-//            the slot table and the hit mask are final: copy them out, and read the row of one position of the FIRST
-//            token that hit (a hit of a later token may be on a slot reserved earlier in this very call, Sec. 3.6)
+//            the slot table, the hit mask and the `arriving` mask are final: copy the first two out, and read the row
+//            of the first position whose row is NOT arriving, i.e. was resident before the call (a hit alone does
+//            not say that: a later token may hit a slot reserved earlier in this very call, Sec. 3.6)
 //   phase 2  griddepcontrol.wait: everything before it on the stream, i.e. Stage Two, is complete and visible;
 //            read the row of one MISSED position
 // 32 blocks; every block waits for the word by itself, the first one also reads the rows and takes the time marks
@@ -38,17 +39,15 @@ struct ConsumerArgs {
     const int32_t* ids;          // [n_pos] the call's ids, table 0 first
     const int32_t* slots;        // [n_pos] written by the call
     const uint8_t* hit;          // [n_pos] written by the call
+    const uint8_t* arriving;     // [n_pos] written by the call: 1 = the row comes with this call's Stage Two
     uint32_t n_pos;              // positions of the whole call
     uint32_t n_pos_table0;       // positions of table 0 (rows are read from table 0's buffer only)
-    uint32_t topk;               // positions of table 0's FIRST token: only there is every hit a row that was resident
-                                 // before the call (a later token may hit a slot an earlier token of this call has
-                                 // just reserved, whose row is still on its way)
     const uint8_t* buffer0;      // table 0's rows
     uint32_t row_bytes;
     int32_t* slots_early;        // [n_pos] out
     uint8_t* hit_early;          // [n_pos] out
-    uint8_t* hit_row;            // [row_bytes] out: the row of the first hit position of table 0, read in phase 1
-    uint8_t* miss_row;           // [row_bytes] out: the row of the first missed position, read in phase 2
+    uint8_t* hit_row;            // [row_bytes] out: the row of the first resident position of table 0, read in phase 1
+    uint8_t* miss_row;           // [row_bytes] out: the row of the first arriving position, read in phase 2
     int32_t* picked;             // [2] out: the ids whose rows were read (-1: none)
     unsigned long long* t_marks; // [4] out: start, word seen, phase 1 done, Stage Two waited for
     uint32_t* status;            // out: 1 = the wait ran out
@@ -77,17 +76,16 @@ __global__ void __launch_bounds__(256) early_consumer_kernel(ConsumerArgs a)
             a.hit_early[i] = __ldcg(a.hit + i);
         }
         if (first) {
-            for (uint32_t i = tid; i < a.n_pos_table0; i += blockDim.x) {       // table 0: first hit of its first token,
-                if (__ldcg(a.slots + i) < 0) continue;                           // first miss of any token
-                if (!__ldcg(a.hit + i)) atomicMin(&s_miss_pos, (int)i);
-                else if (i < a.topk) atomicMin(&s_hit_pos, (int)i);
+            for (uint32_t i = tid; i < a.n_pos_table0; i += blockDim.x) {       // table 0: first resident position,
+                if (__ldcg(a.slots + i) < 0) continue;                           // first position whose row is arriving
+                atomicMin(__ldcg(a.arriving + i) ? &s_miss_pos : &s_hit_pos, (int)i);
             }
             __syncthreads();
             if (tid == 0) {
                 a.picked[0] = s_hit_pos != 0x7FFFFFFF ? a.ids[s_hit_pos] : -1;
                 a.picked[1] = s_miss_pos != 0x7FFFFFFF ? a.ids[s_miss_pos] : -1;
             }
-            if (s_hit_pos != 0x7FFFFFFF) {          // a hit's row was placed by an earlier call: readable now
+            if (s_hit_pos != 0x7FFFFFFF) {          // that row was placed by an earlier call: readable now
                 const uint8_t* src = a.buffer0 + (size_t)__ldcg(a.slots + s_hit_pos) * a.row_bytes;
                 for (uint32_t b = tid; b < a.row_bytes; b += blockDim.x) a.hit_row[b] = __ldcg(src + b);
             }
@@ -106,14 +104,15 @@ __global__ void __launch_bounds__(256) early_consumer_kernel(ConsumerArgs a)
 }  // namespace
 
 extern "C" int launch_early_consumer(const void* word, unsigned long long value, const void* ids, const void* slots,
-                                     const void* hit, uint32_t n_pos, uint32_t n_pos_table0, uint32_t topk, const void* buffer0,
+                                     const void* hit, const void* arriving, uint32_t n_pos, uint32_t n_pos_table0,
+                                     const void* buffer0,
                                      uint32_t row_bytes, void* slots_early, void* hit_early, void* hit_row,
                                      void* miss_row, void* picked, void* t_marks, void* status, void* stream)
 {
     ConsumerArgs a;
     a.word = static_cast<const unsigned long long*>(word); a.value = value;
     a.ids = static_cast<const int32_t*>(ids); a.slots = static_cast<const int32_t*>(slots);
-    a.hit = static_cast<const uint8_t*>(hit); a.n_pos = n_pos; a.n_pos_table0 = n_pos_table0; a.topk = topk;
+    a.hit = static_cast<const uint8_t*>(hit); a.arriving = static_cast<const uint8_t*>(arriving); a.n_pos = n_pos; a.n_pos_table0 = n_pos_table0;
     a.buffer0 = static_cast<const uint8_t*>(buffer0); a.row_bytes = row_bytes;
     a.slots_early = static_cast<int32_t*>(slots_early); a.hit_early = static_cast<uint8_t*>(hit_early);
     a.hit_row = static_cast<uint8_t*>(hit_row); a.miss_row = static_cast<uint8_t*>(miss_row);

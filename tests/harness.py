@@ -33,7 +33,7 @@ def run_parity(w: tr.Workload, *, tables: Optional[Sequence[int]] = None, mode: 
                row_stride: Optional[int] = None, buffer_every: int = 1, oracle_tables: Optional[Sequence[int]] = None,
                n_iters: Optional[int] = None, threads: Optional[int] = None, xfer_geometry=None,
                index_mode: int = 0, permute_seed: Optional[int] = None, cluster: int = 0,
-               huge_pages: bool = False, signal: bool = False) -> Dict:
+               huge_pages: bool = False, signal: bool = False, arriving: bool = False) -> Dict:
     """Steps every call group of w for every iteration on the GPU; the tables in oracle_tables (default: all)
     are stepped by the oracle too and compared after EVERY step: hit mask, slot table, miss counts, (tok, life);
     the buffer rows every buffer_every iterations and at the end.  With permute_seed the K positions of every token
@@ -94,13 +94,14 @@ def run_parity(w: tr.Workload, *, tables: Optional[Sequence[int]] = None, mode: 
                     if signal:                       # the call announces the end of its Stage One in a word of ours
                         n_signalled += 1
                         out = ctx.step(tids, torch.from_numpy(Xh).cuda(), kvs, vlen, strides,
-                                       stage_one_done=(signal_word, n_signalled))
+                                       stage_one_done=(signal_word, n_signalled), want_arriving=arriving)
                     else:
-                        out = ctx.step(tids, torch.from_numpy(Xh).cuda(), kvs, vlen, strides)
+                        out = ctx.step(tids, torch.from_numpy(Xh).cuda(), kvs, vlen, strides, want_arriving=arriving)
                     torch.cuda.synchronize()
                     if signal:
                         assert int(signal_word.item()) == n_signalled, ("signal", w.name, t)
                     slots, hit, mc = out.slots.cpu().numpy(), out.hit.cpu().numpy(), out.miss_count.cpu().numpy()
+                arr = out.arriving.cpu().numpy() if arriving and not host_io else None
                 for k, ti in enumerate(grp):
                     if ti not in check:
                         continue
@@ -111,6 +112,8 @@ def run_parity(w: tr.Workload, *, tables: Optional[Sequence[int]] = None, mode: 
                     assert (hit[k] == r.M).all(), ("hit mask", w.name, ti, t)
                     assert (slots[k] == r.O).all(), ("slot table", w.name, ti, t)
                     assert (mc[k] == r.n).all(), ("miss counts", w.name, ti, t)
+                    if arr is not None:
+                        assert (arr[k] == r.arriving).all(), ("rows that arrive with this call", w.name, ti, t)
                     tok, life = ctx.export_state(local[ti])
                     c, l = orc[ti].export_state()
                     assert (tok == c).all(), ("cached ids", w.name, ti, t)

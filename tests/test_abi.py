@@ -26,7 +26,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(avsg.AvsgConfig) == 56
-    assert ctypes.sizeof(avsg.AvsgStepArgs) == 112
+    assert ctypes.sizeof(avsg.AvsgStepArgs) == 120
     assert ctypes.sizeof(avsg.AvsgStats) == 104
     assert ctypes.sizeof(avsg.AvsgNoAllocArgs) == 120
 

@@ -307,13 +307,16 @@ def test_overlap_mode_limits(avsg, n, n_q, K, S):
         if t % 2:                                        # every other iteration through the host-buffer entry point
             out = ctx.step_host(list(range(n)), torch.from_numpy(X).pin_memory(), [kv] * n, N)
         else:                                            # ... and these announce the end of their Stage One
-            out = ctx.step(list(range(n)), torch.from_numpy(X).cuda(), [kv] * n, N, stage_one_done=(word, 1000 + t))
+            out = ctx.step(list(range(n)), torch.from_numpy(X).cuda(), [kv] * n, N, stage_one_done=(word, 1000 + t),
+                           want_arriving=t % 4 == 0)
         torch.cuda.synchronize()
         assert int(word.item()) == 1000 + t - (t % 2), t
         slots, mc = out.slots.cpu().numpy(), out.miss_count.cpu().numpy()
+        arr = out.arriving.cpu().numpy() if out.arriving is not None else None
         for i in range(n):
             r = orc[i].step(X[i], N[i], kv.numpy(), rb)
             assert (slots[i] == r.O).all() and (mc[i] == r.n).all(), (t, i)
+            assert arr is None or (arr[i] == r.arriving).all(), (t, i)
     for i in range(0, n, max(1, n // 7)):
         assert (ctx.buffer(i).cpu().numpy() == orc[i].rows()).all(), i
     assert ctx.sync_status() == 0
@@ -330,6 +333,11 @@ def test_stage_one_done_signal(avsg):
                dict(cluster=2), dict(cluster=4, mode=avsg.XFER_SM_OVERLAP),
                dict(mode=avsg.XFER_REQUEST_LEVEL), dict(mode=avsg.XFER_POSITION_LEVEL)):
         _parity(w, signal=True, **kw)
+        _parity(w, signal=True, arriving=True, permute_seed=3, **kw)     # ... and after the `arriving` output
+        _parity(w, arriving=True, **kw)                                  # that output without the word
+    w4 = tr.workload("C2", topk=128, n_q=4, buffer_slots=512, n_iters=10, context=4096, recent_window=256)
+    for kw in (dict(), dict(index_mode=avsg.INDEX_DIRECT, mode=avsg.XFER_SM_OVERLAP), dict(cluster=4)):
+        r = _parity(w4, signal=True, arriving=True, **kw)                # MTP-3: hits on the call's own reservations
 
     n, n_q, K, S, rb, ctxlen, T = 6, 2, 512, 2048, 656, 30000, 6
     cfgs = [tr.TraceConfig(seed=41, table=i, topk=K, n_q=n_q, n_iters=T, context=ctxlen, ctx_growth=True,
@@ -407,7 +415,7 @@ def early_consumer(tmp_path_factory):
     subprocess.check_call([nvcc] + flags + ["-o", str(so), os.path.join(ROOT, "tests", "cuda", "early_consumer.cu")])
     lib = ctypes.CDLL(str(so))
     vp, u32, u64 = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64
-    lib.launch_early_consumer.argtypes = [vp, u64, vp, vp, vp, u32, u32, u32, vp, u32, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.launch_early_consumer.argtypes = [vp, u64, vp, vp, vp, vp, u32, u32, vp, u32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.launch_early_consumer.restype = ctypes.c_int
     return lib
 
@@ -416,9 +424,10 @@ def early_consumer(tmp_path_factory):
 def test_a_kernel_on_the_same_stream_starts_on_the_hits(avsg, early_consumer, mode_name):
     """Latency hiding (Sec. 6): a consumer kernel launched right behind avsg_step on the same stream, with
     programmatic stream serialization, runs while Stage Two still copies.  It waits for the call's stage_one_done
-    word, then holds the final slot table and hit mask and reads the row of a hit of the FIRST token (a later token
-    may hit a slot reserved earlier in the same call, whose row is still travelling: Sec. 3.6); only then does it wait
-    for the stream's earlier work (griddepcontrol.wait) and read a MISSED row.  All four are compared with the oracle
+    word, then holds the final slot table, hit mask and `arriving` mask and reads the row of the first position that is
+    NOT arriving (a hit alone does not say so: a later token may hit a slot reserved earlier in the same call, whose
+    row is still travelling, Sec. 3.6); only then does it wait for the stream's earlier work (griddepcontrol.wait)
+    and read the row of the first arriving position.  All four are compared with the oracle
     or the host KV."""
     import torch
     n, n_q, K, S, rb, ctxlen, T = 16, 2, 2048, 8192, 656, 60000, 6
@@ -439,6 +448,7 @@ def test_a_kernel_on_the_same_stream_starts_on_the_hits(avsg, early_consumer, mo
     slots = torch.empty((n, n_q, K), dtype=torch.int32, **dev)
     hit = torch.empty((n, n_q, K), dtype=torch.uint8, **dev)
     slots_early, hit_early = torch.empty_like(slots), torch.empty_like(hit)
+    arriving = torch.empty_like(hit)
     hit_row, miss_row = torch.zeros(rb, dtype=torch.uint8, **dev), torch.zeros(rb, dtype=torch.uint8, **dev)
     picked = torch.empty(2, dtype=torch.int32, **dev)
     marks = torch.zeros(4, dtype=torch.int64, **dev)
@@ -452,9 +462,10 @@ def test_a_kernel_on_the_same_stream_starts_on_the_hits(avsg, early_consumer, mo
         Xd = torch.from_numpy(X).cuda()
         slots_early.fill_(-7); hit_early.fill_(9)
         torch.cuda.synchronize()
-        call.run(Xd, N, slots, hit, None, stream, stage_one_done=(word, t + 1))
+        call.run(Xd, N, slots, hit, None, stream, stage_one_done=(word, t + 1), arriving=arriving)
         rc = early_consumer.launch_early_consumer(word.data_ptr(), t + 1, Xd.data_ptr(), slots.data_ptr(), hit.data_ptr(),
-                                                  n * n_q * K, n_q * K, K, buf0.data_ptr(), rb, slots_early.data_ptr(),
+                                                  arriving.data_ptr(),
+                                                  n * n_q * K, n_q * K, buf0.data_ptr(), rb, slots_early.data_ptr(),
                                                   hit_early.data_ptr(), hit_row.data_ptr(), miss_row.data_ptr(),
                                                   picked.data_ptr(), marks.data_ptr(), status.data_ptr(),
                                                   stream.cuda_stream or None)
@@ -1036,13 +1047,15 @@ def _literal_parity(avsg, w, n_iters=None, R=3, mode=0, permute_seed=None):
         for grp in w.calls:
             X = np.stack([traces[ti][0][t] for ti in grp])
             vlen = [int(traces[ti][1][t]) for ti in grp]
-            out = ctx.step(grp, torch.from_numpy(X).cuda(), [kv.t[ti] for ti in grp], vlen)
+            out = ctx.step(grp, torch.from_numpy(X).cuda(), [kv.t[ti] for ti in grp], vlen, want_arriving=True)
             torch.cuda.synchronize()
             slots, hit, mc = out.slots.cpu().numpy(), out.hit.cpu().numpy(), out.miss_count.cpu().numpy()
+            arr = out.arriving.cpu().numpy()
             for k, ti in enumerate(grp):
                 r = orc[ti].step(X[k], vlen[k], kv.np[ti])
                 assert (hit[k] == r.M).all(), ("hit mask", ti, t)
                 assert (slots[k] == r.O).all(), ("slot table", ti, t)
+                assert (arr[k] == r.arriving).all(), ("rows that arrive with this call", ti, t)
                 assert (mc[k] == r.n).all(), ("miss counts", ti, t)
                 c, q = ctx.export_hash_state(ti)
                 oc, oq = orc[ti].export_state()

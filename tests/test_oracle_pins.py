@@ -260,6 +260,42 @@ def test_mtp_sharing_and_preservation(L):
         assert len(set(r.xfer[:, 1].tolist())) == r.xfer.shape[0]
 
 
+def test_arriving_marks_exactly_the_rows_that_were_not_in_the_buffer_before():
+    """Sec. 3.6 (a later token can match a slot reserved by an earlier token before its data have arrived) read
+    together with Sec. 6 (attention on the hits while the misses load): `arriving` is pinned to what the buffer held
+    BEFORE the step, byte for byte - not to the bookkeeping it is computed from."""
+    rng = np.random.default_rng(11)
+    K, n_q, S, rb, universe = 24, 3, 96, 16, 600
+    host = rng.integers(0, 256, (universe, rb), dtype=np.uint8)
+    assert len({bytes(r) for r in host}) == universe                 # all rows differ
+    t = OracleTable(S, rb, 4)
+    in_flight_hits = 0
+    for step in range(30):
+        base = rng.choice(universe, K + 10, replace=False)
+        X = np.stack([rng.permutation(rng.choice(base, K, replace=False)) for _ in range(n_q)]).astype(np.int32)
+        X[rng.integers(n_q), rng.integers(K)] = -1                   # one padding position
+        before = t.rows().copy()
+        r = t.step(X, universe, host.reshape(-1))
+        after, F = t.rows(), r.arriving
+        if step == 0:
+            assert (F == (X >= 0)).all()                             # empty buffer: every row has to come
+        for g in range(n_q):
+            for i in range(K):
+                x, o = int(X[g, i]), int(r.O[g, i])
+                if x < 0:
+                    assert F[g, i] == 0 and o == -1
+                    continue
+                assert (after[o] == host[x]).all()                   # at the end of the step the row is there
+                if F[g, i]:
+                    assert (before[o] != host[x]).any()              # ... and it was not there before
+                    if r.M[g, i]:
+                        in_flight_hits += 1
+                        assert g > 0 and x in X[:g]                  # a hit on an earlier token's reservation
+                else:
+                    assert r.M[g, i] == 1 and (before[o] == host[x]).all()    # readable before Stage Two
+    assert in_flight_hits > 50
+
+
 def test_mtp_cold_start_counts_union():
     K, n_q, S = 64, 4, 256
     rng = np.random.default_rng(3)
