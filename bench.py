@@ -942,7 +942,7 @@ def run_breakdown(args):
             ctx.close()
             # pass 3: when are the hits usable?  A second stream waits for the word the call writes at the end of
             # its Stage One (avsg_step_args.stage_one_done), not for the call's stream, and records an event
-            hits_at = []
+            hits_at, with_outputs = [], []
             try:
                 from cuda.bindings import driver as drv
             except ImportError:
@@ -954,18 +954,22 @@ def run_breakdown(args):
                 call = ctx.prepare(grp, [kv[t] for t in grp], w.n_q, w.topk)
                 side = torch.cuda.Stream()
                 word = torch.zeros(1, dtype=torch.int64, device="cuda")
+                arriving = torch.empty(X[0].shape, dtype=torch.uint8, device="cuda")
                 for t in range(w.n_iters):
                     flush.fill_(t & 0xFF)
                     torch.cuda.synchronize()
-                    e0, es = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0, e1, es = (torch.cuda.Event(enable_timing=True) for _ in range(3))
                     err, = drv.cuStreamWaitValue64(side.cuda_stream, word.data_ptr(), t + 1,
                                                    drv.CUstreamWaitValue_flags.CU_STREAM_WAIT_VALUE_EQ)
                     assert err == drv.CUresult.CUDA_SUCCESS
                     es.record(side)
-                    e0.record(); call.run(X[t], V[t], slots, None, None, stream, stage_one_done=(word, t + 1))
+                    e0.record()
+                    call.run(X[t], V[t], slots, None, None, stream, stage_one_done=(word, t + 1), arriving=arriving)
+                    e1.record()
                     torch.cuda.synchronize()
                     if t >= w.n_iters // 4:
                         hits_at.append(e0.elapsed_time(es) * 1e3)
+                        with_outputs.append(e0.elapsed_time(e1) * 1e3)
                 ctx.close()
             mean = lambda v: sum(v) / max(1, len(v))
             rows = mean(rows_per)
@@ -979,7 +983,8 @@ def run_breakdown(args):
                              "first_row": first_row - copy_start, "copy": first_done - first_row,
                              "tail": call_k - first_done},
                 "stage_one_kernel_us": mean(marks["last_stage_one_kernel_us"]), "call_kernel_us": call_k,
-                "hits_usable_us": mean(hits_at) if hits_at else None}), flush=True)
+                "hits_usable_us": mean(hits_at) if hits_at else None,
+                "event_us_per_call_with_early_outputs": mean(with_outputs) if with_outputs else None}), flush=True)
         del kv
 
 

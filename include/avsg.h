@@ -234,7 +234,10 @@ typedef struct {
  * buffer plus S state entries per request): allocates all state, every table
  * empty (id -1) and dead (lifetime -1), buffers zeroed.  *out is set only on
  * success.  Tables above 8192 slots are handled by a thread-block cluster
- * per table (stage_one_cluster). */
+ * per table (stage_one_cluster).  Every kernel of the library is loaded here,
+ * so that no later call has to wait for the device's other streams (the CUDA
+ * runtime loads a kernel when it is first used, and that may wait for every
+ * stream - forever, if one of them waits for a call's stage_one_done word). */
 int avsg_create(const avsg_config *cfg, avsg_ctx **out);
 
 /* No passage of the paper: releases everything avsg_create allocated, after

@@ -112,4 +112,11 @@ cudaError_t launch_arriving(const ArrivingParams& p, uint32_t blocks, cudaStream
     return cudaLaunchKernelEx(&cfg, avsg_arriving_kernel, p);
 }
 
+// Loads the kernel (see stage_one_prepare() on why that is not left to its first launch).
+cudaError_t arriving_prepare()
+{
+    cudaFuncAttributes fa;
+    return cudaFuncGetAttributes(&fa, reinterpret_cast<const void*>(avsg_arriving_kernel));
+}
+
 }  // namespace avsg

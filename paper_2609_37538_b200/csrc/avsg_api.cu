@@ -466,7 +466,8 @@ int avsg_create(const avsg_config* cfg, avsg_ctx** out)
     }
     // always raise the kernels' dynamic shared-memory limit to the device maximum: the attribute is
     // per function, so a context with a small table must not lower it under a context with a large one
-    if (stage_one_prepare((size_t)max_smem) != cudaSuccess || stage_one_cluster_prepare((size_t)max_smem) != cudaSuccess) {
+    if (stage_one_prepare((size_t)max_smem) != cudaSuccess || stage_one_cluster_prepare((size_t)max_smem) != cudaSuccess ||
+        transfer_prepare() != cudaSuccess || arriving_prepare() != cudaSuccess) {
         delete c; return AVSG_ECUDA;
     }
     // a cluster shape that fits on paper may still find no home on the device (blocks of one cluster share a GPC)

@@ -223,5 +223,7 @@ struct ArrivingParams {
     uint32_t* status;
 };
 cudaError_t launch_arriving(const ArrivingParams& p, uint32_t blocks, cudaStream_t stream);
+cudaError_t arriving_prepare();
+cudaError_t transfer_prepare();
 
 }  // namespace avsg

@@ -50,7 +50,7 @@ int setup_device(int dev, NoAllocScratch** out)
         if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || !ptr) { cudaGetLastError(); return AVSG_ECUDA; }
         if (cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&g_max_smem[dev], cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
-            stage_one_prepare((size_t)g_max_smem[dev]) != cudaSuccess) {
+            stage_one_prepare((size_t)g_max_smem[dev]) != cudaSuccess || transfer_prepare() != cudaSuccess) {
             cudaGetLastError();
             return AVSG_ECUDA;
         }

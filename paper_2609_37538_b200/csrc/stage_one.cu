@@ -784,6 +784,17 @@ cudaError_t stage_one_prepare(size_t max_smem)
         cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
         if (e != cudaSuccess) return e;
     }
+    // The other kernels of this file are loaded now as well: the runtime loads a kernel at its first use, which may
+    // have to wait for every stream of the device - forever, if a stream is waiting for something that very launch
+    // would produce (a caller who arms a wait for a call's stage_one_done word before its first call).
+    const void* others[] = {reinterpret_cast<const void*>(avsg_all_k_prepare_kernel),
+                            reinterpret_cast<const void*>(avsg_reset_tables_kernel),
+                            reinterpret_cast<const void*>(avsg_direct_index_from_state_kernel)};
+    for (const void* k : others) {
+        cudaFuncAttributes fa;
+        cudaError_t e = cudaFuncGetAttributes(&fa, k);
+        if (e != cudaSuccess) return e;
+    }
     return cudaSuccess;
 }
 

@@ -336,4 +336,18 @@ cudaError_t launch_transfer(const XferParams& p, uint32_t blocks, uint32_t threa
     return cudaLaunchKernelEx(&cfg, avsg_transfer_kernel, p);
 }
 
+// Loads this file's kernels (see stage_one_prepare() on why that is not left to their first launch).
+cudaError_t transfer_prepare()
+{
+    const void* kernels[] = {reinterpret_cast<const void*>(avsg_transfer_kernel),
+                             reinterpret_cast<const void*>(avsg_transfer_overlap_kernel),
+                             reinterpret_cast<const void*>(avsg_transfer_positions_kernel)};
+    for (const void* k : kernels) {
+        cudaFuncAttributes fa;
+        cudaError_t e = cudaFuncGetAttributes(&fa, k);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
 }  // namespace avsg

@@ -491,6 +491,51 @@ def test_a_kernel_on_the_same_stream_starts_on_the_hits(avsg, early_consumer, mo
     ctx.close()
 
 
+_FIRST_CALL_SCRIPT = r"""
+import sys, time
+import numpy as np, torch
+from cuda.bindings import driver as drv
+import avsg_traces as tr
+import paper_2609_37538_b200 as avsg
+mode = getattr(avsg, sys.argv[1])
+n, n_q, K, S, rb, ctxlen = 3, 2, 64, 256, 48, 3000
+kv = avsg.pinned_empty(ctxlen * rb)
+tr.fill_kv(kv.data_ptr(), 1, 0, ctxlen, rb)
+X = torch.from_numpy(np.stack([tr.generate(tr.TraceConfig(seed=1, table=i, topk=K, n_q=n_q, n_iters=1, context=ctxlen,
+                               ctx_growth=True, beta=(9, 1), p_recent=0.5, recent_window=256))[0][0] for i in range(n)])).cuda()
+ctx = avsg.Context(n, S, rb, K, n_q, 16, transfer_mode=mode, index_mode=avsg.INDEX_DIRECT, max_context=ctxlen + n_q)
+side = torch.cuda.Stream()
+word = torch.zeros(1, dtype=torch.int64, device="cuda")
+torch.cuda.synchronize()
+err, = drv.cuStreamWaitValue64(side.cuda_stream, word.data_ptr(), 1, drv.CUstreamWaitValue_flags.CU_STREAM_WAIT_VALUE_EQ)
+assert err == drv.CUresult.CUDA_SUCCESS
+released = torch.cuda.Event()
+released.record(side)
+# the process's FIRST call: none of the call's kernels has been launched before
+out = ctx.step(list(range(n)), X, [kv] * n, [ctxlen] * n, stage_one_done=(word, 1), want_arriving=sys.argv[2] == "1")
+t0 = time.time()
+while not released.query() and time.time() - t0 < 20:
+    time.sleep(0.001)
+assert released.query(), "the waiting stream was not released"
+torch.cuda.synchronize()
+assert ctx.sync_status() == 0 and int(word.item()) == 1
+print("first call ok")
+"""
+
+
+@pytest.mark.parametrize("mode_name,arriving", [("XFER_SM_OVERLAP", 1), ("XFER_SM_BALANCED", 1), ("XFER_SM_OVERLAP", 0)])
+def test_first_call_of_a_process_with_a_waiter_already_armed(mode_name, arriving):
+    """A stream that already waits for a call's stage_one_done word when the process makes its first call: the
+    library has loaded every kernel when the context was created, so no launch has to wait for the device's other
+    streams (the runtime loads a kernel at its first use, which may wait for all streams - here forever)."""
+    import subprocess
+    import sys
+    env = dict(os.environ, PYTHONPATH=ROOT + os.pathsep + os.environ.get("PYTHONPATH", ""))
+    r = subprocess.run([sys.executable, "-c", _FIRST_CALL_SCRIPT, mode_name, str(arriving)], cwd=ROOT, env=env,
+                       capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0 and "first call ok" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
+
+
 @pytest.mark.parametrize("cluster", [0, 2])
 @pytest.mark.parametrize("mode_name", ["XFER_SM_BALANCED", "XFER_SM_OVERLAP"])
 def test_a_captured_call_can_be_replayed(avsg, mode_name, cluster):
