@@ -567,11 +567,17 @@ def test_a_captured_call_can_be_replayed(avsg, mode_name, cluster):
         Nd.copy_(torch.tensor([int(traces[i][1][t]) for i in range(n)], dtype=torch.int32))
         torch.cuda.synchronize()
 
+    word = torch.zeros(1, dtype=torch.int64, device="cuda")
+    arriving = torch.empty((n, n_q, K), dtype=torch.uint8, device="cuda")
+
     def check(t):
         torch.cuda.synchronize()
+        assert int(word.item()) == 5                       # the captured value, written again by every replay
+        word.zero_()
         for i in range(n):
             r = orc[i].step(traces[i][0][t], int(traces[i][1][t]), kv[i].numpy(), rb)
             assert (slots[i].cpu().numpy() == r.O).all() and (mc[i].cpu().numpy() == r.n).all(), (t, i)
+            assert (arriving[i].cpu().numpy() == r.arriving).all(), (t, i)
             assert (ctx.buffer(i).cpu().numpy() == orc[i].rows()).all(), (t, i)
             tok, life = ctx.export_state(i)
             c, l = orc[i].export_state()
@@ -580,11 +586,12 @@ def test_a_captured_call_can_be_replayed(avsg, mode_name, cluster):
     side = torch.cuda.Stream()
     load(0)
     with torch.cuda.stream(side):
-        call.run(X, Nd, slots, None, mc, side)             # eager first call: resolves and caches the host pointers
+        call.run(X, Nd, slots, None, mc, side,             # eager first call: resolves and caches the host pointers
+                 stage_one_done=(word, 5), arriving=arriving)
     check(0)
     graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph, stream=side):
-        call.run(X, Nd, slots, None, mc, torch.cuda.current_stream())
+    with torch.cuda.graph(graph, stream=side):             # three kernels: Stage One, the `arriving` output, Stage Two
+        call.run(X, Nd, slots, None, mc, torch.cuda.current_stream(), stage_one_done=(word, 5), arriving=arriving)
     for t in range(1, T):
         load(t)
         graph.replay()
